@@ -1,0 +1,307 @@
+"""CPU oracle for the POP pruned-prefill path.  TEST INFRASTRUCTURE, not product code.
+
+A plain, slow, step-by-step statement of what the path computes, in plain PyTorch
+CPU ops (fp64 by default), written from the paper's definitions:
+
+  * decoder layer         y_l = x_l + Attn(x_l, K, V);  x_{l+1} = y_l + FFN(y_l)      (Sec. 2.1, Eq. 1)
+  * KV generation         k = RoPE(LN(x_l) W^K),  v = LN(x_l) W^V                     (Eq. 2)
+  * KV append             K_cur = Concat(K_past, k), attention uses the updated cache (Eq. 3)
+  * pruned layer          k_l, v_l from the layer's own LN / W^K / W^V on x_l (Eq. 14);
+                          hidden state passed on unchanged (Eq. 15 = Eq. 4)
+  * boundary handling     pruned prefill covers x_{1:N-1}; x_N is the first decode step
+                          of the full model                                        (Sec. 3.3)
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+module. It shares no code with the CUDA library and never imports it. Weights and
+inputs are handed in by the caller (a provider with ``get(name, layer)``).
+
+Readings taken where the paper is silent (each also listed in the design notes):
+RMSNorm with fp statistics over the feature axis; rotate-half RoPE pairing
+(j, j + hd/2) with angle pos * theta^(-2j/hd), 0-based positions; per-head QK
+RMSNorm (when the model has it) between projection and RoPE; softmax scale
+1/sqrt(hd); sliding window of W keys including the query's own position; query
+head h uses KV head floor(h * n_kv / n_q); tanh-approximated GELU for the
+GELU-gated FFN; logits for the last prompt position only.
+
+``precision="exact"`` evaluates everything in ``dtype``.  ``precision="bf16ops"``
+additionally rounds intermediate tensors to bf16 at the points where a bf16
+tensor-core pipeline stores or feeds them (GEMM operands, q/k/v, softmax
+probabilities entering P.V, attention output, gated activation); it exists so
+that integer decisions (the argmax token) can be compared in the kernel's
+precision.  The residual stream, norm statistics, softmax and all accumulations
+stay in ``dtype`` in both modes.
+
+Pins (tests/test_oracle_*.py): closed forms and invariants of each primitive, an
+independent brute-force single-sequence evaluator with explicit N x N score
+matrices and no cache, prefix-recomputation (causality), the structural
+identities of POP (L_keep = L and L_keep = L-1 reproduce the full prefill; kept
+layers and the first pruned layer have the full model's KV; deeper pruned layers
+equal a separate three-line evaluation of Eq. 14), and fault-injection checks
+that a planted mistake fails them.  The accuracy effect of pruning on trained
+models (the paper's Tables 1, 3, 4) is parity unpinned: it needs trained weights
+and public datasets that are not available to this repository.
+"""
+from __future__ import annotations
+
+import math
+from typing import Optional
+
+import torch
+
+
+# ---------------------------------------------------------------------------------------
+# primitives
+# ---------------------------------------------------------------------------------------
+
+def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
+    """Round to bf16 and back in "bf16ops" mode; identity in "exact" mode."""
+    if precision == "exact":
+        return x
+    return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
+
+
+def rmsnorm(x: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
+    """LN(.) of Eq. 2 for the RMSNorm models evaluated in Sec. 4: x * g / sqrt(mean(x^2) + eps)."""
+    ms = x.pow(2).mean(dim=-1, keepdim=True)
+    return x / torch.sqrt(ms + eps) * gain
+
+
+def rope(x: torch.Tensor, positions: torch.Tensor, theta: float) -> torch.Tensor:
+    """RoPE(.) of Eq. 2. x: [..., T, heads, hd]; positions: [T] (0-based).
+    Pair (j, j + hd/2) is rotated by the angle pos * theta^(-2j/hd)."""
+    hd = x.shape[-1]
+    half = hd // 2
+    j = torch.arange(half, dtype=torch.float64)
+    inv_freq = torch.pow(torch.tensor(float(theta), dtype=torch.float64), -2.0 * j / hd)
+    ang = positions.to(torch.float64)[:, None] * inv_freq[None, :]          # [T, half]
+    cos = torch.cos(ang).to(x.dtype)[:, None, :]
+    sin = torch.sin(ang).to(x.dtype)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1)
+
+
+def gated_act(gate: torch.Tensor, up: torch.Tensor, act: int) -> torch.Tensor:
+    """act(gate) * up: SiLU (act=0) or tanh-approximated GELU (act=1)."""
+    if act == 0:
+        a = gate * torch.sigmoid(gate)
+    else:
+        a = 0.5 * gate * (1.0 + torch.tanh(math.sqrt(2.0 / math.pi) * (gate + 0.044715 * gate.pow(3))))
+    return a * up
+
+
+def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, q_pos: torch.Tensor,
+              window: int, precision: str = "exact") -> torch.Tensor:
+    """Attn of Eq. 1 for one sequence. q: [T, n_q, hd] at absolute positions q_pos [T];
+    k, v: [S, n_kv, hd] holding cache positions 0..S-1. Query at position i sees keys
+    j <= i, and j > i - window when window > 0. Returns [T, n_q, hd]."""
+    T, n_q, hd = q.shape
+    S, n_kv, _ = k.shape
+    out = torch.empty_like(q)
+    kpos = torch.arange(S)
+    allowed = kpos[None, :] <= q_pos[:, None]
+    if window > 0:
+        allowed &= kpos[None, :] > (q_pos[:, None] - window)
+    scale = 1.0 / math.sqrt(hd)
+    for h in range(n_q):
+        g = (h * n_kv) // n_q
+        s = (q[:, h, :] @ k[:, g, :].T) * scale
+        s = s.masked_fill(~allowed, float("-inf"))
+        p = torch.exp(s - s.max(dim=-1, keepdim=True).values)
+        denom = p.sum(dim=-1, keepdim=True)
+        out[:, h, :] = (_rnd(p, precision) @ v[:, g, :]) / denom
+    return out
+
+
+# ---------------------------------------------------------------------------------------
+# model pieces
+# ---------------------------------------------------------------------------------------
+
+def _w(weights, name, layer, dtype):
+    return weights.get(name, layer).to(dtype)
+
+
+def embed(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], dtype) -> torch.Tensor:
+    """x_1 for one sequence: tokens int [N] (a negative id means "take the row of
+    `embeds`"), embeds [N, d] or None."""
+    N = tokens.shape[0]
+    x = torch.empty(N, cfg.d_model, dtype=dtype)
+    is_tok = tokens >= 0
+    if is_tok.any():
+        if hasattr(weights, "embedding_rows"):
+            rows = weights.embedding_rows(tokens[is_tok])
+        else:
+            rows = weights.get("embed", 0)[tokens[is_tok].long()]
+        x[is_tok] = rows.to(dtype)
+    if (~is_tok).any():
+        x[~is_tok] = embeds[~is_tok].to(dtype)
+    return x
+
+
+def kv_generation(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Tensor,
+                  dtype, precision: str):
+    """Eq. 2 (and, applied to a pruned layer's input, Eq. 14): the layer's own input norm,
+    K/V projections, optional per-head K norm, RoPE on k. x: [T, d] -> k, v [T, n_kv, hd]."""
+    h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
+    k = (h @ _w(weights, "wk", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+    v = (h @ _w(weights, "wv", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+    if cfg.qk_norm:
+        k = rmsnorm(k, _w(weights, "k_norm", layer, dtype), cfg.rms_eps)
+    k = rope(k, positions, cfg.rope_theta)
+    return _rnd(k, precision), _rnd(v, precision)
+
+
+def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Tensor,
+                  k_past: Optional[torch.Tensor], v_past: Optional[torch.Tensor],
+                  dtype, precision: str):
+    """One full decoder layer (Eq. 1-3) on the T new positions `positions` of one sequence,
+    given the cache of earlier positions. Returns x_{l+1} [T, d], K_cur, V_cur."""
+    k_new, v_new = kv_generation(cfg, weights, layer, x, positions, dtype, precision)
+    if k_past is not None and k_past.shape[0] > 0:
+        k_cur = torch.cat([k_past, k_new], dim=0)                       # Eq. 3
+        v_cur = torch.cat([v_past, v_new], dim=0)
+    else:
+        k_cur, v_cur = k_new, v_new
+    h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
+    q = (h @ _w(weights, "wq", layer, dtype).T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
+    if cfg.qk_norm:
+        q = rmsnorm(q, _w(weights, "q_norm", layer, dtype), cfg.rms_eps)
+    q = _rnd(rope(q, positions, cfg.rope_theta), precision)
+    a = attention(q, k_cur, v_cur, positions, cfg.layer_window(layer), precision)
+    a = _rnd(a.reshape(-1, cfg.q_dim), precision)
+    o = a @ _w(weights, "wo", layer, dtype).T
+    if cfg.post_norms:
+        o = rmsnorm(o, _w(weights, "post_attn_norm", layer, dtype), cfg.rms_eps)
+    y = x + o                                                           # Eq. 1, first line
+    h2 = _rnd(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps), precision)
+    gate = h2 @ _w(weights, "w_gate", layer, dtype).T
+    up = h2 @ _w(weights, "w_up", layer, dtype).T
+    f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w(weights, "w_down", layer, dtype).T
+    if cfg.post_norms:
+        f = rmsnorm(f, _w(weights, "post_ffn_norm", layer, dtype), cfg.rms_eps)
+    return y + f, k_cur, v_cur                                          # Eq. 1, second line
+
+
+def lm_logits(cfg, weights, x_last: torch.Tensor, dtype) -> torch.Tensor:
+    """Final norm and output head on one position: [d] -> [vocab]."""
+    h = rmsnorm(x_last, _w(weights, "final_norm", 0, dtype), cfg.rms_eps)
+    V = cfg.vocab
+    out = torch.empty(V, dtype=dtype)
+    step = 16384
+    for r0 in range(0, V, step):
+        r1 = min(V, r0 + step)
+        if hasattr(weights, "rows"):
+            w = weights.rows("lm_head", 0, r0, r1 - r0).to(dtype)
+        else:
+            w = weights.get("lm_head", 0)[r0:r1].to(dtype)
+        out[r0:r1] = w @ h
+    return out
+
+
+# ---------------------------------------------------------------------------------------
+# the two prefill procedures
+# ---------------------------------------------------------------------------------------
+
+def full_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor] = None,
+                 dtype=torch.float64, precision: str = "exact", n_layers: Optional[int] = None):
+    """Standard prefill of the unpruned model over x_{1:N} (Sec. 3.3, "standard inference
+    pipeline"). tokens: int [B, N]; embeds: [B, N, d] or None.
+
+    Returns dict: K, V lists over layers of [B, N, n_kv, hd]; logits [B, vocab];
+    hidden [B, N, d] = the state leaving the last evaluated layer."""
+    L = cfg.n_layers if n_layers is None else n_layers
+    B, N = tokens.shape
+    K = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    V = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    hidden = torch.empty(B, N, cfg.d_model, dtype=dtype)
+    logits = torch.empty(B, cfg.vocab, dtype=dtype)
+    pos = torch.arange(N)
+    for b in range(B):
+        x = embed(cfg, weights, tokens[b], None if embeds is None else embeds[b], dtype)
+        for l in range(1, L + 1):
+            x, K[l - 1][b], V[l - 1][b] = layer_forward(cfg, weights, l, x, pos, None, None,
+                                                        dtype, precision)
+        hidden[b] = x
+        logits[b] = lm_logits(cfg, weights, x[N - 1], dtype)
+    return {"K": K, "V": V, "logits": logits, "hidden": hidden}
+
+
+def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], l_keep: int,
+                dtype=torch.float64, precision: str = "exact"):
+    """POP inference up to the first generated token, in the paper's two phases (Sec. 3.3).
+
+    Phase 1, pruned prefill on x_{1:N-1}: layers 1..L_keep run in full; each layer
+    l > L_keep only stores k_l, v_l computed from its own norm and projections on the state
+    it receives (Eq. 14) and passes that state on unchanged (Eq. 15), so all pruned layers
+    of the deep suffix see H = x_{L_keep+1}.
+
+    Phase 2, first decode step on x_N: one position through all L layers, each appending
+    its k, v to the cache (Eq. 2-3) and attending over positions 1..N.
+
+    Returns dict: K, V (N entries for every layer), logits [B, vocab],
+    H [B, N-1, d] (the state leaving the kept stack in phase 1)."""
+    L = cfg.n_layers
+    assert 1 <= l_keep <= L
+    B, N = tokens.shape
+    K = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    V = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    H = torch.empty(B, max(N - 1, 0), cfg.d_model, dtype=dtype)
+    logits = torch.empty(B, cfg.vocab, dtype=dtype)
+    for b in range(B):
+        x_all = embed(cfg, weights, tokens[b], None if embeds is None else embeds[b], dtype)
+        kc = [None] * L
+        vc = [None] * L
+        # ---- phase 1: pruned prefill on positions 0..N-2
+        if N > 1:
+            pos = torch.arange(N - 1)
+            x = x_all[: N - 1]
+            for l in range(1, L + 1):
+                if l <= l_keep:
+                    x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, pos, None, None,
+                                                            dtype, precision)
+                else:
+                    kc[l - 1], vc[l - 1] = kv_generation(cfg, weights, l, x, pos, dtype, precision)
+                    # Eq. 15: x is handed to layer l+1 unchanged
+            H[b] = x
+        # ---- phase 2: x_N as the first decode step of the full model
+        posN = torch.tensor([N - 1])
+        x = x_all[N - 1: N]
+        for l in range(1, L + 1):
+            x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1],
+                                                    dtype, precision)
+        for l in range(L):
+            K[l][b], V[l][b] = kc[l], vc[l]
+        logits[b] = lm_logits(cfg, weights, x[0], dtype)
+    return {"K": K, "V": V, "logits": logits, "H": H}
+
+
+# ---------------------------------------------------------------------------------------
+# cost model (counts of the work the method defines; no arithmetic of the method)
+# ---------------------------------------------------------------------------------------
+
+def layer_params(cfg) -> int:
+    return cfg.d_model * (cfg.q_dim + 2 * cfg.kv_dim) + cfg.q_dim * cfg.d_model + 3 * cfg.d_model * cfg.d_ffn
+
+
+def kv_param_share(cfg) -> float:
+    """Share of a layer's matrix parameters held by W^K and W^V (compare Sec. 3.3's "<5%")."""
+    return 2 * cfg.kv_dim * cfg.d_model / layer_params(cfg)
+
+
+def attention_pairs(n: int, window: int) -> int:
+    if window <= 0 or window >= n:
+        return n * (n + 1) // 2
+    return window * (window + 1) // 2 + (n - window) * window
+
+
+def prefill_flops(cfg, batch: int, n: int, l_keep: Optional[int]) -> float:
+    """Algorithmic FLOPs: full layers on n positions (GEMMs + unmasked attention pairs) and,
+    when l_keep < L, the K/V projections of pruned layers on n-1 positions. The boundary
+    token's deep-layer pass and the head are bandwidth terms and are not counted."""
+    L = cfg.n_layers
+    lk = L if l_keep is None else l_keep
+    total = 0.0
+    for l in range(1, lk + 1):
+        total += 2.0 * n * batch * layer_params(cfg)
+        total += 4.0 * cfg.q_dim * batch * attention_pairs(n, cfg.layer_window(l))
+    total += (L - lk) * 2.0 * (n - 1) * batch * cfg.d_model * 2 * cfg.kv_dim
+    return total

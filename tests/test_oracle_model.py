@@ -1,0 +1,404 @@
+"""Pins for the oracle's two prefill procedures.
+
+* an independent brute-force evaluator (pure Python / numpy loops, explicit N x N score
+  matrix, no cache, every position recomputed from its prefix) on tiny shapes;
+* third-party decoder implementations (transformers' Llama and Qwen3 modules) loaded with
+  the same synthetic weights, as a library routine the textbook model reduces to;
+* the structural identities that the paper's definitions of POP imply (Sec. 2.2, 3.3);
+* planted mistakes in the oracle that these pins must catch.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import pop_synth as ps
+from oracle import pop_oracle as po
+
+D = torch.float64
+
+TINY = ps.ModelConfig("pin", 3, 16, 4, 2, 4, 24, 40, 1e-5, 100.0, distinct_gains=True, weight_std=0.3)
+VARIANTS = {
+    "llama": TINY,
+    "qknorm": TINY.replace(qk_norm=1),
+    "gemma": TINY.replace(n_layers=4, act=1, post_norms=1, window=3, global_every=2, head_dim=8),
+}
+
+
+class DictWeights:
+    def __init__(self, cfg, seed=11):
+        sw = ps.SynthWeights(cfg, seed)
+        self.t = {}
+        for l in range(1, cfg.n_layers + 1):
+            for name in ps.layer_tensor_shapes(cfg):
+                self.t[(name, l)] = sw.get(name, l)
+        for name in ps.global_tensor_shapes(cfg):
+            self.t[(name, 0)] = sw.get(name, 0)
+
+    def get(self, name, layer=0):
+        return self.t[(name, layer)]
+
+
+# ------------------------------------------------------------------ brute force (numpy, loops)
+
+def _np(w, name, l):
+    return w.get(name, l).double().numpy()
+
+
+def _bf_norm(x, g, eps):
+    return [x[i] * g[i] / math.sqrt(sum(v * v for v in x) / len(x) + eps) for i in range(len(x))]
+
+
+def _bf_rope(vec, pos, theta):
+    hd = len(vec)
+    out = list(vec)
+    for j in range(hd // 2):
+        a = pos * theta ** (-2.0 * j / hd)
+        out[j] = vec[j] * math.cos(a) - vec[j + hd // 2] * math.sin(a)
+        out[j + hd // 2] = vec[j + hd // 2] * math.cos(a) + vec[j] * math.sin(a)
+    return out
+
+
+def brute_force_layer(cfg, w, l, X):
+    """One decoder layer over all rows of X (list of N vectors), returning the new X and the
+    K, V of every position, through an explicit N x N masked score matrix."""
+    N = len(X)
+    hd, nq, nkv = cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads
+    Wq, Wk, Wv, Wo = (_np(w, n, l) for n in ("wq", "wk", "wv", "wo"))
+    Q, K, V = [], [], []
+    for i in range(N):
+        h = np.array(_bf_norm(list(X[i]), _np(w, "ln_in", l), cfg.rms_eps))
+        q, k, v = Wq @ h, Wk @ h, Wv @ h
+        qh, kh = [], []
+        for a in range(nq):
+            t = list(q[a * hd:(a + 1) * hd])
+            if cfg.qk_norm:
+                t = _bf_norm(t, _np(w, "q_norm", l), cfg.rms_eps)
+            qh.append(_bf_rope(t, i, cfg.rope_theta))
+        for a in range(nkv):
+            t = list(k[a * hd:(a + 1) * hd])
+            if cfg.qk_norm:
+                t = _bf_norm(t, _np(w, "k_norm", l), cfg.rms_eps)
+            kh.append(_bf_rope(t, i, cfg.rope_theta))
+        Q.append(qh)
+        K.append(kh)
+        V.append([list(v[a * hd:(a + 1) * hd]) for a in range(nkv)])
+    win = cfg.layer_window(l)
+    newX = []
+    for i in range(N):
+        att = []
+        for a in range(nq):
+            g = a * nkv // nq
+            scores = np.full(N, -np.inf)
+            for j in range(N):
+                if j <= i and (win <= 0 or j > i - win):
+                    scores[j] = sum(Q[i][a][c] * K[j][g][c] for c in range(hd)) / math.sqrt(hd)
+            p = np.exp(scores - scores.max())
+            p /= p.sum()
+            att += [sum(p[j] * V[j][g][c] for j in range(N)) for c in range(hd)]
+        o = Wo @ np.array(att)
+        if cfg.post_norms:
+            o = np.array(_bf_norm(list(o), _np(w, "post_attn_norm", l), cfg.rms_eps))
+        y = np.array(X[i]) + o
+        h2 = np.array(_bf_norm(list(y), _np(w, "ln_ffn", l), cfg.rms_eps))
+        gate, up = _np(w, "w_gate", l) @ h2, _np(w, "w_up", l) @ h2
+        if cfg.act == 0:
+            a_ = gate / (1 + np.exp(-gate))
+        else:
+            a_ = 0.5 * gate * (1 + np.tanh(math.sqrt(2 / math.pi) * (gate + 0.044715 * gate ** 3)))
+        f = _np(w, "w_down", l) @ (a_ * up)
+        if cfg.post_norms:
+            f = np.array(_bf_norm(list(f), _np(w, "post_ffn_norm", l), cfg.rms_eps))
+        newX.append(y + f)
+    return newX, np.array(K), np.array(V)
+
+
+def brute_force_full(cfg, w, tokens):
+    emb = _np(w, "embed", 0)
+    X = [emb[t] for t in tokens]
+    Ks, Vs = [], []
+    for l in range(1, cfg.n_layers + 1):
+        X, K, V = brute_force_layer(cfg, w, l, X)
+        Ks.append(K)
+        Vs.append(V)
+    h = np.array(_bf_norm(list(X[-1]), _np(w, "final_norm", 0), cfg.rms_eps))
+    return Ks, Vs, _np(w, "lm_head", 0) @ h
+
+
+@pytest.mark.parametrize("variant", list(VARIANTS))
+def test_full_prefill_matches_brute_force(variant):
+    cfg = VARIANTS[variant]
+    w = DictWeights(cfg)
+    tokens = ps.uniform_tokens(3, 1, 6, cfg.vocab)
+    out = po.full_prefill(cfg, w, tokens)
+    Ks, Vs, logits = brute_force_full(cfg, w, tokens[0].tolist())
+    for l in range(cfg.n_layers):
+        assert np.allclose(out["K"][l][0].numpy(), Ks[l], atol=1e-10)
+        assert np.allclose(out["V"][l][0].numpy(), Vs[l], atol=1e-10)
+    assert np.allclose(out["logits"][0].numpy(), logits, atol=1e-10)
+
+
+def test_full_prefill_is_causal_prefix_recomputation():
+    cfg = VARIANTS["gemma"]
+    w = DictWeights(cfg)
+    tokens = ps.uniform_tokens(4, 1, 7, cfg.vocab)
+    out = po.full_prefill(cfg, w, tokens)
+    for n in (1, 4):
+        pre = po.full_prefill(cfg, w, tokens[:, :n])
+        for l in range(cfg.n_layers):
+            assert torch.allclose(pre["K"][l][0], out["K"][l][0, :n], atol=1e-12)
+            assert torch.allclose(pre["V"][l][0], out["V"][l][0, :n], atol=1e-12)
+
+
+def test_batch_rows_are_independent_sequences():
+    cfg = VARIANTS["llama"]
+    w = DictWeights(cfg)
+    tokens = ps.uniform_tokens(5, 2, 5, cfg.vocab)
+    both = po.pop_prefill(cfg, w, tokens, None, 2)
+    one = po.pop_prefill(cfg, w, tokens[1:], None, 2)
+    assert torch.allclose(both["logits"][1], one["logits"][0], atol=1e-12)
+    assert torch.allclose(both["K"][2][1], one["K"][2][0], atol=1e-12)
+
+
+# ------------------------------------------------------------------ third-party decoders
+
+def _load_hf(model, cfg, w):
+    sd = {}
+    pre = "model."
+    sd[pre + "embed_tokens.weight"] = w.get("embed").double()
+    sd[pre + "norm.weight"] = w.get("final_norm").double()
+    sd["lm_head.weight"] = w.get("lm_head").double()
+    names = {"wq": "self_attn.q_proj", "wk": "self_attn.k_proj", "wv": "self_attn.v_proj",
+             "wo": "self_attn.o_proj", "w_gate": "mlp.gate_proj", "w_up": "mlp.up_proj",
+             "w_down": "mlp.down_proj", "ln_in": "input_layernorm", "ln_ffn": "post_attention_layernorm",
+             "q_norm": "self_attn.q_norm", "k_norm": "self_attn.k_norm"}
+    for l in range(1, cfg.n_layers + 1):
+        for n in ps.layer_tensor_shapes(cfg):
+            sd[f"{pre}layers.{l-1}.{names[n]}.weight"] = w.get(n, l).double()
+    missing, unexpected = model.load_state_dict(sd, strict=False)
+    assert not unexpected and all("rotary" in m or "inv_freq" in m for m in missing), (missing, unexpected)
+
+
+@pytest.mark.parametrize("family", ["llama", "qwen3"])
+def test_full_prefill_matches_third_party_decoder(family):
+    tr = pytest.importorskip("transformers")
+    cfg = ps.ModelConfig("hf", 3, 32, 4, 2, 8, 48, 64, 1e-5, 10000.0, distinct_gains=True,
+                         weight_std=0.2, qk_norm=1 if family == "qwen3" else 0)
+    w = DictWeights(cfg)
+    kw = dict(vocab_size=cfg.vocab, hidden_size=cfg.d_model, intermediate_size=cfg.d_ffn,
+              num_hidden_layers=cfg.n_layers, num_attention_heads=cfg.n_q_heads,
+              num_key_value_heads=cfg.n_kv_heads, head_dim=cfg.head_dim, rms_norm_eps=cfg.rms_eps,
+              rope_theta=cfg.rope_theta, max_position_embeddings=64, tie_word_embeddings=False,
+              attention_bias=False, hidden_act="silu", attn_implementation="eager")
+    try:
+        if family == "llama":
+            hf_cfg = tr.LlamaConfig(mlp_bias=False, **kw)
+            model = tr.LlamaForCausalLM(hf_cfg)
+        else:
+            hf_cfg = tr.Qwen3Config(use_sliding_window=False, **kw)
+            model = tr.Qwen3ForCausalLM(hf_cfg)
+    except Exception as e:  # library API drift: the other pins still hold
+        pytest.skip(f"cannot build the third-party model: {e}")
+    model = model.double().eval()
+    _load_hf(model, cfg, w)
+    tokens = ps.uniform_tokens(6, 2, 9, cfg.vocab)
+    with torch.no_grad():
+        ref = model(input_ids=tokens.long(), use_cache=True)
+    out = po.full_prefill(cfg, w, tokens)
+    # the library keeps its rotary tables in fp32, hence 1e-5 and not round-off of fp64
+    assert torch.allclose(out["logits"], ref.logits[:, -1].double(), atol=1e-5)
+    pkv = ref.past_key_values
+    for l in range(cfg.n_layers):
+        try:
+            k_ref, v_ref = pkv.layers[l].keys, pkv.layers[l].values
+        except AttributeError:
+            k_ref, v_ref = pkv[l][0], pkv[l][1]
+        assert torch.allclose(out["K"][l], k_ref.transpose(1, 2).double(), atol=1e-5)
+        assert torch.allclose(out["V"][l], v_ref.transpose(1, 2).double(), atol=1e-5)
+
+
+# ------------------------------------------------------------------ POP structure
+
+def _setup(variant="gemma", n=8, batch=1, seed=9):
+    cfg = VARIANTS[variant]
+    w = DictWeights(cfg)
+    tokens = ps.uniform_tokens(seed, batch, n, cfg.vocab)
+    return cfg, w, tokens
+
+
+def _maxdiff(a, b):
+    return (a - b).abs().max().item()
+
+
+@pytest.mark.parametrize("variant", list(VARIANTS))
+def test_keeping_all_layers_is_the_full_prefill(variant):
+    cfg, w, tokens = _setup(variant)
+    full = po.full_prefill(cfg, w, tokens)
+    pop = po.pop_prefill(cfg, w, tokens, None, cfg.n_layers)
+    assert _maxdiff(full["logits"], pop["logits"]) < 1e-11
+    for l in range(cfg.n_layers):
+        assert _maxdiff(full["K"][l], pop["K"][l]) < 1e-11
+        assert _maxdiff(full["V"][l], pop["V"][l]) < 1e-11
+
+
+@pytest.mark.parametrize("variant", list(VARIANTS))
+def test_pruning_only_the_last_layer_changes_nothing(variant):
+    # the single pruned layer receives the exact x_L, so Eq. 14 equals Eq. 2 there, and the
+    # boundary token runs the whole stack: cache and logits equal the full model's
+    cfg, w, tokens = _setup(variant)
+    full = po.full_prefill(cfg, w, tokens)
+    pop = po.pop_prefill(cfg, w, tokens, None, cfg.n_layers - 1)
+    assert _maxdiff(full["logits"], pop["logits"]) < 1e-11
+    for l in range(cfg.n_layers):
+        assert _maxdiff(full["K"][l], pop["K"][l]) < 1e-11
+        assert _maxdiff(full["V"][l], pop["V"][l]) < 1e-11
+
+
+def test_kept_layers_and_first_pruned_layer_have_the_full_models_cache():
+    cfg, w, tokens = _setup("gemma")
+    L = cfg.n_layers
+    full = po.full_prefill(cfg, w, tokens)
+    for l_keep in (1, 2):
+        pop = po.pop_prefill(cfg, w, tokens, None, l_keep)
+        for l in range(l_keep + 1):            # layers 1..L_keep and layer L_keep+1
+            assert _maxdiff(full["K"][l], pop["K"][l]) < 1e-11
+            assert _maxdiff(full["V"][l], pop["V"][l]) < 1e-11
+        # deeper layers hold an approximation: they must differ from the full model's ...
+        assert _maxdiff(full["K"][L - 1][:, :-1], pop["K"][L - 1][:, :-1]) > 1e-3
+        # ... and so does the first token's distribution
+        assert _maxdiff(full["logits"], pop["logits"]) > 1e-4
+
+
+def test_pruned_layers_hold_eq14_of_the_kept_stacks_output():
+    cfg, w, tokens = _setup("qknorm", n=7)
+    l_keep = 1
+    pop = po.pop_prefill(cfg, w, tokens, None, l_keep)
+    N = tokens.shape[1]
+    # H = x_{L_keep+1} on positions 0..N-2, from an independent run of the kept stack alone
+    H = po.full_prefill(cfg, w, tokens[:, : N - 1], n_layers=l_keep)["hidden"][0]
+    assert _maxdiff(H, pop["H"][0]) < 1e-12
+    for l in range(l_keep + 1, cfg.n_layers + 1):
+        g = w.get("ln_in", l).double()
+        h = H * g / torch.sqrt(H.pow(2).mean(-1, keepdim=True) + cfg.rms_eps)
+        k = (h @ w.get("wk", l).double().T).reshape(N - 1, cfg.n_kv_heads, cfg.head_dim)
+        v = (h @ w.get("wv", l).double().T).reshape(N - 1, cfg.n_kv_heads, cfg.head_dim)
+        gk = w.get("k_norm", l).double()
+        k = k * gk / torch.sqrt(k.pow(2).mean(-1, keepdim=True) + cfg.rms_eps)
+        # rotate with complex arithmetic instead of the oracle's rotate-half code
+        half = cfg.head_dim // 2
+        ang = torch.arange(N - 1, dtype=D)[:, None] * cfg.rope_theta ** (-2.0 * torch.arange(half, dtype=D) / cfg.head_dim)
+        z = torch.complex(k[..., :half], k[..., half:]) * torch.polar(torch.ones_like(ang), ang)[:, None, :]
+        k = torch.cat([z.real, z.imag], dim=-1)
+        assert _maxdiff(pop["K"][l - 1][0, : N - 1], k) < 1e-11
+        assert _maxdiff(pop["V"][l - 1][0, : N - 1], v) < 1e-11
+
+
+def test_boundary_entry_of_deep_layers_comes_from_the_full_stack_state():
+    # the last prompt position is a decode step of the full model (Sec. 3.3): its deep-layer
+    # k, v come from the state that position really has there, not from H
+    cfg, w, tokens = _setup("llama", n=6)
+    pop = po.pop_prefill(cfg, w, tokens, None, 1)
+    N = tokens.shape[1]
+    l = cfg.n_layers
+    H_all = po.full_prefill(cfg, w, tokens, n_layers=1)["hidden"][0]
+    k_from_H, _ = po.kv_generation(cfg, w, l, H_all[N - 1:], torch.tensor([N - 1]), D, "exact")
+    assert _maxdiff(pop["K"][l - 1][0, N - 1:], k_from_H) > 1e-4
+
+
+def test_two_phase_boundary_equals_running_the_kept_stack_on_all_positions():
+    # causality: in layers <= L_keep position N-1 depends on exact states only, so "prefill
+    # N-1 then decode one" and "prefill N through the kept stack" agree
+    cfg, w, tokens = _setup("gemma", n=9)
+    l_keep = 2
+    pop = po.pop_prefill(cfg, w, tokens, None, l_keep)
+    fused = po.full_prefill(cfg, w, tokens, n_layers=l_keep)
+    for l in range(l_keep):
+        assert _maxdiff(pop["K"][l], fused["K"][l]) < 1e-11
+        assert _maxdiff(pop["V"][l], fused["V"][l]) < 1e-11
+    assert _maxdiff(pop["H"][0], fused["hidden"][0, :-1]) < 1e-11
+
+
+def test_first_token_depends_on_the_projected_cache():
+    cfg, w, tokens = _setup("llama", n=8)
+    pop = po.pop_prefill(cfg, w, tokens, None, 1)
+
+    class Zeroed(DictWeights):
+        pass
+    wz = Zeroed(cfg)
+    wz.t[("wv", 3)] = torch.zeros_like(wz.t[("wv", 3)])
+    popz = po.pop_prefill(cfg, wz, tokens, None, 1)
+    assert _maxdiff(pop["logits"], popz["logits"]) > 1e-4
+
+
+def test_single_token_prompt_has_an_empty_first_phase():
+    cfg, w, tokens = _setup("llama", n=1)
+    pop = po.pop_prefill(cfg, w, tokens, None, 1)
+    full = po.full_prefill(cfg, w, tokens)
+    assert pop["H"].shape[1] == 0
+    assert _maxdiff(pop["logits"], full["logits"]) < 1e-12
+
+
+def test_embedding_rows_can_replace_tokens():
+    cfg, w, tokens = _setup("llama", n=6)
+    emb = w.get("embed")[tokens[0].long()].reshape(1, 6, -1)
+    mixed = tokens.clone()
+    mixed[:, :4] = -1
+    a = po.pop_prefill(cfg, w, tokens, None, 2)
+    b = po.pop_prefill(cfg, w, mixed, emb, 2)
+    assert _maxdiff(a["logits"], b["logits"]) < 1e-12
+
+
+def test_kernel_precision_mode_stays_close_to_exact_mode():
+    cfg, w, tokens = _setup("gemma", n=8)
+    a = po.pop_prefill(cfg, w, tokens, None, 2)
+    b = po.pop_prefill(cfg, w, tokens, None, 2, precision="bf16ops")
+    err = _maxdiff(a["logits"], b["logits"])
+    assert 0 < err < 0.1 * a["logits"].abs().max().item()
+
+
+# ------------------------------------------------------------------ planted mistakes
+
+def _pins_hold(cfg, w, tokens):
+    """Re-runs the cheap structural and brute-force pins; True when all hold."""
+    try:
+        out = po.full_prefill(cfg, w, tokens)
+        Ks, Vs, logits = brute_force_full(cfg, w, tokens[0].tolist())
+        ok = np.allclose(out["logits"][0].numpy(), logits, atol=1e-9)
+        ok &= all(np.allclose(out["K"][l][0].numpy(), Ks[l], atol=1e-9) for l in range(cfg.n_layers))
+        ok &= all(np.allclose(out["V"][l][0].numpy(), Vs[l], atol=1e-9) for l in range(cfg.n_layers))
+        pop = po.pop_prefill(cfg, w, tokens, None, cfg.n_layers - 1)
+        ok &= _maxdiff(out["logits"], pop["logits"]) < 1e-9
+        ok &= all(_maxdiff(out["K"][l], pop["K"][l]) < 1e-9 for l in range(cfg.n_layers))
+        pop1 = po.pop_prefill(cfg, w, tokens, None, 1)
+        ok &= _maxdiff(out["K"][1], pop1["K"][1]) < 1e-9 and _maxdiff(out["V"][1], pop1["V"][1]) < 1e-9
+        return bool(ok)
+    except Exception:
+        return False
+
+
+MISTAKES = {
+    "rope_sign": ("rope", lambda orig: (lambda x, p, t: orig(x, -p, t))),
+    "rope_interleaved_pairs": ("rope", lambda orig: (lambda x, p, t: orig(
+        x.reshape(*x.shape[:-1], -1, 2).transpose(-1, -2).reshape(x.shape), p, t))),
+    "norm_without_gain": ("rmsnorm", lambda orig: (lambda x, g, e: orig(x, torch.ones_like(g), e))),
+    "norm_eps_outside_root": ("rmsnorm", lambda orig: (lambda x, g, e: x / (x.pow(2).mean(-1, keepdim=True).sqrt() + e) * g)),
+    "window_off_by_one": ("attention", lambda orig: (lambda q, k, v, qp, w, pr="exact": orig(q, k, v, qp, w + 1 if w > 0 else 0, pr))),
+    "act_swapped": ("gated_act", lambda orig: (lambda g, u, a: orig(g, u, 1 - a))),
+    "gate_up_swapped": ("gated_act", lambda orig: (lambda g, u, a: orig(u, g, a))),
+    "pruned_layer_uses_previous_layers_weights": ("kv_generation", lambda orig: (
+        lambda cfg, w, l, x, pos, dt, pr: orig(cfg, w, l - 1 if x.shape[0] > 1 and l == cfg.n_layers else l, x, pos, dt, pr))),
+}
+
+
+def test_pins_hold_unmodified():
+    cfg, w, tokens = _setup("gemma", n=6)
+    assert _pins_hold(cfg, w, tokens)
+
+
+@pytest.mark.parametrize("name", list(MISTAKES))
+def test_planted_mistake_is_caught(name, monkeypatch):
+    cfg, w, tokens = _setup("gemma", n=6)
+    attr, make = MISTAKES[name]
+    monkeypatch.setattr(po, attr, make(getattr(po, attr)))
+    assert not _pins_hold(cfg, w, tokens)
