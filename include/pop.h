@@ -1,0 +1,134 @@
+/* pop.h - C ABI of the POP (Prefill-Only Pruning) prefill library for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates the prefill stage of a decoder-only transformer in two ways:
+ *
+ *   pop_full_prefill  the standard prefill: all L layers over the prompt x_1..x_N
+ *                     (paper Sec. 2.1, Eq. 1-3), logits of the last prompt position;
+ *   pop_prefill       POP's pruned prefill (paper Sec. 3.3): layers 1..L_keep run in full; each
+ *                     deeper layer only stores k = RoPE(LN(H) W^K), v = LN(H) W^V computed from the
+ *                     state H leaving the kept stack (Eq. 14) and passes H on unchanged (Eq. 15);
+ *                     the last prompt token x_N is then run through ALL L layers as the first
+ *                     decode step (boundary handling), so its logits use the whole model.
+ *
+ * Conventions
+ *   - Every pointer named dev_* or documented "device" is CUDA device memory owned by the caller.
+ *     The library borrows it; it allocates no device memory of its own and frees none.
+ *   - `stream` is a cudaStream_t passed as void*. Calls enqueue work on it and return without
+ *     synchronising (pop_last_status is the exception).
+ *   - Return value: POP_OK (0) or a negative pop_status code. A call that returns an error has
+ *     enqueued nothing and written nothing.
+ *   - Matrices are row-major bf16 [out_features, in_features] (y = x W^T). Norm gains are fp32.
+ *   - Sequences of a batch have equal length; positions are 0-based.
+ */
+#ifndef POP_H_
+#define POP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  POP_OK = 0,
+  POP_E_INVALID = -1,        /* null pointer, size out of range, shape inconsistent with the config */
+  POP_E_NOSPACE = -2,        /* weight arena, workspace or KV pages too small */
+  POP_E_CUDA = -3,           /* a CUDA runtime / driver call or a launch failed */
+  POP_E_DEVICE_TIMEOUT = -4, /* a bounded device-side wait expired (seen through pop_last_status) */
+  POP_E_MISSING = -5         /* pop_load_weights: a required tensor was not supplied */
+} pop_status;
+
+typedef struct pop_model pop_model_t; /* opaque */
+
+/* Model shape. struct_size must be sizeof(pop_config_t) (guards against ABI drift). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rms_eps;
+  float rope_theta;
+  int32_t act;          /* 0: SiLU-gated FFN, 1: tanh-GELU-gated FFN */
+  int32_t qk_norm;      /* 1: per-head RMSNorm on q and k between projection and RoPE */
+  int32_t post_norms;   /* 1: RMSNorm on the attention and FFN outputs before the residual add */
+  int32_t window;       /* sliding-window size in keys, own position included; 0: all layers global */
+  int32_t global_every; /* with window > 0: 1-based layer l is global iff l % global_every == 0 */
+} pop_config_t;
+
+/* One named weight tensor handed to pop_load_weights.
+ * name: "embed", "final_norm", "lm_head", or "layers.<l>.<t>" with 1-based l and t one of
+ *   ln_in, wq, wk, wv, wo, ln_ffn, w_gate, w_up, w_down, q_norm, k_norm, post_attn_norm, post_ffn_norm.
+ * dev_ptr: device memory, contiguous; dtype 0 = bf16 (matrices), 1 = fp32 (norm gains). */
+typedef struct {
+  const char* name;
+  const void* dev_ptr;
+  int32_t dtype;
+  int32_t ndim;
+  int64_t shape[2];
+} pop_tensor_t;
+
+/* Paged KV cache, caller-owned device memory.
+ * k_pool, v_pool: bf16 [n_layers][num_pages][page_size][n_kv_heads][head_dim].
+ * block_table:    device int32 [batch][max_pages_per_seq]; entry (b, j) is the page that holds
+ *                 positions j*page_size .. (j+1)*page_size-1 of sequence b.
+ * page_size must be a multiple of 16. Entries of a page beyond seq_len are left untouched. */
+typedef struct {
+  void* k_pool;
+  void* v_pool;
+  const int32_t* block_table;
+  int32_t page_size, num_pages, max_pages_per_seq;
+} pop_kv_cache_t;
+
+/* Prompt. tokens: device int32 [batch][seq_len]. embeds: device bf16 [batch][seq_len][d_model] or
+ * NULL; when given, a position whose token id is negative takes its input row from embeds (visual
+ * or other pre-computed embeddings) instead of the embedding table. */
+typedef struct {
+  const int32_t* tokens;
+  const void* embeds;
+} pop_input_t;
+
+/* Bytes of device memory pop_load_weights needs for the repacked weights of `cfg`. */
+size_t pop_weight_arena_bytes(const pop_config_t* cfg);
+
+/* Repack the given tensors into dev_arena (fused QKV, tile-interleaved gate/up, concatenated K/V
+ * projections for the pruned-layer pass) on `stream` and return a model handle. The source tensors
+ * may be released once the stream has drained. Errors: POP_E_INVALID, POP_E_NOSPACE, POP_E_MISSING,
+ * POP_E_CUDA. The handle (host memory) is released with pop_free; the arena stays the caller's. */
+int pop_load_weights(const pop_config_t* cfg, const pop_tensor_t* tensors, int32_t n_tensors,
+                     void* dev_arena, size_t arena_bytes, void* stream, pop_model_t** out);
+
+/* Scratch bytes a prefill of `batch` sequences of `seq_len` tokens needs (activations, fp32
+ * residual stream, rotary table, split-KV partials). */
+size_t pop_workspace_bytes(const pop_model_t* m, int32_t seq_len, int32_t batch);
+
+/* Lend the library a workspace of `bytes` bytes (device, 1024-byte aligned). It is used by every
+ * later prefill call until replaced; calls that overlap on the GPU must not share one. */
+int pop_set_workspace(pop_model_t* m, void* dev_ws, size_t bytes);
+
+/* POP pruned prefill with boundary handling (paper Sec. 3.3, Eq. 14-15). 1 <= L_keep <= n_layers.
+ * On completion kv_cache_out holds seq_len entries for EVERY layer and sequence: layers <= L_keep
+ * and position seq_len-1 of all layers from full layer evaluations, positions 0..seq_len-2 of
+ * layers > L_keep from the independent K/V projections of H. logits_out: device fp32
+ * [batch][vocab], the next-token logits at the last prompt position. L_keep == n_layers gives
+ * exactly pop_full_prefill. */
+int pop_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
+                int32_t L_keep, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
+
+/* Standard full-depth prefill of the unpruned model (paper Sec. 2.1, Eq. 1-3; the reference path
+ * POP is compared with in Sec. 4.3). Same outputs as pop_prefill. */
+int pop_full_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
+                     pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
+
+/* Synchronise `stream`, then read and clear the device status word: POP_OK, or
+ * POP_E_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or POP_E_CUDA. */
+int pop_last_status(pop_model_t* m, void* stream);
+
+/* Number of kernel launches the last prefill call on this model enqueued. */
+int64_t pop_last_launch_count(const pop_model_t* m);
+
+void pop_free(pop_model_t* m);
+const char* pop_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POP_H_ */

@@ -1,0 +1,337 @@
+// bf16 GEMM on the 5th-generation tensor cores: D[M,N] = A[M,K] * B[N,K]^T, fp32 accumulation.
+//
+// One persistent CTA per SM walks 128 x 256 output tiles. Warp roles:
+//   warp 0      TMA producer: streams 128x64 (A) and 256x64 (B) bf16 blocks into a 4-stage
+//               shared-memory ring (128-byte swizzle), signalling `full` mbarriers;
+//   warp 1      allocates TMEM, issues tcgen05.mma (128x256x16 per instruction) into one of two
+//               256-column fp32 accumulators, frees ring stages with tcgen05.commit;
+//   warps 2..5  epilogue: tcgen05.ld the finished accumulator (one output row per thread, 32
+//               columns at a time), apply the fused epilogue and store, while the MMA warp already
+//               fills the other accumulator with the next tile.
+// Used for the QKV, O, gate/up and down projections of kept layers (paper Eq. 1-2) and, batched
+// over the pruned layers, for their independent K/V projections (Eq. 14).
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace pop {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int GEMM_THREADS = 192;
+constexpr int GROUP_M = 16;
+constexpr uint32_t TMEM_COLS = 512;
+
+struct __align__(1024) GemmSmem {
+  uint8_t a[STAGES][A_BYTES];
+  uint8_t b[STAGES][B_BYTES];
+  uint64_t full[STAGES];
+  uint64_t empty[STAGES];
+  uint64_t tfull[2];
+  uint64_t tempty[2];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+struct GemmDev {
+  void* out;
+  int64_t ldo, out_batch_stride;
+  int M, N, K, batch;
+  int m_tiles, n_tiles;
+  int act, n_valid;
+};
+
+__device__ __forceinline__ void tile_coords(const GemmDev& p, int t, int& g, int& m, int& n) {
+  const int per_batch = p.m_tiles * p.n_tiles;
+  g = t / per_batch;
+  const int r = t - g * per_batch;
+  const int span = GROUP_M * p.n_tiles;
+  const int grp = r / span;
+  const int first_m = grp * GROUP_M;
+  const int gsize = min(GROUP_M, p.m_tiles - first_m);
+  const int rr = r - grp * span;
+  m = first_m + rr % gsize;
+  n = rr / gsize;
+}
+
+__device__ __forceinline__ float act_fn(float g, int act) {
+  if (act == 0) return g / (1.0f + expf(-g));
+  const float c = 0.7978845608028654f;
+  return 0.5f * g * (1.0f + tanhf(c * (g + 0.044715f * g * g * g)));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p,
+            int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  GemmSmem& s = *reinterpret_cast<GemmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
+  const int k_blocks = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(&s.full[i], 1);
+      mbar_init(&s.empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s.tfull[i], 1);
+      mbar_init(&s.tempty[i], 4);
+    }
+    s.abort = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(&s.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = blockIdx.x; t < total_tiles && !s.abort; t += gridDim.x) {
+        int g, m, n;
+        tile_coords(p, t, g, m, n);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&s.empty[stage], phase ^ 1)) {
+            s.abort = 1;
+            atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+            break;
+          }
+          mbar_expect_tx(&s.full[stage], A_BYTES + B_BYTES);
+          tma_load_3d(s.a[stage], &tmA, &s.full[stage], kb * BK, m * BM, g);
+          tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BK, n * BN, g);
+          if (++stage == STAGES) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int t = blockIdx.x; t < total_tiles && !s.abort; t += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t bphase = (it >> 1) & 1;
+        if (!mbar_wait(&s.tempty[buf], bphase ^ 1)) {
+          s.abort = 1;
+          atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&s.full[stage], phase)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(s.a[stage]);
+          const uint32_t b_addr = smem_u32(s.b[stage]);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t ad = umma_smem_desc(a_addr + k * 32, 16, 1024);
+            const uint64_t bd = umma_smem_desc(b_addr + k * 32, 16, 1024);
+            umma_bf16_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&s.empty[stage]);
+          if (++stage == STAGES) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+        if (!ok) {
+          s.abort = 1;
+          atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+          break;
+        }
+        umma_commit(&s.tfull[buf]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps)
+    const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    int it = 0;
+    for (int t = blockIdx.x; t < total_tiles && !s.abort; t += gridDim.x, ++it) {
+      const int buf = it & 1;
+      const uint32_t bphase = (it >> 1) & 1;
+      int g, m, n;
+      tile_coords(p, t, g, m, n);
+      if (!mbar_wait(&s.tfull[buf], bphase)) {
+        s.abort = 1;
+        atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const int row = m * BM + row_in_tile;
+      const bool row_ok = row < p.M;
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+      if (EPI == EPI_GATED_BF16) {
+        bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t gr[32], ur[32];
+          tmem_ld_32x32b_x32(taddr + c * 32, gr);
+          tmem_ld_32x32b_x32(taddr + 128 + c * 32, ur);
+          tmem_wait_ld();
+          const int col0 = n * 128 + c * 32;
+          if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + v * 8 + 8 <= p.n_valid) {
+                uint32_t w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int e = v * 8 + j * 2;
+                  const float x0 = act_fn(__uint_as_float(gr[e]), p.act) * __uint_as_float(ur[e]);
+                  const float x1 = act_fn(__uint_as_float(gr[e + 1]), p.act) * __uint_as_float(ur[e + 1]);
+                  w[j] = pack_bf16(x0, x1);
+                }
+                *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(taddr + c * 32, r);
+          tmem_wait_ld();
+          const int col0 = n * BN + c * 32;
+          if (row_ok) {
+            if (EPI == EPI_STORE_BF16) {
+              bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                if (col0 + v * 8 + 8 <= p.N) {
+                  uint32_t w[4];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j)
+                    w[j] = pack_bf16(__uint_as_float(r[v * 8 + j * 2]), __uint_as_float(r[v * 8 + j * 2 + 1]));
+                  *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+              }
+            } else {
+              float* out = reinterpret_cast<float*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll
+              for (int v = 0; v < 8; ++v) {
+                if (col0 + v * 4 + 4 <= p.N) {
+                  float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                         __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+                  float4* dst = reinterpret_cast<float4*>(out + col0 + v * 4);
+                  if (EPI == EPI_ADD_F32) {
+                    const float4 o = *dst;
+                    x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
+                  }
+                  *dst = x;
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.tempty[buf]);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (s.abort && threadIdx.x == 0) {
+    // give bulk copies that may still be in flight into this CTA's shared memory time to land
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int EPI>
+int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, int grid, cudaStream_t stream) {
+  const size_t smem = sizeof(GemmSmem) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return POP_E_CUDA;
+    configured = true;
+  }
+  gemm_kernel<EPI><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status_word());
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+}  // namespace
+
+int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
+  if (!a.A || !a.B || !a.out || a.M < 1 || a.N < 1 || a.K < 1 || a.batch < 1) return POP_E_INVALID;
+  if (a.K % 8 || a.lda % 8 || a.ldb % 8 || a.a_batch_stride % 8 || a.b_batch_stride % 8) return POP_E_INVALID;
+  if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.out)) & 15)
+    return POP_E_INVALID;
+  if (a.epilogue == EPI_GATED_BF16) {
+    if (a.N % 256 || a.n_valid % 8 || a.n_valid > a.N / 2 || a.ldo % 8) return POP_E_INVALID;
+  } else if (a.epilogue == EPI_STORE_BF16) {
+    if (a.N % 8 || a.ldo % 8) return POP_E_INVALID;
+  } else {
+    if (a.N % 4 || a.ldo % 4) return POP_E_INVALID;
+  }
+  CUtensorMap ta, tb;
+  int rc = make_tmap_bf16_3d(&ta, a.A, a.K, a.M, a.batch, a.lda, a.a_batch_stride ? a.a_batch_stride : a.lda * a.M,
+                             BK, BM);
+  if (rc) return rc;
+  rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
+                         BN);
+  if (rc) return rc;
+  GemmDev p;
+  p.out = a.out;
+  p.ldo = a.ldo;
+  p.out_batch_stride = a.out_batch_stride;
+  p.M = a.M; p.N = a.N; p.K = a.K; p.batch = a.batch;
+  p.m_tiles = ceil_div(a.M, BM);
+  p.n_tiles = ceil_div(a.N, BN);
+  p.act = a.act;
+  p.n_valid = a.n_valid;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return POP_E_CUDA;
+  const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
+  const int grid = (int)(total < sms ? total : sms);
+  switch (a.epilogue) {
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, p, grid, stream);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, p, grid, stream);
+    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, p, grid, stream);
+    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, p, grid, stream);
+  }
+  return POP_E_INVALID;
+}
+
+}  // namespace pop
