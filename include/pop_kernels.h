@@ -26,6 +26,53 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
                int64_t ldo, int64_t o_bs, int32_t M, int32_t N, int32_t K, int32_t batch, int32_t epilogue,
                int32_t act, int32_t n_valid, void* stream);
 
+/* Causal GQA attention of a decoder layer over the paged cache (paper Eq. 1, Attn(x_l, K, V) after
+ * the append of Eq. 3): for sequence b, query row i (absolute position q_pos0 + i) and head h,
+ *   out[b][i][h] = sum_j softmax_j(q[b][i][h] . k[b][j][g] / sqrt(hd)) v[b][j][g],  g = h*n_kv/n_q,
+ * over cache positions j <= q_pos0 + i, and j > q_pos0 + i - window when window > 0.
+ * q: device bf16 [batch*seq_len][ldq] (head h at column h*hd); k_pool/v_pool: ONE layer of the
+ * cache, bf16 [num_pages][page_size][n_kv][hd]; block_table as in pop_kv_cache_t; out: bf16
+ * [batch*seq_len][ldo]. kv_len = valid cache positions (>= q_pos0 + seq_len). hd in {64,128,256}. */
+int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool, const int32_t* block_table,
+                    void* out, int64_t ldo, int32_t batch, int32_t seq_len, int32_t q_pos0, int32_t kv_len,
+                    int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t page_size, int32_t num_pages,
+                    int32_t max_pages_per_seq, int32_t window, void* stream);
+
+/* RMSNorm, the LN of paper Eq. 2 / Eq. 14: out[g][r][:] = x[r][:] * rsqrt(mean(x[r]^2)+eps) * gain[g][:].
+ * x fp32 [rows][ldx]; gain fp32, group g at gain + g*gain_stride; out bf16 (out_f32 = 0) or fp32,
+ * group stride out_gs elements. */
+int pop_k_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_stride, void* out, int64_t ldo,
+                  int64_t out_gs, int32_t rows, int32_t d, int32_t groups, float eps, int32_t out_f32, void* stream);
+
+/* Rotary table: table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)) as float2, pos < n_pos, j < hd/2. */
+int pop_k_rope_table(void* table, int32_t n_pos, int32_t head_dim, float theta, void* stream);
+
+/* KV generation and append (paper Eq. 2-3; Eq. 14 when applied to a pruned layer): rows of fp32
+ * projections [q heads | k heads | v heads] * hd get the optional per-head RMSNorm (q, k), RoPE
+ * (q, k), rounding to bf16; q goes to q_out [rows][ldq], k and v into cache layer layer0 + g of
+ * the pools [layer][page][slot][n_kv][hd] (pool_layer_stride elements per layer). Row r belongs to
+ * sequence r / rows_per_seq at position pos0 + r % rows_per_seq; rows with r % rows_per_seq >=
+ * rows_written are skipped. n_q may be 0 (pruned layers: no query). */
+int pop_k_rope_cache(const float* in, int64_t ld_in, int64_t in_gs, void* q_out, int64_t ldq, void* k_pool,
+                     void* v_pool, int64_t pool_layer_stride, int32_t layer0, const int32_t* block_table,
+                     int32_t max_pages_per_seq, int32_t page_size, const float* q_gain, const float* k_gain,
+                     int64_t gain_gs, const void* table, int32_t n_q, int32_t n_kv, int32_t head_dim, int32_t rows,
+                     int32_t rows_per_seq, int32_t rows_written, int32_t pos0, int32_t groups, float eps,
+                     void* stream);
+
+/* Weight-streaming GEMV of the boundary-token path (paper Sec. 3.3) and of the output head:
+ * out[b][n] = sum_k x[b][k] * W[n][k] for a few rows b. x bf16 or fp32 (x_f32) [B][ldx]; W bf16
+ * [N][ldw]. mode 0: fp32 store; 2: fp32 +=; 3: gated (W rows in 128-gate/128-up blocks) -> bf16. */
+int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t ldw, void* out, int64_t ldo,
+               int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid, void* stream);
+
+/* Scratch floats pop_k_decode_attention needs: batch * n_q * 64 * (hd + 2). Single-query attention
+ * of the boundary token (one query per sequence at position kv_len-1) over one cache layer. */
+int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
+                           const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
+                           void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
+                           int32_t kv_len, int32_t window, void* stream);
+
 /* Synchronise the stream, then read and clear the library's device status word. */
 int pop_k_status(void* stream);
 

@@ -67,6 +67,13 @@ SIGNATURES = {
     "pop_strerror": (C.c_char_p, [C.c_int]),
     "pop_k_gemm": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _I32, _I32, _I32,
                              _I32, _P]),
+    "pop_k_attention": (C.c_int, [_P, _I64, _P, _P, _P, _P, _I64] + [_I32] * 11 + [_P]),
+    "pop_k_rmsnorm": (C.c_int, [_P, _I64, _P, _I64, _P, _I64, _I64, _I32, _I32, _I32, _F, _I32, _P]),
+    "pop_k_rope_table": (C.c_int, [_P, _I32, _I32, _F, _P]),
+    "pop_k_rope_cache": (C.c_int, [_P, _I64, _I64, _P, _I64, _P, _P, _I64, _I32, _P, _I32, _I32, _P, _P, _I64, _P]
+                         + [_I32] * 8 + [_F, _P]),
+    "pop_k_gemv": (C.c_int, [_P, _I64, _I32, _P, _I64, _P, _I64] + [_I32] * 6 + [_P]),
+    "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_status": (C.c_int, [_P]),
     "pop_k_launch_count": (_I64, []),
     "pop_k_reset_launch_count": (None, []),
@@ -130,8 +137,64 @@ class PopLibrary:
         return out
 
 
-class PopModel:
-    """Placeholder until the model-level calls are bound (see PopLibrary for kernel-level calls)."""
+    def attention(self, q, k_pool, v_pool, block_table, out, batch, seq_len, kv_len, n_q, n_kv, hd, page_size,
+                  window=0, q_pos0=0, stream=None):
+        """q [batch*seq_len, >= n_q*hd] bf16; k_pool/v_pool one cache layer [pages, page_size, n_kv, hd]."""
+        code = self.dll.pop_k_attention(q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(),
+                                        block_table.data_ptr(), out.data_ptr(), out.stride(0), batch, seq_len,
+                                        q_pos0, kv_len, n_q, n_kv, hd, page_size, k_pool.shape[0],
+                                        block_table.shape[1], window, _stream_ptr(stream))
+        self.check(code, "pop_k_attention")
+        return out
+
+    def rmsnorm(self, x, gain, out, eps, stream=None):
+        """x fp32 [rows, d]; gain fp32 [d] or [groups, d]; out bf16/fp32 [rows, d] or [groups, rows, d]."""
+        groups = 1 if gain.dim() == 1 else gain.shape[0]
+        rows, d = x.shape
+        code = self.dll.pop_k_rmsnorm(x.data_ptr(), x.stride(0), gain.data_ptr(),
+                                      0 if gain.dim() == 1 else gain.stride(0), out.data_ptr(), out.stride(-2),
+                                      0 if out.dim() == 2 else out.stride(0), rows, d, groups, eps,
+                                      1 if out.dtype == torch.float32 else 0, _stream_ptr(stream))
+        self.check(code, "pop_k_rmsnorm")
+        return out
+
+    def rope_table(self, table, n_pos, hd, theta, stream=None):
+        self.check(self.dll.pop_k_rope_table(table.data_ptr(), n_pos, hd, theta, _stream_ptr(stream)),
+                   "pop_k_rope_table")
+        return table
+
+    def rope_cache(self, x, q_out, k_pool, v_pool, layer0, block_table, page_size, q_gain, k_gain, table, n_q, n_kv,
+                   hd, rows_per_seq, rows_written, pos0, eps, stream=None):
+        """x fp32 [rows, (n_q+2 n_kv) hd] or [groups, rows, ...]; pools [layers, pages, page_size, n_kv, hd]."""
+        groups = 1 if x.dim() == 2 else x.shape[0]
+        rows = x.shape[-2]
+        gain_gs = 0 if (k_gain is None or k_gain.dim() == 1) else k_gain.stride(0)
+        code = self.dll.pop_k_rope_cache(x.data_ptr(), x.stride(-2), 0 if x.dim() == 2 else x.stride(0),
+                                         _ptr(q_out), 0 if q_out is None else q_out.stride(0), k_pool.data_ptr(),
+                                         v_pool.data_ptr(), k_pool.stride(0), layer0, block_table.data_ptr(),
+                                         block_table.shape[1], page_size, _ptr(q_gain), _ptr(k_gain), gain_gs,
+                                         table.data_ptr(), n_q, n_kv, hd, rows, rows_per_seq, rows_written, pos0,
+                                         groups, eps, _stream_ptr(stream))
+        self.check(code, "pop_k_rope_cache")
+
+    def gemv(self, x, w, out, mode=0, act=0, n_valid=0, stream=None):
+        B, K = x.shape
+        code = self.dll.pop_k_gemv(x.data_ptr(), x.stride(0), 1 if x.dtype == torch.float32 else 0, w.data_ptr(),
+                                   w.stride(0), out.data_ptr(), out.stride(0), B, w.shape[0], K, mode, act, n_valid,
+                                   _stream_ptr(stream))
+        self.check(code, "pop_k_gemv")
+        return out
+
+    def decode_attention(self, q, k_pool, v_pool, block_table, out, n_q, n_kv, hd, kv_len, page_size, window=0,
+                         stream=None):
+        batch = q.shape[0]
+        partial = torch.empty(batch * n_q * 64 * (hd + 2), dtype=torch.float32, device=q.device)
+        code = self.dll.pop_k_decode_attention(q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(),
+                                               block_table.data_ptr(), block_table.shape[1], page_size,
+                                               partial.data_ptr(), out.data_ptr(), out.stride(0), batch, n_q, n_kv,
+                                               hd, kv_len, window, _stream_ptr(stream))
+        self.check(code, "pop_k_decode_attention")
+        return out
 
 
 _LIB: Optional[PopLibrary] = None
@@ -143,3 +206,149 @@ def lib() -> PopLibrary:
     if _LIB is None:
         _LIB = PopLibrary()
     return _LIB
+
+
+def make_config(cfg) -> pop_config_t:
+    """pop_config_t from any object with the fields of pop_synth.ModelConfig."""
+    c = pop_config_t()
+    c.struct_size = C.sizeof(pop_config_t)
+    for f in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "act", "qk_norm",
+              "post_norms", "window", "global_every"):
+        setattr(c, f, int(getattr(cfg, f)))
+    c.rms_eps = float(cfg.rms_eps)
+    c.rope_theta = float(cfg.rope_theta)
+    return c
+
+
+class KVCache:
+    """Caller-owned paged KV cache: bf16 pools [n_layers, num_pages, page_size, n_kv, hd] and an
+    int32 block table [batch, max_pages_per_seq] (identity paging unless `block_table` is given)."""
+
+    def __init__(self, cfg, batch: int, seq_len: int, page_size: int = 128, device="cuda",
+                 block_table: Optional[torch.Tensor] = None, num_pages: Optional[int] = None, fill: float = 0.0):
+        pps = (seq_len + page_size - 1) // page_size
+        self.page_size = page_size
+        self.num_pages = num_pages or batch * pps
+        shape = (cfg.n_layers, self.num_pages, page_size, cfg.n_kv_heads, cfg.head_dim)
+        self.k = torch.full(shape, fill, dtype=torch.bfloat16, device=device)
+        self.v = torch.full(shape, fill, dtype=torch.bfloat16, device=device)
+        if block_table is None:
+            block_table = torch.arange(batch * pps, dtype=torch.int32).reshape(batch, pps)
+        self.block_table = block_table.to(device=device, dtype=torch.int32).contiguous()
+        self.batch, self.seq_len = batch, seq_len
+
+    def struct(self) -> pop_kv_cache_t:
+        s = pop_kv_cache_t()
+        s.k_pool, s.v_pool, s.block_table = self.k.data_ptr(), self.v.data_ptr(), self.block_table.data_ptr()
+        s.page_size, s.num_pages, s.max_pages_per_seq = self.page_size, self.num_pages, self.block_table.shape[1]
+        return s
+
+    def gather(self, layer: int, seq_len: Optional[int] = None):
+        """(K, V) of 0-based `layer` as dense [batch, seq_len, n_kv, hd] tensors (a host-side view for checks)."""
+        n = seq_len or self.seq_len
+        pos = torch.arange(n, device=self.k.device)
+        pages = self.block_table[:, pos // self.page_size].long()          # [batch, n]
+        slots = (pos % self.page_size)[None, :].expand_as(pages)
+        return self.k[layer][pages, slots], self.v[layer][pages, slots]
+
+
+class PopModel:
+    """A loaded model: repacked weights in a device arena plus a workspace, both torch tensors."""
+
+    def __init__(self, cfg, weights, library: Optional[PopLibrary] = None, device="cuda"):
+        """`weights.get(name, layer)` must return bf16 matrices / fp32 gains on `device`
+        (layer 1-based, 0 for embed, final_norm, lm_head)."""
+        self.lib = library or lib()
+        self.cfg = cfg
+        self.device = device
+        self.c_cfg = make_config(cfg)
+        nbytes = self.lib.dll.pop_weight_arena_bytes(C.byref(self.c_cfg))
+        if nbytes == 0:
+            raise PopError(POP_E_INVALID, "pop_weight_arena_bytes")
+        self.arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        base = (self.arena.data_ptr() + 1023) // 1024 * 1024
+        names = [("embed", 0), ("final_norm", 0), ("lm_head", 0)]
+        per_layer = ["ln_in", "wq", "wk", "wv", "wo", "ln_ffn", "w_gate", "w_up", "w_down"]
+        if cfg.qk_norm:
+            per_layer += ["q_norm", "k_norm"]
+        if cfg.post_norms:
+            per_layer += ["post_attn_norm", "post_ffn_norm"]
+        self.handle = C.c_void_p()
+        # load layer by layer so that only one layer's source tensors are alive at a time
+        groups = [names] + [[(n, l) for n in per_layer] for l in range(1, cfg.n_layers + 1)]
+        tensors, keep = [], []
+        for grp in groups:
+            for name, layer in grp:
+                t = weights.get(name, layer).to(device).contiguous()
+                keep.append(t)
+                pt = pop_tensor_t()
+                pt.name = (name if layer == 0 else f"layers.{layer}.{name}").encode()
+                pt.dev_ptr = t.data_ptr()
+                pt.dtype = 0 if t.dtype == torch.bfloat16 else 1
+                pt.ndim = t.dim()
+                pt.shape[0] = t.shape[0]
+                pt.shape[1] = t.shape[1] if t.dim() > 1 else 0
+                tensors.append(pt)
+        arr = (pop_tensor_t * len(tensors))(*tensors)
+        code = self.lib.dll.pop_load_weights(C.byref(self.c_cfg), arr, len(tensors), base, nbytes,
+                                             _stream_ptr(None), C.byref(self.handle))
+        self.lib.check(code, "pop_load_weights")
+        torch.cuda.current_stream().synchronize()
+        del keep
+        self.ws = None
+        self.ws_shape = None
+
+    def ensure_workspace(self, seq_len: int, batch: int):
+        need = self.lib.dll.pop_workspace_bytes(self.handle, seq_len, batch)
+        if self.ws is None or self.ws.numel() < need + 1024:
+            self.ws = torch.empty(need + 1024, dtype=torch.uint8, device=self.device)
+        base = (self.ws.data_ptr() + 1023) // 1024 * 1024
+        self.lib.check(self.lib.dll.pop_set_workspace(self.handle, base, self.ws.numel() - 1024),
+                       "pop_set_workspace")
+
+    def _input(self, tokens, embeds):
+        inp = pop_input_t()
+        inp.tokens = tokens.data_ptr()
+        inp.embeds = None if embeds is None else embeds.data_ptr()
+        return inp
+
+    def prefill(self, tokens, embeds, l_keep: int, cache: KVCache, logits: Optional[torch.Tensor] = None,
+                stream=None):
+        """pop_prefill on device tensors: tokens int32 [B, N], embeds bf16 [B, N, d] or None."""
+        B, N = tokens.shape
+        self.ensure_workspace(N, B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_prefill(self.handle, C.byref(inp), N, B, l_keep, C.byref(kc), logits.data_ptr(),
+                                        _stream_ptr(stream))
+        self.lib.check(code, "pop_prefill")
+        return logits
+
+    def full_prefill(self, tokens, embeds, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):
+        B, N = tokens.shape
+        self.ensure_workspace(N, B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_full_prefill(self.handle, C.byref(inp), N, B, C.byref(kc), logits.data_ptr(),
+                                             _stream_ptr(stream))
+        self.lib.check(code, "pop_full_prefill")
+        return logits
+
+    def last_status(self, stream=None) -> int:
+        return self.lib.dll.pop_last_status(self.handle, _stream_ptr(stream))
+
+    def last_launch_count(self) -> int:
+        return self.lib.dll.pop_last_launch_count(self.handle)
+
+    def close(self):
+        if self.handle:
+            self.lib.dll.pop_free(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

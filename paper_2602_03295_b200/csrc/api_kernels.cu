@@ -18,6 +18,74 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
   return launch_gemm(a, static_cast<cudaStream_t>(stream));
 }
 
+int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool, const int32_t* block_table,
+                    void* out, int64_t ldo, int32_t batch, int32_t seq_len, int32_t q_pos0, int32_t kv_len,
+                    int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t page_size, int32_t num_pages,
+                    int32_t max_pages_per_seq, int32_t window, void* stream) {
+  AttnArgs a{};
+  a.q = static_cast<const bf16*>(q); a.ldq = ldq;
+  a.k_pool = static_cast<const bf16*>(k_pool); a.v_pool = static_cast<const bf16*>(v_pool);
+  a.block_table = block_table; a.out = static_cast<bf16*>(out); a.ldo = ldo;
+  a.batch = batch; a.seq_len = seq_len; a.q_pos0 = q_pos0; a.kv_len = kv_len;
+  a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.head_dim = head_dim;
+  a.page_size = page_size; a.num_pages = num_pages; a.max_pages_per_seq = max_pages_per_seq; a.window = window;
+  return launch_attention(a, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_stride, void* out, int64_t ldo,
+                  int64_t out_gs, int32_t rows, int32_t d, int32_t groups, float eps, int32_t out_f32, void* stream) {
+  if (!x || !gain || !out) return POP_E_INVALID;
+  return launch_rmsnorm(x, ldx, gain, gain_stride, out, ldo, out_gs, rows, d, groups, eps, out_f32 != 0,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_rope_table(void* table, int32_t n_pos, int32_t head_dim, float theta, void* stream) {
+  if (!table || n_pos < 1 || head_dim < 2) return POP_E_INVALID;
+  return launch_rope_table(static_cast<float2*>(table), n_pos, head_dim, theta, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_rope_cache(const float* in, int64_t ld_in, int64_t in_gs, void* q_out, int64_t ldq, void* k_pool,
+                     void* v_pool, int64_t pool_layer_stride, int32_t layer0, const int32_t* block_table,
+                     int32_t max_pages_per_seq, int32_t page_size, const float* q_gain, const float* k_gain,
+                     int64_t gain_gs, const void* table, int32_t n_q, int32_t n_kv, int32_t head_dim, int32_t rows,
+                     int32_t rows_per_seq, int32_t rows_written, int32_t pos0, int32_t groups, float eps,
+                     void* stream) {
+  if (!in || !k_pool || !v_pool || !block_table || !table || (n_q > 0 && !q_out)) return POP_E_INVALID;
+  RopeArgs r{};
+  r.in = in; r.ld_in = ld_in; r.in_group_stride = in_gs;
+  r.q_out = static_cast<bf16*>(q_out); r.ldq = ldq;
+  r.k_pool = static_cast<bf16*>(k_pool); r.v_pool = static_cast<bf16*>(v_pool);
+  r.pool_layer_stride = pool_layer_stride; r.layer0 = layer0;
+  r.block_table = block_table; r.max_pages_per_seq = max_pages_per_seq; r.page_size = page_size;
+  r.q_gain = q_gain; r.k_gain = k_gain; r.gain_group_stride = gain_gs;
+  r.table = static_cast<const float2*>(table);
+  r.n_q = n_q; r.n_kv = n_kv; r.hd = head_dim;
+  r.rows = rows; r.rows_per_seq = rows_per_seq; r.rows_written = rows_written; r.pos0 = pos0; r.groups = groups;
+  r.eps = eps;
+  return launch_rope_cache(r, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t ldw, void* out, int64_t ldo,
+               int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid, void* stream) {
+  GemvArgs v{};
+  v.x = x; v.ldx = ldx; v.x_f32 = x_f32 != 0; v.w = static_cast<const bf16*>(w); v.ldw = ldw;
+  v.out = out; v.ldo = ldo; v.B = B; v.N = N; v.K = K; v.mode = mode; v.act = act; v.n_valid = n_valid;
+  return launch_gemv(v, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
+                           const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
+                           void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
+                           int32_t kv_len, int32_t window, void* stream) {
+  DecAttnArgs a{};
+  a.q = static_cast<const bf16*>(q); a.ldq = ldq;
+  a.k_pool = static_cast<const bf16*>(k_pool); a.v_pool = static_cast<const bf16*>(v_pool);
+  a.block_table = block_table; a.max_pages_per_seq = max_pages_per_seq; a.page_size = page_size;
+  a.partial = partial; a.out = static_cast<bf16*>(out); a.ldo = ldo;
+  a.batch = batch; a.n_q = n_q; a.n_kv = n_kv; a.head_dim = head_dim; a.kv_len = kv_len; a.window = window;
+  return launch_decode_attention(a, static_cast<cudaStream_t>(stream));
+}
+
 const char* pop_strerror(int status) {
   switch (status) {
     case POP_OK: return "ok";

@@ -1,0 +1,451 @@
+// Causal, GQA-aware flash-attention prefill on tcgen05 (the Attn(x_l, K, V) of paper Eq. 1, reading
+// the cache that Eq. 2-3 just filled), with an optional sliding window.
+//
+// One CTA owns 128 consecutive query positions of NQT query heads that share a KV head (NQT = 2
+// when the GQA ratio allows it: both tiles see the same keys and the same mask, so every K/V
+// tile staged in shared memory is used twice). Warp roles:
+//   NQT softmax warpgroups (128 threads each, one query row per thread): read S = Q K^T from TMEM,
+//       keep the running row maximum / sum in fp32, write P = exp2(S - m) as bf16 into shared
+//       memory in the swizzled K-major layout the tensor core reads, rescale the O accumulator in
+//       TMEM only when the maximum grew by more than 2^8, and finally normalise and store O;
+//   1 TMA warp: Q tiles once, then K and V tiles of the paged cache through a ring of stages;
+//   1 MMA warp: allocates TMEM, issues S_t = Q_t K^T and O_t += P_t V for both tiles, ordered so
+//       that one tile's softmax overlaps the other tile's matrix products.
+// K/V come straight from the paged cache [page][slot][kv head][hd] with 4-D tensor maps; cache
+// positions >= kv_len are never dereferenced through the block table and never reach the output.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace pop {
+namespace {
+
+template <int HD, int NQT>
+struct AC {
+  static constexpr int BKV = (HD == 256) ? 64 : 128;
+  static constexpr int STAGES = (HD == 128) ? 3 : 4;
+  static constexpr int KV_TILE_BYTES = BKV * HD * 2;
+  static constexpr int KV_SUB_BYTES = BKV * 128;     // one 64-wide slice of head_dim
+  static constexpr int Q_TILE_BYTES = 128 * HD * 2;
+  static constexpr int P_TILE_BYTES = 128 * BKV * 2;
+  static constexpr int THREADS = NQT * 128 + 64;
+  static constexpr int S_COL = 0;                    // S_t at t * BKV
+  static constexpr int O_COL = NQT * BKV;            // O_t at O_COL + t * HD
+  static_assert(NQT * (BKV + HD) <= 512, "TMEM budget");
+};
+
+template <int HD, int NQT>
+struct __align__(1024) AttnSmem {
+  using C = AC<HD, NQT>;
+  uint8_t q[NQT][C::Q_TILE_BYTES];
+  uint8_t p[NQT][C::P_TILE_BYTES];
+  uint8_t kv[C::STAGES][C::KV_TILE_BYTES];
+  uint64_t q_full;
+  uint64_t kv_full[C::STAGES];
+  uint64_t kv_empty[C::STAGES];
+  uint64_t s_full[NQT];
+  uint64_t p_ready[NQT];
+  uint64_t pv_done[NQT];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+struct AttnDev {
+  bf16* out;            // [batch*seq][ldo]
+  int64_t ldo;
+  const int32_t* block_table;
+  int max_pages_per_seq;
+  int page_size;
+  int rows_per_load;    // min(page_size, BKV)
+  int seq_len;          // query rows per sequence (positions q_pos0 .. q_pos0 + seq_len - 1)
+  int q_pos0;
+  int kv_len;           // valid cache positions per sequence
+  int n_q_heads, n_kv_heads;
+  int window;
+  int q_tiles;
+  float scale_log2;     // log2(e) / sqrt(hd)
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+#define POP_ABORT(S, status)                          \
+  do {                                                \
+    (S).abort = 1;                                    \
+    atomicMin((status), (int)POP_E_DEVICE_TIMEOUT);   \
+  } while (0)
+
+template <int HD, int NQT>
+__global__ void __launch_bounds__(AC<HD, NQT>::THREADS, 1)
+attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+            const __grid_constant__ CUtensorMap tmV, const AttnDev p, int* __restrict__ status) {
+  using C = AC<HD, NQT>;
+  constexpr int BKV = C::BKV;
+  constexpr int STAGES = C::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  AttnSmem<HD, NQT>& s =
+      *reinterpret_cast<AttnSmem<HD, NQT>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  // heaviest query tiles (latest positions) first
+  const int q_tile = p.q_tiles - 1 - (int)blockIdx.x;
+  const int head0 = blockIdx.y * NQT;
+  const int b = blockIdx.z;
+  const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
+  const int q_row0 = q_tile * 128;                       // row within the sequence
+  const int pos0 = p.q_pos0 + q_row0;                    // absolute position of row 0
+  const int last_pos = min(pos0 + 127, p.q_pos0 + p.seq_len - 1);
+  const int j_hi = min(last_pos, p.kv_len - 1) / BKV;
+  const int j_lo = p.window > 0 ? max(0, pos0 - p.window + 1) / BKV : 0;
+  const int n_tiles = j_hi - j_lo + 1;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&s.q_full, 1);
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(&s.kv_full[i], 1);
+      mbar_init(&s.kv_empty[i], 1);
+    }
+    for (int t = 0; t < NQT; ++t) {
+      mbar_init(&s.s_full[t], 1);
+      mbar_init(&s.p_ready[t], 128);
+      mbar_init(&s.pv_done[t], 1);
+    }
+    s.abort = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+  }
+  if (warp == NQT * 4 + 1) {
+    tmem_alloc(&s.tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s.tmem_base;
+
+  if (warp == NQT * 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(&s.q_full, NQT * C::Q_TILE_BYTES);
+      for (int t = 0; t < NQT; ++t)
+        for (int c = 0; c < HD / 64; ++c)
+          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, b * p.seq_len + q_row0);
+      const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
+      const int loads_per_tile = BKV / p.rows_per_load;
+      int ring = 0;
+      for (int jj = 0; jj < n_tiles && !s.abort; ++jj) {
+        const int kv0 = (j_lo + jj) * BKV;
+        for (int which = 0; which < 2; ++which, ++ring) {   // 0: K tile, 1: V tile
+          const int stage = ring % STAGES;
+          const uint32_t phase = (ring / STAGES) & 1;
+          if (!mbar_wait(&s.kv_empty[stage], phase ^ 1)) {
+            POP_ABORT(s, status);
+            break;
+          }
+          int n_loads = 0;
+          for (int r = 0; r < loads_per_tile; ++r)
+            if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
+          mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
+          const CUtensorMap* tm = which ? &tmV : &tmK;
+          for (int r = 0; r < n_loads; ++r) {
+            const int pos = kv0 + r * p.rows_per_load;
+            const int page = bt[pos / p.page_size];
+            const int slot = pos % p.page_size;
+            for (int c = 0; c < HD / 64; ++c)
+              tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
+                          c * 64, kv_head, slot, page);
+          }
+        }
+      }
+    }
+  } else if (warp == NQT * 4 + 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc_bf16(128, BKV, 0, 0);
+      constexpr uint32_t idesc_o = umma_idesc_bf16(128, HD, 0, 1);
+      auto issue_s = [&](int t, int stage) {
+        const uint32_t qa = smem_u32(s.q[t]);
+        const uint32_t ka = smem_u32(s.kv[stage]);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint64_t ad = umma_smem_desc(qa + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = umma_smem_desc(ka + (kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32, 16, 1024);
+          umma_bf16_ss(tmem_base + C::S_COL + t * BKV, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+        }
+        umma_commit(&s.s_full[t]);
+      };
+      auto issue_pv = [&](int t, int stage, bool acc) {
+        const uint32_t pa = smem_u32(s.p[t]);
+        const uint32_t va = smem_u32(s.kv[stage]);
+#pragma unroll
+        for (int kk = 0; kk < BKV / 16; ++kk) {
+          const uint64_t ad = umma_smem_desc(pa + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = umma_smem_desc(va + kk * 2048, C::KV_SUB_BYTES, 1024);
+          umma_bf16_ss(tmem_base + C::O_COL + t * HD, ad, bd, idesc_o, (acc || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(&s.pv_done[t]);
+      };
+      bool ok = mbar_wait(&s.q_full, 0);
+      // ring position of K_jj is 2*jj, of V_jj is 2*jj+1
+      if (ok) ok = mbar_wait(&s.kv_full[0], 0);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < NQT; ++t) issue_s(t, 0);
+        umma_commit(&s.kv_empty[0]);
+      }
+      for (int jj = 0; jj < n_tiles && ok && !s.abort; ++jj) {
+        const int rv = 2 * jj + 1, rk = 2 * jj + 2;
+        const int sv = rv % STAGES, sk = rk % STAGES;
+        const bool more = jj + 1 < n_tiles;
+        ok = mbar_wait(&s.kv_full[sv], (rv / STAGES) & 1);
+        if (ok && more) ok = mbar_wait(&s.kv_full[sk], (rk / STAGES) & 1);
+        for (int t = 0; t < NQT && ok; ++t) {
+          ok = mbar_wait(&s.p_ready[t], jj & 1);
+          if (!ok) break;
+          tc_fence_after();
+          if (more) {
+            issue_s(t, sk);
+            if (t == NQT - 1) umma_commit(&s.kv_empty[sk]);
+          }
+          issue_pv(t, sv, jj > 0);
+        }
+        if (ok) umma_commit(&s.kv_empty[sv]);
+      }
+      if (!ok) POP_ABORT(s, status);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warpgroups
+    const int t = warp >> 2;                              // query tile of this warpgroup
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;                  // row in the tile == TMEM lane
+    const int pos = pos0 + row;                           // absolute query position
+    const uint32_t lane_addr = uint32_t(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + lane_addr + C::S_COL + t * BKV;
+    const uint32_t o_addr = tmem_base + lane_addr + C::O_COL + t * HD;
+    uint8_t* p_row = s.p[t] + row * 128;
+    const int sw = row & 7;
+    float m_run = -INFINITY;      // running (possibly stale) maximum, log2 domain
+    float l_run = 0.f;
+    bool ok = true;
+
+    for (int jj = 0; jj < n_tiles && !s.abort; ++jj) {
+      const int kv0 = (j_lo + jj) * BKV;
+      if (!mbar_wait(&s.s_full[t], jj & 1)) { ok = false; break; }
+      tc_fence_after();
+      float sv[BKV];
+#pragma unroll
+      for (int c = 0; c < BKV / 32; ++c)
+        tmem_ld_32x32b_x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+      tmem_wait_ld();
+      // mask + scale, row maximum
+      const bool partial = (kv0 + BKV - 1 > pos0) || (p.window > 0 && kv0 <= pos0 + 127 - p.window);
+      float mx = -INFINITY;
+      if (partial) {
+        const int lo = p.window > 0 ? pos - p.window : -1;   // valid keys: lo < j <= pos
+#pragma unroll
+        for (int i = 0; i < BKV; ++i) {
+          const int j = kv0 + i;
+          const float v = (j <= pos && j > lo) ? sv[i] * p.scale_log2 : -INFINITY;
+          sv[i] = v;
+          mx = fmaxf(mx, v);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < BKV; ++i) {
+          sv[i] *= p.scale_log2;
+          mx = fmaxf(mx, sv[i]);
+        }
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const bool need = (m_new - m_run > 8.0f) || (m_run == -INFINITY && m_new > -INFINITY);
+      bool waited_pv = false;
+      if (__any_sync(0xffffffffu, need)) {
+        const float factor = (m_new == -INFINITY) ? 1.0f : ex2(m_run - m_new);   // ex2(-inf) = 0
+        if (jj > 0) {
+          if (!mbar_wait(&s.pv_done[t], (jj - 1) & 1)) { ok = false; break; }
+          waited_pv = true;
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld_32x32b_x32(o_addr + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+            tmem_st_32x32b_x32(o_addr + c * 32, o);
+          }
+          tmem_wait_st();
+        }
+        l_run *= factor;
+        m_run = m_new;
+      }
+      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < BKV; ++i) {
+        sv[i] = ex2(sv[i] - m_use);
+        sum += sv[i];
+      }
+      l_run += sum;
+      if (jj > 0 && !waited_pv) {
+        if (!mbar_wait(&s.pv_done[t], (jj - 1) & 1)) { ok = false; break; }
+      }
+      // P -> shared memory, K-major 128-byte-swizzled rows (16-byte chunk c of row r sits at c ^ (r & 7))
+#pragma unroll
+      for (int c = 0; c < BKV / 8; ++c) {
+        uint4 w;
+        w.x = pack2(sv[c * 8 + 0], sv[c * 8 + 1]);
+        w.y = pack2(sv[c * 8 + 2], sv[c * 8 + 3]);
+        w.z = pack2(sv[c * 8 + 4], sv[c * 8 + 5]);
+        w.w = pack2(sv[c * 8 + 6], sv[c * 8 + 7]);
+        *reinterpret_cast<uint4*>(p_row + (c >> 3) * 16384 + (((c & 7) ^ sw) << 4)) = w;
+      }
+      // cache rows at positions >= kv_len may hold anything: zero them in the staged V tile so that
+      // 0 * garbage cannot poison the accumulator (only the last tile can contain such rows)
+      if (kv0 + BKV > p.kv_len) {
+        const int rv = 2 * jj + 1;
+        if (!mbar_wait(&s.kv_full[rv % STAGES], (rv / STAGES) & 1)) { ok = false; break; }
+        if (t == 0) {
+          for (int r = row; r < BKV; r += 128) {
+            if (kv0 + r >= p.kv_len) {
+              for (int c = 0; c < HD / 64; ++c) {
+                uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + r * 128);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) dst[q] = make_uint4(0, 0, 0, 0);
+              }
+            }
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(&s.p_ready[t]);
+    }
+    if (ok && !s.abort) {
+      if (!mbar_wait(&s.pv_done[t], (n_tiles - 1) & 1)) {
+        ok = false;
+      } else {
+        tc_fence_after();
+        const float inv = 1.0f / l_run;
+        const int seq_row = q_row0 + row;
+        const bool store = seq_row < p.seq_len;
+        bf16* out = p.out + ((int64_t)b * p.seq_len + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
+#pragma unroll 1
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld_32x32b_x32(o_addr + c * 32, o);
+          tmem_wait_ld();
+          if (store) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 w;
+              w.x = pack2(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
+              w.y = pack2(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
+              w.z = pack2(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
+              w.w = pack2(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
+              *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
+            }
+          }
+        }
+      }
+    }
+    if (!ok) POP_ABORT(s, status);
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (s.abort && threadIdx.x == 0) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let in-flight bulk copies land
+  }
+  __syncthreads();
+  if (warp == NQT * 4 + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int HD, int NQT>
+int launch_t(const AttnArgs& a, cudaStream_t stream) {
+  using C = AC<HD, NQT>;
+  AttnDev p;
+  p.out = a.out;
+  p.ldo = a.ldo;
+  p.block_table = a.block_table;
+  p.max_pages_per_seq = a.max_pages_per_seq;
+  p.page_size = a.page_size;
+  p.rows_per_load = a.page_size < C::BKV ? a.page_size : C::BKV;
+  p.seq_len = a.seq_len;
+  p.q_pos0 = a.q_pos0;
+  p.kv_len = a.kv_len;
+  p.n_q_heads = a.n_q_heads;
+  p.n_kv_heads = a.n_kv_heads;
+  p.window = a.window;
+  p.q_tiles = ceil_div(a.seq_len, 128);
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  if (C::BKV % p.rows_per_load) return POP_E_INVALID;
+
+  CUtensorMap tq, tk, tv;
+  // Q [batch*seq][heads][hd] (row stride ldq)
+  {
+    const uint64_t dims[5] = {(uint64_t)HD, (uint64_t)a.n_q_heads, (uint64_t)a.batch * a.seq_len, 1, 1};
+    const uint64_t str[4] = {(uint64_t)HD, (uint64_t)a.ldq, (uint64_t)a.ldq * a.batch * a.seq_len,
+                             (uint64_t)a.ldq * a.batch * a.seq_len};
+    const uint32_t box[5] = {64, 1, 128, 1, 1};
+    int rc = make_tmap_bf16_nd(&tq, a.q, 3, dims, str, box);
+    if (rc) return rc;
+  }
+  {
+    const uint64_t dims[5] = {(uint64_t)HD, (uint64_t)a.n_kv_heads, (uint64_t)a.page_size, (uint64_t)a.num_pages, 1};
+    const uint64_t str[4] = {(uint64_t)HD, (uint64_t)HD * a.n_kv_heads, (uint64_t)HD * a.n_kv_heads * a.page_size,
+                             (uint64_t)HD * a.n_kv_heads * a.page_size * a.num_pages};
+    const uint32_t box[5] = {64, 1, (uint32_t)p.rows_per_load, 1, 1};
+    int rc = make_tmap_bf16_nd(&tk, a.k_pool, 4, dims, str, box);
+    if (rc) return rc;
+    rc = make_tmap_bf16_nd(&tv, a.v_pool, 4, dims, str, box);
+    if (rc) return rc;
+  }
+  const size_t smem = sizeof(AttnSmem<HD, NQT>) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_kernel<HD, NQT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return POP_E_CUDA;
+    configured = true;
+  }
+  dim3 grid(p.q_tiles, a.n_q_heads / NQT, a.batch);
+  attn_kernel<HD, NQT><<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status_word());
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+}  // namespace
+
+int launch_attention(const AttnArgs& a, cudaStream_t stream) {
+  if (!a.q || !a.k_pool || !a.v_pool || !a.block_table || !a.out) return POP_E_INVALID;
+  if (a.batch < 1 || a.seq_len < 1 || a.kv_len < 1 || a.n_q_heads < 1 || a.n_kv_heads < 1) return POP_E_INVALID;
+  if (a.n_q_heads % a.n_kv_heads || a.page_size < 16 || a.page_size % 16 || a.ldq % 8 || a.ldo % 8)
+    return POP_E_INVALID;
+  if (a.q_pos0 + a.seq_len > a.kv_len) return POP_E_INVALID;
+  if ((int64_t)ceil_div(a.kv_len, a.page_size) > a.max_pages_per_seq) return POP_E_NOSPACE;
+  const bool pair = (a.n_q_heads / a.n_kv_heads) % 2 == 0;
+  switch (a.head_dim) {
+    case 64: return pair ? launch_t<64, 2>(a, stream) : launch_t<64, 1>(a, stream);
+    case 128: return pair ? launch_t<128, 2>(a, stream) : launch_t<128, 1>(a, stream);
+    case 256: return launch_t<256, 1>(a, stream);
+  }
+  return POP_E_INVALID;
+}
+
+}  // namespace pop

@@ -27,9 +27,10 @@ void reset_launch_count();
 // box = [1][box1][box0]; box0 must be 64 (128 bytes).
 int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
                       uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1);
-// 5-D bf16 tensor, used for the paged KV pools [layer][page][slot][head][hd].
-int make_tmap_bf16_5d(CUtensorMap* out, const void* base, const uint64_t dims[5], const uint64_t strides_elems[4],
-                      const uint32_t box[5]);
+// rank-`rank` (3..5) bf16 tensor, dims/strides/box given innermost first (strides in elements, for
+// dims 1..rank-1), 128-byte swizzle. Used for Q and for the paged KV pools [page][slot][head][hd].
+int make_tmap_bf16_nd(CUtensorMap* out, const void* base, int rank, const uint64_t dims[5],
+                      const uint64_t strides_elems[4], const uint32_t box[5]);
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -53,5 +54,65 @@ struct GemmArgs {
   int n_valid;      // EPI_GATED_BF16: number of valid output columns (d_ffn); others: ignored
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t stream);
+
+// ------------------------------------------------------------------------------------ attention
+// out[b][i][h][:] = softmax_j(q[b][i][h] . k[b][j][g(h)] / sqrt(hd)) v[b][j][g(h)] over cache positions
+// j <= q_pos0 + i (and j > q_pos0 + i - window when window > 0), g(h) = h * n_kv / n_q.
+struct AttnArgs {
+  const bf16* q; int64_t ldq;            // [batch*seq_len][ldq], head h at column h*head_dim
+  const bf16* k_pool; const bf16* v_pool; // one layer of the paged cache: [num_pages][page_size][n_kv][hd]
+  const int32_t* block_table;            // device [batch][max_pages_per_seq]
+  bf16* out; int64_t ldo;                // [batch*seq_len][ldo]
+  int batch, seq_len, q_pos0, kv_len;
+  int n_q_heads, n_kv_heads, head_dim;
+  int page_size, num_pages, max_pages_per_seq;
+  int window;
+};
+int launch_attention(const AttnArgs& a, cudaStream_t stream);
+
+// ------------------------------------------------------------------------------------ elementwise
+int launch_embed(const int32_t* tokens, const bf16* table, const bf16* embeds, float* x, int rows, int d, int vocab,
+                 cudaStream_t s);
+// out[g][row][:] = x[row][:] * rsqrt(mean(x[row]^2) + eps) * gain[g][:]; bf16 or fp32 output
+int launch_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_stride, void* out, int64_t ldo,
+                   int64_t out_group_stride, int rows, int d, int groups, float eps, bool out_f32, cudaStream_t s);
+// x[row][:] += rmsnorm(t[row][:]) * gain
+int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, const float* gain, int rows, int d,
+                        float eps, cudaStream_t s);
+// table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)), pos < n_pos, j < hd/2
+int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
+struct RopeArgs {
+  const float* in; int64_t ld_in; int64_t in_group_stride;   // fp32 rows [q heads | k heads | v heads] * hd
+  bf16* q_out; int64_t ldq;                                  // may be null when n_q == 0
+  bf16* k_pool; bf16* v_pool; int64_t pool_layer_stride;     // pools [layer][page][slot][n_kv][hd]
+  int layer0;                                                // cache layer (0-based) of group 0
+  const int32_t* block_table; int max_pages_per_seq; int page_size;
+  const float* q_gain; const float* k_gain; int64_t gain_group_stride;   // per-head norm gains or null
+  const float2* table;
+  int n_q, n_kv, hd;
+  int rows, rows_per_seq, rows_written, pos0, groups;
+  float eps;
+};
+int launch_rope_cache(const RopeArgs& a, cudaStream_t s);
+int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s);
+
+// ------------------------------------------------------------------------------------ boundary path
+struct GemvArgs {
+  const void* x; int64_t ldx; bool x_f32;    // [B][K] bf16 or fp32
+  const bf16* w; int64_t ldw;                // [N][K]
+  void* out; int64_t ldo;                    // mode 0: fp32 store; 2: fp32 +=; 3: gated -> bf16 [B][n_valid]
+  int B, N, K, mode, act, n_valid;
+};
+int launch_gemv(const GemvArgs& a, cudaStream_t s);
+struct DecAttnArgs {
+  const bf16* q; int64_t ldq;
+  const bf16* k_pool; const bf16* v_pool;    // one layer of the cache
+  const int32_t* block_table; int max_pages_per_seq; int page_size;
+  float* partial;                            // [batch][n_q][splits][hd + 2] fp32 scratch
+  bf16* out; int64_t ldo;
+  int batch, n_q, n_kv, head_dim, kv_len, window;
+};
+int decode_attn_splits(int kv_len, int window);
+int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);
 
 }  // namespace pop

@@ -72,10 +72,10 @@ int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_
   return r == CUDA_SUCCESS ? POP_OK : POP_E_CUDA;
 }
 
-int make_tmap_bf16_5d(CUtensorMap* out, const void* base, const uint64_t dims[5], const uint64_t strides_elems[4],
-                      const uint32_t box[5]) {
+int make_tmap_bf16_nd(CUtensorMap* out, const void* base, int rank, const uint64_t dims[5],
+                      const uint64_t strides_elems[4], const uint32_t box[5]) {
   EncodeTiledFn fn = encode_fn();
-  if (!fn) return POP_E_CUDA;
+  if (!fn || rank < 3 || rank > 5) return POP_E_CUDA;
   cuuint64_t d[5], st[4];
   cuuint32_t b[5], estr[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < 5; ++i) {
@@ -83,7 +83,7 @@ int make_tmap_bf16_5d(CUtensorMap* out, const void* base, const uint64_t dims[5]
     b[i] = box[i];
   }
   for (int i = 0; i < 4; ++i) st[i] = strides_elems[i] * 2;
-  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), d, st, b, estr,
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? POP_OK : POP_E_CUDA;
