@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the POP pruned-prefill path on B200.
+
+A step is one pop_prefill call (embedding, L_keep full layers over the prompt, the pruned layers'
+independent K/V projections, the boundary token through the deep layers, final norm + output
+head) on one batch of seeded synthetic input. Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1]
+                  [--seq-len S --batch B --l-keep L] [--impl reference]
+
+N > 1 (under torchrun): independent replicas, one prompt batch per GPU, no data-path collective
+("weak" scaling); time is the maximum over ranks.  --impl reference times the CPU oracle, as it
+stands, on a bounded slice of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import pop_synth as ps  # noqa: E402
+
+METRIC = "pop_prefill_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(ps.WORKLOADS))
+    ap.add_argument("--seq-len", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--l-keep", type=int, default=0)
+    ap.add_argument("--page-size", type=int, default=128)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def resolve_workload(a) -> ps.Workload:
+    wl = ps.WORKLOADS[a.workload]
+    n = a.seq_len or wl.seq_len
+    nv = min(wl.n_visual, n - 1) if wl.n_visual else 0
+    return ps.Workload(wl.key, wl.model, a.batch or wl.batch, n, a.l_keep or wl.l_keep, nv)
+
+
+def load_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v == "Active":
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def replica_seed(rank: int) -> int:
+    """Prompt seed of replica `rank`: every replica works on its own batch of prompts."""
+    return ps.DEFAULT_SEED + 101 * rank
+
+
+def max_over_ranks(ms: float, device="cpu") -> float:
+    """Elapsed time of the slowest replica (all-reduce MAX when a process group is up)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def aggregate_tokens_per_s(tokens_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas timed by the slowest one."""
+    return tokens_per_replica * world / (ms_per_step * 1e-3)
+
+
+# ------------------------------------------------------------------------------------ CPU oracle legs
+
+class _CachedWeights:
+    def __init__(self, w):
+        self.w, self.c = w, {}
+
+    def get(self, name, layer=0):
+        if (name, layer) not in self.c:
+            self.c[(name, layer)] = self.w.get(name, layer)
+        return self.c[(name, layer)]
+
+    def embedding_rows(self, ids):
+        return self.w.embedding_rows(ids)
+
+
+def oracle_layer_sample(wl: ps.Workload, sample_tokens: int, repeats: int, warmup: int):
+    """Times the oracle's full decoder layer (layer 1, fp32) on the first `sample_tokens`
+    positions of the workload's first sequence. Returns the list of timed durations in s."""
+    from oracle import pop_oracle as po
+    cfg = wl.model
+    tokens, embeds = ps.make_prompt(wl)
+    w = _CachedWeights(ps.SynthWeights(cfg))
+    n = min(sample_tokens, wl.seq_len)
+    x = po.embed(cfg, w, tokens[0, :n], None if embeds is None else embeds[0, :n], torch.float32)
+    for name in ps.layer_tensor_shapes(cfg):
+        w.get(name, 1)
+    pos = torch.arange(n)
+    times = []
+    for i in range(warmup + repeats):
+        t0 = time.perf_counter()
+        po.layer_forward(cfg, w, 1, x, pos, None, None, torch.float32, "exact")
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    return times, n
+
+
+def run_reference(a, wl):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    sample = min(wl.seq_len, 2048)
+    times, n = oracle_layer_sample(wl, sample, a.steps, a.warmup)
+    t = sum(times) / len(times)
+    value = n * wl.batch / (wl.l_keep * t) / 1.0
+    cores = torch.get_num_threads()
+    desc = (f"oracle full decoder layer (fp32, torch CPU ops) on the first {n} of {wl.seq_len} positions; "
+            f"tokens/s = {n} / (L_keep={wl.l_keep} x layer time): kept stack only, extrapolated from one layer")
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": a.gpus,
+           "steps": a.steps, "warmup": a.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": workload_config(wl, a), "gpu_launches": 0,
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+def workload_config(wl, a):
+    cfg = wl.model
+    return {"workload": f"{wl.key}: {cfg.name}, L={cfg.n_layers}, batch {wl.batch} x {wl.seq_len} tokens"
+                        f"{' (' + str(wl.n_visual) + ' as embeddings)' if wl.n_visual else ''}, L_keep={wl.l_keep}",
+            "global_batch": wl.batch * max(1, a.gpus), "seq_len": wl.seq_len, "l_keep": wl.l_keep,
+            "page_size": a.page_size, "parallelism": f"replicas x{max(1, a.gpus)}",
+            "l2": "inputs larger than L2 (weights 2x params bytes stream every step)"}
+
+
+# ------------------------------------------------------------------------------------ GPU leg
+
+def run_ours(a, wl):
+    from oracle import pop_oracle as po   # cost model + cpu_baseline leg only
+    import paper_2602_03295_b200 as pk
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    cfg = wl.model
+    lib = pk.lib()
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+    tokens_h, embeds_h = ps.make_prompt(wl, replica_seed(rank))
+    tokens_h = tokens_h.pin_memory()
+    embeds_h = None if embeds_h is None else embeds_h.pin_memory()
+    tokens = tokens_h.to(dev)
+    embeds = None if embeds_h is None else embeds_h.to(dev)
+    cache = KVCache(cfg, wl.batch, wl.seq_len, a.page_size, device=dev)
+    logits = torch.empty(wl.batch, cfg.vocab, dtype=torch.float32, device=dev)
+    logits_h = torch.empty(wl.batch, cfg.vocab, dtype=torch.float32).pin_memory()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        model.prefill(tokens, embeds, wl.l_keep, cache, logits)
+
+    def step_e2e():
+        t = tokens_h.to(dev, non_blocking=True)
+        e = None if embeds_h is None else embeds_h.to(dev, non_blocking=True)
+        model.prefill(t, e, wl.l_keep, cache, logits)
+        logits_h.copy_(logits, non_blocking=True)
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1), dev)
+
+    for _ in range(max(a.warmup, 3)):
+        step()
+    sampler = ClockSampler(local if world > 1 else 0)
+    sampler.start()
+    total_ms = timed(step, a.steps)
+    clocks = sampler.stop()
+    status = model.last_status()
+    launches = model.last_launch_count()
+    ms_step = total_ms / a.steps
+    n_tok = wl.batch * wl.seq_len * world
+    value = aggregate_tokens_per_s(wl.batch * wl.seq_len, world, ms_step)
+
+    # end to end: host tokens (and embeddings) in, host logits out, copies inside the timed region
+    step_e2e()
+    e2e_ms = timed(step_e2e, a.steps) / a.steps
+    h2d = tokens_h.numel() * 4 + (0 if embeds_h is None else embeds_h.numel() * 2)
+    d2h = logits_h.numel() * 4
+
+    # the library's own full-depth prefill, for the speedup POP is about
+    def step_full():
+        model.full_prefill(tokens, embeds, cache, logits)
+    step_full()
+    full_ms = timed(step_full, max(2, a.steps // 2)) / max(2, a.steps // 2)
+
+    # per-kernel-class durations of one more step, CUDA events on the launching stream
+    lib.profile(True)
+    step()
+    torch.cuda.synchronize()
+    lib.profile(False)
+    prof = lib.profile_summary()
+    peaks = load_peaks()
+    gemm_ms, gemm_flops, gemm_n = prof["gemm"]
+    att_ms, att_flops, att_n = prof["attention"]
+    flops = po.prefill_flops(cfg, wl.batch, wl.seq_len, wl.l_keep)
+    peak_tf = peaks["bf16_tflops_sustained"]          # the GEMM runs inside a long step
+    achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    breakdown = {k: {"ms": round(v[0], 3), "launches": v[2]} for k, v in prof.items()}
+    breakdown["attention"]["tflops"] = round(att_flops / (att_ms * 1e-3) / 1e12, 1) if att_ms > 0 else None
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(a.warmup, 3),
+           "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16", "data": "synthetic", "config": workload_config(wl, a),
+           "ttft_ms": ms_step, "full_prefill_ms": full_ms, "speedup_vs_full_prefill": full_ms / ms_step,
+           "speedup_ceiling_flop_ratio": po.prefill_flops(cfg, wl.batch, wl.seq_len, None) / flops,
+           "algorithmic_tflop": flops / 1e12,
+           "path_tflops": flops / (ms_step * 1e-3) / 1e12,
+           "path_frac_of_measured_burst_peak": flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+           "path_frac_of_nominal_2250": flops / (ms_step * 1e-3) / 1e12 / 2250.0,
+           "device_status": status,
+           "clocks": clocks,
+           "e2e": {"value": n_tok / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+           "gpu_launches": int(launches * a.steps),
+           "roofline": {"kernel": "gemm_kernel (tcgen05 projection GEMM, all epilogues)", "bound": "tensor",
+                        "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                        "frac": achieved_tf / peak_tf if peak_tf else None,
+                        "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})",
+                        "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": None},
+           "kernel_breakdown": breakdown}
+    if rank == 0 and world == 1 and not a.no_cpu_baseline:
+        times, n = oracle_layer_sample(wl, min(wl.seq_len, 4096), 1, 0)
+        t = times[0]
+        out["cpu_baseline"] = {
+            "value": n * wl.batch / (wl.l_keep * t), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"one full decoder layer of the oracle (fp32) on the first {n} of {wl.seq_len} positions "
+                      f"took {t:.2f} s; tokens/s = {n} / (L_keep={wl.l_keep} x that): kept stack only, extrapolated"}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    a = parse_args()
+    wl = resolve_workload(a)
+    if a.impl == "reference":
+        run_reference(a, wl)
+    else:
+        run_ours(a, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -70,7 +70,8 @@ typedef struct {
  * k_pool, v_pool: bf16 [n_layers][num_pages][page_size][n_kv_heads][head_dim].
  * block_table:    device int32 [batch][max_pages_per_seq]; entry (b, j) is the page that holds
  *                 positions j*page_size .. (j+1)*page_size-1 of sequence b.
- * page_size must be a multiple of 16. Entries of a page beyond seq_len are left untouched. */
+ * page_size must be 16, 32, 64 or a multiple of 128, so that no 128-position attention tile
+ * straddles pages unevenly. Entries of a page beyond seq_len are left untouched. */
 typedef struct {
   void* k_pool;
   void* v_pool;

@@ -32,7 +32,7 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
  * over cache positions j <= q_pos0 + i, and j > q_pos0 + i - window when window > 0.
  * q: device bf16 [batch*seq_len][ldq] (head h at column h*hd); k_pool/v_pool: ONE layer of the
  * cache, bf16 [num_pages][page_size][n_kv][hd]; block_table as in pop_kv_cache_t; out: bf16
- * [batch*seq_len][ldo]. kv_len = valid cache positions (>= q_pos0 + seq_len). hd in {64,128,256}. */
+ * [batch*seq_len][ldo]. kv_len = valid cache positions (>= q_pos0 + seq_len). hd in {64,128,256}; page_size as in pop.h. */
 int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool, const int32_t* block_table,
                     void* out, int64_t ldo, int32_t batch, int32_t seq_len, int32_t q_pos0, int32_t kv_len,
                     int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t page_size, int32_t num_pages,
@@ -75,6 +75,14 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
 
 /* Synchronise the stream, then read and clear the library's device status word. */
 int pop_k_status(void* stream);
+
+/* Per-kernel timing for benchmarks. pop_k_profile(1) makes every launch of this library record a
+ * CUDA-event pair on its stream; pop_k_profile_summary waits for the recorded events of one kind
+ * (0 projection GEMM, 1 prefill attention, 2 elementwise, 3 GEMV, 4 decode attention), returns
+ * their summed duration in ms, their summed algorithmic work (flops for kinds 0-1, bytes
+ * otherwise) and their count, and forgets them. Off by default; costs nothing when off. */
+void pop_k_profile(int32_t enable);
+int pop_k_profile_summary(int32_t kind, double* total_ms, double* total_work, int64_t* launches);
 
 /* Kernel launches enqueued by this library since the last pop_k_reset_launch_count(). */
 int64_t pop_k_launch_count(void);

@@ -74,6 +74,8 @@ SIGNATURES = {
                          + [_I32] * 8 + [_F, _P]),
     "pop_k_gemv": (C.c_int, [_P, _I64, _I32, _P, _I64, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _I64] + [_I32] * 6 + [_P]),
+    "pop_k_profile": (None, [_I32]),
+    "pop_k_profile_summary": (C.c_int, [_I32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_I64)]),
     "pop_k_status": (C.c_int, [_P]),
     "pop_k_launch_count": (_I64, []),
     "pop_k_reset_launch_count": (None, []),
@@ -117,6 +119,21 @@ class PopLibrary:
 
     def reset_launch_count(self):
         self.dll.pop_k_reset_launch_count()
+
+    PROF_KINDS = ("gemm", "attention", "elementwise", "gemv", "decode_attention")
+
+    def profile(self, enable: bool):
+        self.dll.pop_k_profile(1 if enable else 0)
+
+    def profile_summary(self) -> dict:
+        """{kind: (total_ms, total_work, launches)} of the launches recorded since the last call."""
+        out = {}
+        for i, name in enumerate(self.PROF_KINDS):
+            ms, work, n = C.c_double(), C.c_double(), _I64()
+            self.check(self.dll.pop_k_profile_summary(i, C.byref(ms), C.byref(work), C.byref(n)),
+                       "pop_k_profile_summary")
+            out[name] = (ms.value, work.value, n.value)
+        return out
 
     # -------------------------------------------------------------- kernel-level calls
     def gemm(self, A: torch.Tensor, B: torch.Tensor, out: torch.Tensor, epilogue: int = 0, act: int = 0,

@@ -298,7 +298,7 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
   const pop_config_t& c = m->cfg;
   if (N < 1 || B < 1 || L_keep < 1 || L_keep > c.n_layers) return POP_E_INVALID;
   if ((int64_t)N * B > (int64_t)1 << 24) return POP_E_INVALID;
-  if (kc->page_size < 16 || kc->page_size % 16 || kc->num_pages < 1) return POP_E_INVALID;
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
   if ((int64_t)ceil_div(N, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
   if ((int64_t)ceil_div(N, kc->page_size) * B > kc->num_pages) return POP_E_NOSPACE;
   if (!m->ws) return POP_E_NOSPACE;

@@ -99,6 +99,10 @@ const char* pop_strerror(int status) {
 }
 
 int pop_k_status(void* stream) { return read_and_clear_status(static_cast<cudaStream_t>(stream)); }
+void pop_k_profile(int32_t enable) { prof_enable(enable != 0); }
+int pop_k_profile_summary(int32_t kind, double* total_ms, double* total_work, int64_t* launches) {
+  return prof_summary(kind, total_ms, total_work, launches);
+}
 int64_t pop_k_launch_count(void) { return launch_count(); }
 void pop_k_reset_launch_count(void) { reset_launch_count(); }
 

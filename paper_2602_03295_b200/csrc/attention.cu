@@ -425,6 +425,15 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
     configured = true;
   }
   dim3 grid(p.q_tiles, a.n_q_heads / NQT, a.batch);
+  // algorithmic work: 4 * hd flops per unmasked (query, key) pair and query head
+  double pairs = 0;
+  if (prof_enabled()) {
+    for (int r = 0; r < a.seq_len; ++r) {
+      const int pos = a.q_pos0 + r;
+      pairs += (a.window > 0 && a.window < pos + 1) ? a.window : pos + 1;
+    }
+  }
+  ProfScope prof(PROF_ATTENTION, 4.0 * HD * pairs * a.n_q_heads * a.batch, stream);
   attn_kernel<HD, NQT><<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status_word());
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
@@ -435,7 +444,7 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
 int launch_attention(const AttnArgs& a, cudaStream_t stream) {
   if (!a.q || !a.k_pool || !a.v_pool || !a.block_table || !a.out) return POP_E_INVALID;
   if (a.batch < 1 || a.seq_len < 1 || a.kv_len < 1 || a.n_q_heads < 1 || a.n_kv_heads < 1) return POP_E_INVALID;
-  if (a.n_q_heads % a.n_kv_heads || a.page_size < 16 || a.page_size % 16 || a.ldq % 8 || a.ldo % 8)
+  if (a.n_q_heads % a.n_kv_heads || !page_size_ok(a.page_size) || a.ldq % 8 || a.ldo % 8)
     return POP_E_INVALID;
   if (a.q_pos0 + a.seq_len > a.kv_len) return POP_E_INVALID;
   if ((int64_t)ceil_div(a.kv_len, a.page_size) > a.max_pages_per_seq) return POP_E_NOSPACE;

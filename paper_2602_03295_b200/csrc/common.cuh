@@ -22,6 +22,19 @@ void count_launch();
 int64_t launch_count();
 void reset_launch_count();
 
+// Optional per-kernel timing: when enabled, every launch wrapper brackets its kernel with CUDA
+// events on the launching stream; prof_summary() synchronises them and sums by kind.
+enum ProfKind { PROF_GEMM = 0, PROF_ATTENTION = 1, PROF_ELEMENTWISE = 2, PROF_GEMV = 3, PROF_DECODE_ATTN = 4,
+                PROF_KINDS = 5 };
+void prof_enable(bool on);
+bool prof_enabled();
+struct ProfScope {   // records the start event on construction, the end event on destruction
+  ProfScope(int kind, double work, cudaStream_t s);
+  ~ProfScope();
+  int kind; double work; cudaStream_t stream; cudaEvent_t e0, e1; bool active;
+};
+int prof_summary(int kind, double* total_ms, double* total_work, int64_t* launches);   // clears that kind
+
 // Tensor-map encoding through the driver entry point (no link-time dependency on libcuda).
 // 3-D bf16 tensor [dim2][dim1][dim0] with dim0 contiguous; strides in elements; 128-byte swizzle;
 // box = [1][box1][box0]; box0 must be 64 (128 bytes).
@@ -32,6 +45,8 @@ int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_
 int make_tmap_bf16_nd(CUtensorMap* out, const void* base, int rank, const uint64_t dims[5],
                       const uint64_t strides_elems[4], const uint32_t box[5]);
 
+// page sizes the attention tiles can walk: 16, 32, 64 or a multiple of 128 positions
+inline bool page_size_ok(int ps) { return ps == 16 || ps == 32 || ps == 64 || (ps >= 128 && ps % 128 == 0); }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

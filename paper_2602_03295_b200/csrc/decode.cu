@@ -273,6 +273,7 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
     p.ldo = a.ldo;
     p.B = a.B - b0 < GEMV_MAXB ? a.B - b0 : GEMV_MAXB;
     p.N = a.N; p.K = a.K; p.mode = a.mode; p.act = a.act; p.n_valid = a.n_valid;
+    ProfScope prof(PROF_GEMV, (double)a.N * a.K * 2, s);
     if (a.x_f32) gemv_kernel<true><<<blocks, 256, 0, s>>>(p);
     else gemv_kernel<false><<<blocks, 256, 0, s>>>(p);
     count_launch();
@@ -298,6 +299,8 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.splits = decode_attn_splits(a.kv_len, a.window);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)a.head_dim);
   dim3 grid(a.n_kv, p.splits, a.batch), grid2(a.n_q, a.batch);
+  const int span = (a.window > 0 && a.window < a.kv_len) ? a.window : a.kv_len;
+  ProfScope prof(PROF_DECODE_ATTN, (double)a.batch * span * a.n_kv * a.head_dim * 4, s);
   switch (a.head_dim) {
     case 64:
       dec_attn_kernel<64><<<grid, 128, 0, s>>>(p);

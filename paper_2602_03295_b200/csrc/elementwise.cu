@@ -220,6 +220,7 @@ __global__ void gather_rows_kernel(const float* __restrict__ src, float* __restr
 int launch_embed(const int32_t* tokens, const bf16* table, const bf16* embeds, float* x, int rows, int d, int vocab,
                  cudaStream_t s) {
   if (d % 8) return POP_E_INVALID;
+  ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 6, s);
   embed_kernel<<<rows, 256, 0, s>>>(tokens, table, embeds, x, d, vocab);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
@@ -230,6 +231,7 @@ int launch_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_
   if (d % 4 || ldx % 4 || ldo % 4 || rows < 1 || groups < 1) return POP_E_INVALID;
   dim3 grid(rows, groups);
   const int threads = d >= 2048 ? 256 : 128;
+  ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * (4.0 + groups * (out_f32 ? 4.0 : 2.0)), s);
   if (out_f32)
     rmsnorm_kernel<true><<<grid, threads, 0, s>>>(x, ldx, gain, gain_stride, out, ldo, out_group_stride, d, eps);
   else
@@ -241,6 +243,7 @@ int launch_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_
 int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, const float* gain, int rows, int d,
                         float eps, cudaStream_t s) {
   if (d % 4 || ldx % 4 || ldt % 4) return POP_E_INVALID;
+  ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 12, s);
   postnorm_add_kernel<<<rows, d >= 2048 ? 256 : 128, 0, s>>>(x, ldx, t, ldt, gain, d, eps);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
@@ -268,6 +271,7 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   const int heads = a.n_q + 2 * a.n_kv;
   const int64_t items = (int64_t)a.rows * heads;
   dim3 grid((unsigned)((items + 7) / 8), a.groups);
+  ProfScope prof(PROF_ELEMENTWISE, (double)items * a.groups * a.hd * 6, s);
   switch (a.hd) {
     case 64: rope_cache_kernel<64><<<grid, 256, 0, s>>>(p); break;
     case 128: rope_cache_kernel<128><<<grid, 256, 0, s>>>(p); break;

@@ -284,6 +284,7 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, i
       return POP_E_CUDA;
     configured = true;
   }
+  ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
   gemm_kernel<EPI><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status_word());
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;

@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 namespace pop {
 
@@ -40,6 +41,48 @@ static std::atomic<int64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 int64_t launch_count() { return g_launches.load(std::memory_order_relaxed); }
 void reset_launch_count() { g_launches.store(0, std::memory_order_relaxed); }
+
+struct ProfRecord { cudaEvent_t e0, e1; double work; };
+static std::atomic<bool> g_prof_on{false};
+static std::mutex g_prof_mu;
+static std::vector<ProfRecord> g_prof[PROF_KINDS];
+
+void prof_enable(bool on) { g_prof_on.store(on); }
+bool prof_enabled() { return g_prof_on.load(std::memory_order_relaxed); }
+
+ProfScope::ProfScope(int kind_, double work_, cudaStream_t s)
+    : kind(kind_), work(work_), stream(s), e0(nullptr), e1(nullptr), active(false) {
+  if (!prof_enabled()) return;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return;
+  active = true;
+  cudaEventRecord(e0, stream);
+}
+ProfScope::~ProfScope() {
+  if (!active) return;
+  cudaEventRecord(e1, stream);
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  g_prof[kind].push_back({e0, e1, work});
+}
+
+int prof_summary(int kind, double* total_ms, double* total_work, int64_t* launches) {
+  if (kind < 0 || kind >= PROF_KINDS) return POP_E_INVALID;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  double ms = 0, work = 0;
+  for (auto& r : g_prof[kind]) {
+    float t = 0;
+    if (cudaEventSynchronize(r.e1) != cudaSuccess || cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess)
+      return POP_E_CUDA;
+    ms += t;
+    work += r.work;
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  if (total_ms) *total_ms = ms;
+  if (total_work) *total_work = work;
+  if (launches) *launches = (int64_t)g_prof[kind].size();
+  g_prof[kind].clear();
+  return POP_OK;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

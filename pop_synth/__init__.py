@@ -69,21 +69,44 @@ def _hash_at(key: int, counter: torch.Tensor) -> torch.Tensor:
     return _mix(counter * _s64(_GOLDEN) + _s64(key))
 
 
-_CHUNK = 1 << 22
+_CHUNK = 1 << 20
+
+
+def _mix_(z: torch.Tensor, t: torch.Tensor) -> torch.Tensor:
+    """In-place splitmix64 finaliser; `t` is scratch of the same shape."""
+    for shift, mult in ((30, _M1), (27, _M2)):
+        torch.bitwise_right_shift(z, shift, out=t)
+        t.bitwise_and_((1 << (64 - shift)) - 1)
+        z.bitwise_xor_(t)
+        z.mul_(_s64(mult))
+    torch.bitwise_right_shift(z, 31, out=t)
+    t.bitwise_and_((1 << 33) - 1)
+    z.bitwise_xor_(t)
+    return z
 
 
 def _irwin_hall_int(key: int, start: int, count: int, device) -> torch.Tensor:
     """Centred sum of twelve 16-bit uniforms for elements [start, start+count): int64,
-    value = 2 * (sum - 12 * 32767.5), i.e. an even/odd-exact integer in [-786420, 786420]."""
+    value = 2 * (sum - 12 * 32767.5), an exact integer in [-786420, 786420]."""
     out = torch.empty(count, dtype=torch.int64, device=device)
     for c0 in range(0, count, _CHUNK):
         c1 = min(count, c0 + _CHUNK)
-        idx = torch.arange(start + c0, start + c1, dtype=torch.int64, device=device)
-        acc = torch.zeros(c1 - c0, dtype=torch.int64, device=device)
+        idx3 = torch.arange(start + c0, start + c1, dtype=torch.int64, device=device).mul_(3)
+        acc = out[c0:c1].zero_()
+        z = torch.empty_like(idx3)
+        t = torch.empty_like(idx3)
         for j in range(3):
-            h = _hash_at(key, idx * 3 + j)
-            acc += (h & 0xFFFF) + (_lsr(h, 16) & 0xFFFF) + (_lsr(h, 32) & 0xFFFF) + _lsr(h, 48)
-        out[c0:c1] = 2 * acc - 786420
+            torch.add(idx3, j, out=z)
+            z.mul_(_s64(_GOLDEN)).add_(_s64(key))
+            _mix_(z, t)
+            for sh in (0, 16, 32):
+                torch.bitwise_right_shift(z, sh, out=t)
+                t.bitwise_and_(0xFFFF)
+                acc.add_(t)
+            torch.bitwise_right_shift(z, 48, out=t)
+            t.bitwise_and_(0xFFFF)
+            acc.add_(t)
+        acc.mul_(2).sub_(786420)
     return out
 
 
