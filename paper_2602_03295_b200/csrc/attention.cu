@@ -46,6 +46,7 @@ struct __align__(1024) AttnSmem {
   uint64_t p_ready[NQT];
   uint64_t pv_done[NQT];
   uint32_t tmem_base;
+  uint32_t raised;
   volatile uint32_t abort;
 };
 
@@ -107,6 +108,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int j_lo = p.window > 0 ? max(0, pos0 - p.window + 1) / BKV : 0;
   const int n_tiles = j_hi - j_lo + 1;
 
+  if (status_raised(status, &s.raised)) return;
   if (threadIdx.x == 0) {
     mbar_init(&s.q_full, 1);
     for (int i = 0; i < STAGES; ++i) {
@@ -433,8 +435,10 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
       pairs += (a.window > 0 && a.window < pos + 1) ? a.window : pos + 1;
     }
   }
+  int* status = status_word();
+  if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_ATTENTION, 4.0 * HD * pairs * a.n_q_heads * a.batch, stream);
-  attn_kernel<HD, NQT><<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status_word());
+  attn_kernel<HD, NQT><<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

@@ -31,6 +31,7 @@ struct __align__(1024) GemmSmem {
   uint64_t tfull[2];
   uint64_t tempty[2];
   uint32_t tmem_base;
+  uint32_t raised;
   volatile uint32_t abort;
 };
 
@@ -77,6 +78,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
   const int k_blocks = (p.K + BK - 1) / BK;
 
+  if (status_raised(status, &s.raised)) return;
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
       mbar_init(&s.full[i], 1);
@@ -284,8 +286,10 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, i
       return POP_E_CUDA;
     configured = true;
   }
+  int* status = status_word();
+  if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
-  gemm_kernel<EPI><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status_word());
+  gemm_kernel<EPI><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

@@ -44,14 +44,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait. try_wait itself blocks for a hardware time slice, so the cap of 2^22 polls is
-// seconds of wall time: far beyond any legitimate wait, short enough to hand the GPU back.
-constexpr uint32_t kWaitLimit = 1u << 22;
+// Bounded wait: polls in bursts and gives up once kWaitLimitNs of wall time have passed, which is
+// far beyond any legitimate wait and short enough to hand the GPU back promptly.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
   }
-  return false;
+}
+
+// A kernel of this library does nothing once the status word is raised: after one kernel gave up
+// on a wait, the launches queued behind it return at once instead of each running into its own
+// limit. Thread 0 samples the word, so every thread of the CTA takes the same branch.
+__device__ __forceinline__ bool status_raised(const int* status, uint32_t* flag_smem) {
+  if (threadIdx.x == 0) *flag_smem = (*reinterpret_cast<const volatile int*>(status) != 0) ? 1u : 0u;
+  __syncthreads();
+  return *reinterpret_cast<volatile uint32_t*>(flag_smem) != 0;
 }
 
 // ----------------------------------------------------------------------------- TMA
