@@ -33,6 +33,8 @@ import pop_synth as ps  # noqa: E402
 
 METRIC = "pop_prefill_tokens_per_s"
 UNIT = "tokens/s"
+KERNELS = ["gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down", "kvproj", "attention", "attention_local", "gemv_head",
+           "decode_attention", "rmsnorm", "rope_cache"]
 
 
 def parse_args():
@@ -47,6 +49,9 @@ def parse_args():
     ap.add_argument("--l-keep", type=int, default=0)
     ap.add_argument("--page-size", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", default="", choices=[""] + KERNELS,
+                    help="time ONE kernel of the path alone, at the workload's per-layer shape, through its "
+                         "kernel-level C-ABI entry point (a small case for profiling)")
     return ap.parse_args()
 
 
@@ -55,6 +60,22 @@ def resolve_workload(a) -> ps.Workload:
     n = a.seq_len or wl.seq_len
     nv = min(wl.n_visual, n - 1) if wl.n_visual else 0
     return ps.Workload(wl.key, wl.model, a.batch or wl.batch, n, a.l_keep or wl.l_keep, nv)
+
+
+# DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
+# summarised in profiles/gemm_kernel_down_proj_c2.md; valid only for the kernel source it was taken on.
+GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
+                "gemm_cu_sha256": "0cd292d5435b33e04aa27c8308810f12952a5fe6fa50a344301f45c389346823"}
+
+
+def gemm_traffic():
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "paper_2602_03295_b200", "csrc", "gemm.cu"), "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return GEMM_TRAFFIC["bytes_per_launch"] if sha == GEMM_TRAFFIC["gemm_cu_sha256"] else None
 
 
 def load_peaks():
@@ -314,7 +335,8 @@ def run_ours(a, wl):
                         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                         "frac": achieved_tf / peak_tf if peak_tf else None,
                         "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})",
-                        "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": None},
+                        "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": gemm_traffic(),
+                        "traffic_launch": GEMM_TRAFFIC["launch"]},
            "kernel_breakdown": breakdown}
     if rank == 0 and world == 1 and not a.no_cpu_baseline:
         times, n = oracle_layer_sample(wl, min(wl.seq_len, 4096), 1, 0)
@@ -329,10 +351,136 @@ def run_ours(a, wl):
         torch.distributed.destroy_process_group()
 
 
+def run_kernel(a, wl):
+    """One kernel alone at the workload's per-layer shape: W warm-up launches, K timed launches between
+    CUDA events on the launching stream. Every launch reads operands larger than L2 or, where they are
+    smaller, rotates through enough operand sets to exceed it."""
+    import paper_2602_03295_b200 as pk
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    lib = pk.lib()
+    cfg = wl.model
+    M, d, F, hd = wl.batch * wl.seq_len, cfg.d_model, cfg.d_ffn, cfg.head_dim
+    qd, kvd = cfg.n_q_heads * hd, cfg.n_kv_heads * hd
+    P = max(1, cfg.n_layers - wl.l_keep)
+    g = torch.Generator(device=dev).manual_seed(ps.DEFAULT_SEED)
+
+    def rnd(*shape, std=0.5, dtype=torch.bfloat16):
+        return (torch.randn(*shape, generator=g, device=dev, dtype=torch.float32) * std).to(dtype)
+
+    peaks = load_peaks()
+    k = a.kernel
+    bound, work, sets = "tensor", 0.0, 1
+    if k.startswith("gemm_") or k == "kvproj":
+        f_pad = (F + 127) // 128 * 128
+        shapes = {"gemm_qkv": (1, qd + 2 * kvd, d, 1), "gemm_o": (1, d, qd, 2), "gemm_gateup": (1, 2 * f_pad, d, 3),
+                  "gemm_down": (1, d, F, 2), "kvproj": (P, 2 * kvd, d, 1)}
+        G, N, K, epi = shapes[k]
+        A, B = rnd(G, M, K), rnd(G, N, K, std=0.02)
+        if epi == 3:
+            out = torch.zeros(G, M, F, dtype=torch.bfloat16, device=dev)
+        else:
+            out = torch.zeros(G, M, N, dtype=torch.float32, device=dev)
+        work = 2.0 * G * M * N * K
+
+        def launch(i):
+            lib.gemm(A if G > 1 else A[0], B if G > 1 else B[0], out if G > 1 else out[0], epilogue=epi, act=cfg.act,
+                     n_valid=F if epi == 3 else 0)
+    elif k in ("attention", "attention_local"):
+        from paper_2602_03295_b200.binding import KVCache
+        window = cfg.window if k == "attention_local" else 0
+        q = rnd(M, qd, std=1.0)
+        cache = KVCache(cfg.replace(n_layers=1), wl.batch, wl.seq_len, a.page_size, device=dev)
+        cache.k.copy_(rnd(*cache.k.shape, std=1.0))
+        cache.v.copy_(rnd(*cache.v.shape, std=1.0))
+        out = torch.zeros(M, qd, dtype=torch.bfloat16, device=dev)
+        N = wl.seq_len
+        pairs = N * (N + 1) / 2 if not window or window >= N else window * (window + 1) / 2 + (N - window) * window
+        work = 4.0 * hd * pairs * cfg.n_q_heads * wl.batch
+
+        def launch(i):
+            lib.attention(q, cache.k[0], cache.v[0], cache.block_table, out, wl.batch, N, N, cfg.n_q_heads,
+                          cfg.n_kv_heads, hd, a.page_size, window)
+    elif k == "gemv_head":
+        bound = "hbm"
+        W = rnd(cfg.vocab, d, std=0.02)
+        x = rnd(wl.batch, d, dtype=torch.float32)
+        out = torch.zeros(wl.batch, cfg.vocab, dtype=torch.float32, device=dev)
+        work = 2.0 * cfg.vocab * d
+
+        def launch(i):
+            lib.gemv(x, W, out, mode=0)
+    elif k == "decode_attention":
+        from paper_2602_03295_b200.binding import KVCache
+        bound = "hbm"
+        N = wl.seq_len
+        per_set = 4.0 * wl.batch * N * kvd
+        sets = int(2 * 126e6 // per_set) + 2
+        cache = KVCache(cfg.replace(n_layers=sets), wl.batch, N, a.page_size, device=dev)
+        cache.k.copy_(rnd(*cache.k.shape, std=1.0))
+        cache.v.copy_(rnd(*cache.v.shape, std=1.0))
+        q = rnd(wl.batch, qd, std=1.0)
+        out = torch.zeros(wl.batch, qd, dtype=torch.bfloat16, device=dev)
+        work = per_set
+
+        def launch(i):
+            lib.decode_attention(q, cache.k[i % sets], cache.v[i % sets], cache.block_table, out, cfg.n_q_heads,
+                                 cfg.n_kv_heads, hd, N, a.page_size, 0)
+    elif k == "rmsnorm":
+        bound = "hbm"
+        x = rnd(M, d, dtype=torch.float32)
+        gain = torch.ones(d, dtype=torch.float32, device=dev)
+        out = torch.zeros(M, d, dtype=torch.bfloat16, device=dev)
+        work = 6.0 * M * d
+
+        def launch(i):
+            lib.rmsnorm(x, gain, out, cfg.rms_eps)
+    else:   # rope_cache
+        from paper_2602_03295_b200.binding import KVCache
+        bound = "hbm"
+        N = wl.seq_len
+        x = rnd(M, qd + 2 * kvd, dtype=torch.float32)
+        cache = KVCache(cfg.replace(n_layers=1), wl.batch, N, a.page_size, device=dev)
+        table = torch.zeros(N, hd // 2, 2, dtype=torch.float32, device=dev)
+        lib.rope_table(table, N, hd, cfg.rope_theta)
+        q_out = torch.zeros(M, qd, dtype=torch.bfloat16, device=dev)
+        work = 6.0 * M * (qd + 2 * kvd)
+
+        def launch(i):
+            lib.rope_cache(x, q_out, cache.k, cache.v, 0, cache.block_table, a.page_size, None, None, table,
+                           cfg.n_q_heads, cfg.n_kv_heads, hd, N, N, 0, cfg.rms_eps)
+
+    for i in range(max(a.warmup, 3)):
+        launch(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(a.steps):
+        launch(i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / a.steps
+    assert lib.status() == 0
+    if bound == "tensor":
+        achieved, peak, unit = work / (ms * 1e-3) / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+    else:
+        achieved, peak, unit = work / (ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
+    print(json.dumps({"kernel": k, "config": workload_config(wl, a), "steps": a.steps, "warmup": max(a.warmup, 3),
+                      "ms_per_launch": ms, "operand_sets": sets,
+                      "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                                   "frac": achieved / peak, "peak_source": peaks["source"] + " burst"},
+                      "clocks": clocks}), flush=True)
+
+
 def main():
     a = parse_args()
     wl = resolve_workload(a)
-    if a.impl == "reference":
+    if a.kernel:
+        run_kernel(a, wl)
+    elif a.impl == "reference":
         run_reference(a, wl)
     else:
         run_ours(a, wl)
