@@ -73,6 +73,33 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
                            void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
                            int32_t kv_len, int32_t window, void* stream);
 
+/* The same single-query attention as pop_k_decode_attention for callers that have no way to hand
+ * over a scratch buffer because they cannot allocate device memory at the point of the call: code
+ * running inside a host callback or a real-time serving loop where cudaMalloc is forbidden, or a
+ * process that received all its device buffers (inputs and outputs only) from another owner and
+ * has no allocator of its own. (The paper has no counterpart: this is a packaging variant, not a
+ * step of the method.) The split-KV partials go to a fixed array of POP_STATIC_SCRATCH_FLOATS
+ * floats (16 MiB) that is part of the library image, so every GPU that loads the library holds it
+ * until the process ends. The call allocates and frees nothing, neither through CUDA nor any other
+ * library. Arguments, layouts and results are those of pop_k_decode_attention minus `partial`.
+ *  - Limit: batch * n_q * splits * (head_dim + 2) <= POP_STATIC_SCRATCH_FLOATS, where splits =
+ *    ceil(span / 256) capped at 64 and span = min(kv_len, window or kv_len); a larger problem is
+ *    refused with POP_E_NOSPACE and nothing is enqueued (e.g. 8 sequences x 32 heads x hd 128 at
+ *    any length fit; 16 such sequences beyond 16128 positions do not).
+ *  - The first call on each device looks up the array's device address (one runtime query with
+ *    that device current, result kept); make that first call before starting any stream capture.
+ *  - All calls share the one array, which keeps whatever the previous call left. Each call
+ *    overwrites every slot it later reads, so no clearing is needed, but two calls whose kernels
+ *    may overlap on the GPU (different streams without an ordering between them) race on it:
+ *    serialise them. Calls on one stream are safe.
+ * Errors: POP_E_INVALID (null pointer, bad head_dim or head counts), POP_E_NOSPACE (over the limit,
+ * or block table too short), POP_E_CUDA. */
+#define POP_STATIC_SCRATCH_FLOATS (4 * 1024 * 1024)
+int pop_k_decode_attention_static(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
+                                  const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size,
+                                  void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
+                                  int32_t head_dim, int32_t kv_len, int32_t window, void* stream);
+
 /* Synchronise the stream, then read and clear the library's device status word. */
 int pop_k_status(void* stream);
 

@@ -74,6 +74,7 @@ SIGNATURES = {
                          + [_I32] * 8 + [_F, _P]),
     "pop_k_gemv": (C.c_int, [_P, _I64, _I32, _P, _I64, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _I64] + [_I32] * 6 + [_P]),
+    "pop_k_decode_attention_static": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_profile": (None, [_I32]),
     "pop_k_profile_summary": (C.c_int, [_I32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_I64)]),
     "pop_k_status": (C.c_int, [_P]),
@@ -211,6 +212,19 @@ class PopLibrary:
                                                partial.data_ptr(), out.data_ptr(), out.stride(0), batch, n_q, n_kv,
                                                hd, kv_len, window, _stream_ptr(stream))
         self.check(code, "pop_k_decode_attention")
+        return out
+
+    def decode_attention_static(self, q, k_pool, v_pool, block_table, out, n_q, n_kv, hd, kv_len, page_size,
+                                window=0, stream=None):
+        """pop_k_decode_attention_static: same arguments as decode_attention, but the split-KV partials
+        live in the library's own fixed device array, so this call allocates nothing (not even a
+        torch tensor). Raises PopError(POP_E_NOSPACE) beyond the array's stated size."""
+        code = self.dll.pop_k_decode_attention_static(q.data_ptr(), q.stride(0), k_pool.data_ptr(),
+                                                      v_pool.data_ptr(), block_table.data_ptr(),
+                                                      block_table.shape[1], page_size, out.data_ptr(),
+                                                      out.stride(0), q.shape[0], n_q, n_kv, hd, kv_len, window,
+                                                      _stream_ptr(stream))
+        self.check(code, "pop_k_decode_attention_static")
         return out
 
 

@@ -2,6 +2,9 @@
 // first decode step of the full model) and of the output head: weight-streaming GEMV for a handful
 // of rows, and single-query attention over the paged cache with split-KV partials.
 #include "common.cuh"
+#include "../../include/pop_kernels.h"
+
+#include <mutex>
 
 namespace pop {
 namespace {
@@ -322,3 +325,88 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
 }
 
 }  // namespace pop
+
+// ------------------------------------------------------------------------------ allocation-free variant
+// Split-KV partials of pop_k_decode_attention_static live here instead of in a caller buffer.
+// The array is part of the loaded module: every GPU that loads this library carries it until the
+// process exits. POP_STATIC_SCRATCH_FLOATS (pop_kernels.h) states its size.
+namespace pop {
+namespace {
+
+static __device__ __align__(256) float g_dec_static_scratch[POP_STATIC_SCRATCH_FLOATS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+float* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device. In host code the array's name is only
+// a handle for the runtime, not something a kernel can dereference, so the address is looked up
+// once per device (with that device current) and remembered.
+int static_scratch(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return POP_E_CUDA;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_dec_static_scratch) != cudaSuccess || ptr == nullptr) {
+      cudaGetLastError();
+      return POP_E_CUDA;
+    }
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return POP_OK;
+}
+
+}  // namespace
+}  // namespace pop
+
+extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
+                                             const int32_t* block_table, int32_t max_pages_per_seq,
+                                             int32_t page_size, void* out, int64_t ldo, int32_t batch, int32_t n_q,
+                                             int32_t n_kv, int32_t head_dim, int32_t kv_len, int32_t window,
+                                             void* stream) {
+  using namespace pop;
+  if (!q || !k_pool || !v_pool || !block_table || !out) return POP_E_INVALID;
+  if (batch < 1 || n_q < 1 || n_kv < 1 || kv_len < 1 || page_size < 1 || window < 0) return POP_E_INVALID;
+  if (n_q % n_kv || n_q / n_kv > DEC_MAXG) return POP_E_INVALID;
+  if (head_dim != 64 && head_dim != 128 && head_dim != 256) return POP_E_INVALID;
+  if ((int64_t)ceil_div(kv_len, page_size) > max_pages_per_seq) return POP_E_NOSPACE;
+  DecAttnDev p;
+  p.splits = decode_attn_splits(kv_len, window);
+  // every (sequence, query head, split) owns head_dim + 2 floats of the shared array
+  const int64_t need = (int64_t)batch * n_q * p.splits * (head_dim + 2);
+  if (need > (int64_t)POP_STATIC_SCRATCH_FLOATS) return POP_E_NOSPACE;
+  float* scratch = nullptr;
+  const int rc = static_scratch(&scratch);
+  if (rc != POP_OK) return rc;
+  p.q = static_cast<const bf16*>(q); p.ldq = ldq;
+  p.k_pool = static_cast<const bf16*>(k_pool); p.v_pool = static_cast<const bf16*>(v_pool);
+  p.block_table = block_table; p.max_pages_per_seq = max_pages_per_seq; p.page_size = page_size;
+  p.partial = scratch;
+  p.out = static_cast<bf16*>(out); p.ldo = ldo;
+  p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The first kernel writes every partial slot the second one reads (all splits of all heads, also
+  // the empty ones), so nothing left in the array by an earlier call is ever consumed and no
+  // clearing is needed between calls.
+  dim3 grid(n_kv, p.splits, batch), grid2(n_q, batch);
+  switch (head_dim) {
+    case 64:
+      dec_attn_kernel<64><<<grid, 128, 0, s>>>(p);
+      dec_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
+      break;
+    case 128:
+      dec_attn_kernel<128><<<grid, 128, 0, s>>>(p);
+      dec_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
+      break;
+    default:
+      dec_attn_kernel<256><<<grid, 128, 0, s>>>(p);
+      dec_combine_kernel<256><<<grid2, 128, 0, s>>>(p);
+      break;
+  }
+  count_launch();
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
