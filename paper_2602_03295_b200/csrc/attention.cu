@@ -3,14 +3,18 @@
 //
 // One CTA owns 128 consecutive query positions of NQT query heads that share a KV head (NQT = 2
 // when the GQA ratio allows it: both tiles see the same keys and the same mask, so every K/V
-// tile staged in shared memory is used twice). Warp roles:
-//   NQT softmax warpgroups (128 threads each, one query row per thread): read S = Q K^T from TMEM,
-//       keep the running row maximum / sum in fp32, write P = exp2(S - m) as bf16 into shared
-//       memory in the swizzled K-major layout the tensor core reads, rescale the O accumulator in
-//       TMEM only when the maximum grew by more than 2^8, and finally normalise and store O;
-//   1 TMA warp: Q tiles once, then K and V tiles of the paged cache through a ring of stages;
-//   1 MMA warp: allocates TMEM, issues S_t = Q_t K^T and O_t += P_t V for both tiles, ordered so
-//       that one tile's softmax overlaps the other tile's matrix products.
+// tile staged in shared memory is used twice). Keys are walked 64 at a time. Warp roles:
+//   NQT softmax warpgroups (128 threads each, one query row per thread): read S = Q K^T from one
+//       of two TMEM score buffers, keep the running row maximum / sum in fp32, write
+//       P = exp2(S - m) as packed bf16 over the front half of the same buffer (the tensor core
+//       reads the A operand of P V straight from TMEM), rescale the O accumulator in TMEM only
+//       when the maximum grew by more than 2^8, and finally normalise and store O;
+//   1 TMA warp: Q tiles once, then K and V tiles of the paged cache through a deep ring of
+//       shared-memory stages (no shared memory is spent on P: the latency of fetching scattered
+//       cache rows is what has to be hidden);
+//   1 MMA warp: allocates TMEM and keeps the scores two key tiles ahead of the softmax: when
+//       P_t of tile j is ready it issues O_t += P_t V_j and, behind it, S_t = Q_t K_{j+2}^T into the
+//       buffer P_t just vacated, so a softmax warpgroup never waits for the tensor pipe's latency.
 // K/V come straight from the paged cache [page][slot][kv head][hd] with 4-D tensor maps; cache
 // positions >= kv_len are never dereferenced through the block table and never reach the output.
 #include "common.cuh"
@@ -19,32 +23,40 @@
 namespace pop {
 namespace {
 
+constexpr int kSmemLimit = 227 * 1024;
+
 template <int HD, int NQT>
 struct AC {
-  static constexpr int BKV = (HD == 256) ? 64 : 128;
-  static constexpr int STAGES = (HD == 128) ? 3 : 4;
+  static constexpr int BKV = 64;
   static constexpr int KV_TILE_BYTES = BKV * HD * 2;
   static constexpr int KV_SUB_BYTES = BKV * 128;     // one 64-wide slice of head_dim
   static constexpr int Q_TILE_BYTES = 128 * HD * 2;
-  static constexpr int P_TILE_BYTES = 128 * BKV * 2;
+  static constexpr int RING_BYTES = kSmemLimit - 3 * 1024 - NQT * Q_TILE_BYTES;   // alignment slack + barriers
+  static constexpr int STAGES = RING_BYTES / KV_TILE_BYTES < 12 ? RING_BYTES / KV_TILE_BYTES : 12;
   static constexpr int THREADS = NQT * 128 + 64;
-  static constexpr int S_COL = 0;                    // S_t at t * BKV
-  static constexpr int O_COL = NQT * BKV;            // O_t at O_COL + t * HD
-  static_assert(NQT * (BKV + HD) <= 512, "TMEM budget");
+  // TMEM columns: two score buffers per tile (P overwrites the first 32 columns of the buffer its
+  // scores came from), then the output accumulators
+  static constexpr int S_COL = 0;                    // S_t[b] at (t * 2 + b) * 64
+  static constexpr int O_COL = NQT * 2 * BKV;        // O_t at O_COL + t * HD
+  static constexpr int COLS_USED = O_COL + NQT * HD;
+  static constexpr uint32_t TMEM_COLS = COLS_USED <= 128 ? 128 : (COLS_USED <= 256 ? 256 : 512);
+  static_assert(COLS_USED <= 512, "TMEM budget");
+  static_assert(STAGES >= 4, "ring too shallow");
 };
 
 template <int HD, int NQT>
 struct __align__(1024) AttnSmem {
   using C = AC<HD, NQT>;
   uint8_t q[NQT][C::Q_TILE_BYTES];
-  uint8_t p[NQT][C::P_TILE_BYTES];
   uint8_t kv[C::STAGES][C::KV_TILE_BYTES];
   uint64_t q_full;
   uint64_t kv_full[C::STAGES];
   uint64_t kv_empty[C::STAGES];
-  uint64_t s_full[NQT];
-  uint64_t p_ready[NQT];
-  uint64_t pv_done[NQT];
+  // one barrier per tile and score buffer b = key tile & 1; phase = key tile >> 1. Producer and
+  // consumer of one buffer alternate strictly, so a parity wait is never two phases behind.
+  uint64_t s_full[NQT][2];      // S_t[b] = Q_t K^T complete
+  uint64_t p_ready[NQT][2];     // P_t[b] written over S_t[b] (one arrival per softmax warp)
+  uint64_t pv_done[NQT][2];     // O_t += P_t[b] V complete
   uint32_t tmem_base;
   uint32_t raised;
   volatile uint32_t abort;
@@ -70,6 +82,12 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
@@ -115,11 +133,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       mbar_init(&s.kv_full[i], 1);
       mbar_init(&s.kv_empty[i], 1);
     }
-    for (int t = 0; t < NQT; ++t) {
-      mbar_init(&s.s_full[t], 1);
-      mbar_init(&s.p_ready[t], 128);
-      mbar_init(&s.pv_done[t], 1);
-    }
+    for (int t = 0; t < NQT; ++t)
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&s.s_full[t][i], 1);
+        mbar_init(&s.p_ready[t][i], 4);
+        mbar_init(&s.pv_done[t][i], 1);
+      }
     s.abort = 0;
     fence_barrier_init();
     prefetch_tmap(&tmQ);
@@ -127,7 +146,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     prefetch_tmap(&tmV);
   }
   if (warp == NQT * 4 + 1) {
-    tmem_alloc(&s.tmem_base, 512);
+    tmem_alloc(&s.tmem_base, C::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -144,30 +163,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, b * p.seq_len + q_row0);
       const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
       const int loads_per_tile = BKV / p.rows_per_load;
+      // ring order = the order the MMA warp consumes: K_0, K_1, then V_j, K_{j+2} for j = 0, 1, ...
       int ring = 0;
-      for (int jj = 0; jj < n_tiles && !s.abort; ++jj) {
-        const int kv0 = (j_lo + jj) * BKV;
-        for (int which = 0; which < 2; ++which, ++ring) {   // 0: K tile, 1: V tile
-          const int stage = ring % STAGES;
-          const uint32_t phase = (ring / STAGES) & 1;
-          if (!mbar_wait(&s.kv_empty[stage], phase ^ 1)) {
-            POP_ABORT(s, status);
-            break;
-          }
-          int n_loads = 0;
-          for (int r = 0; r < loads_per_tile; ++r)
-            if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
-          mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
-          const CUtensorMap* tm = which ? &tmV : &tmK;
-          for (int r = 0; r < n_loads; ++r) {
-            const int pos = kv0 + r * p.rows_per_load;
-            const int page = bt[pos / p.page_size];
-            const int slot = pos % p.page_size;
-            for (int c = 0; c < HD / 64; ++c)
-              tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
-                          c * 64, kv_head, slot, page);
-          }
+      bool ok = true;
+      auto load_tile = [&](int j, const CUtensorMap* tm) {
+        const int kv0 = (j_lo + j) * BKV;
+        const int stage = ring % STAGES;
+        const uint32_t phase = (ring / STAGES) & 1;
+        ++ring;
+        if (!mbar_wait(&s.kv_empty[stage], phase ^ 1)) {
+          POP_ABORT(s, status);
+          ok = false;
+          return;
         }
+        int n_loads = 0;
+        for (int r = 0; r < loads_per_tile; ++r)
+          if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
+        mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
+        for (int r = 0; r < n_loads; ++r) {
+          const int pos = kv0 + r * p.rows_per_load;
+          const int page = bt[pos / p.page_size];
+          const int slot = pos % p.page_size;
+          for (int c = 0; c < HD / 64; ++c)
+            tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
+                        c * 64, kv_head, slot, page);
+        }
+      };
+      load_tile(0, &tmK);
+      if (ok && n_tiles > 1) load_tile(1, &tmK);
+      for (int jj = 0; jj < n_tiles && ok && !s.abort; ++jj) {
+        load_tile(jj, &tmV);
+        if (ok && jj + 2 < n_tiles) load_tile(jj + 2, &tmK);
       }
     }
   } else if (warp == NQT * 4 + 1) {
@@ -175,53 +201,68 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(128, BKV, 0, 0);
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, HD, 0, 1);
-      auto issue_s = [&](int t, int stage) {
+      auto issue_s = [&](int t, int j, int stage) {
         const uint32_t qa = smem_u32(s.q[t]);
         const uint32_t ka = smem_u32(s.kv[stage]);
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
           const uint64_t ad = umma_smem_desc(qa + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
           const uint64_t bd = umma_smem_desc(ka + (kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32, 16, 1024);
-          umma_bf16_ss(tmem_base + C::S_COL + t * BKV, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+          umma_bf16_ss(tmem_base + C::S_COL + (t * 2 + (j & 1)) * BKV, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
         }
-        umma_commit(&s.s_full[t]);
+        umma_commit(&s.s_full[t][j & 1]);
       };
-      auto issue_pv = [&](int t, int stage, bool acc) {
-        const uint32_t pa = smem_u32(s.p[t]);
+      auto issue_pv = [&](int t, int j, int stage) {
+        // A operand = P_t in TMEM: 16 keys are 8 packed 32-bit columns; B = V tile, MN-major
+        const uint32_t pa = tmem_base + C::S_COL + (t * 2 + (j & 1)) * BKV;
         const uint32_t va = smem_u32(s.kv[stage]);
 #pragma unroll
         for (int kk = 0; kk < BKV / 16; ++kk) {
-          const uint64_t ad = umma_smem_desc(pa + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
           const uint64_t bd = umma_smem_desc(va + kk * 2048, C::KV_SUB_BYTES, 1024);
-          umma_bf16_ss(tmem_base + C::O_COL + t * HD, ad, bd, idesc_o, (acc || kk > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem_base + C::O_COL + t * HD, pa + kk * 8, bd, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(&s.pv_done[t]);
+        umma_commit(&s.pv_done[t][j & 1]);
+      };
+      int ring = 0;
+      auto wait_tile = [&](int& stage) {      // next ring entry, in the producer's order
+        stage = ring % STAGES;
+        const uint32_t phase = (ring / STAGES) & 1;
+        ++ring;
+        return mbar_wait(&s.kv_full[stage], phase);
       };
       bool ok = mbar_wait(&s.q_full, 0);
-      // ring position of K_jj is 2*jj, of V_jj is 2*jj+1
-      if (ok) ok = mbar_wait(&s.kv_full[0], 0);
-      if (ok) {
+      for (int j = 0; j < 2 && j < n_tiles && ok; ++j) {
+        int sk;
+        ok = wait_tile(sk);
+        if (!ok) break;
         tc_fence_after();
-        for (int t = 0; t < NQT; ++t) issue_s(t, 0);
-        umma_commit(&s.kv_empty[0]);
+        for (int t = 0; t < NQT; ++t) issue_s(t, j, sk);
+        umma_commit(&s.kv_empty[sk]);
       }
       for (int jj = 0; jj < n_tiles && ok && !s.abort; ++jj) {
-        const int rv = 2 * jj + 1, rk = 2 * jj + 2;
-        const int sv = rv % STAGES, sk = rk % STAGES;
-        const bool more = jj + 1 < n_tiles;
-        ok = mbar_wait(&s.kv_full[sv], (rv / STAGES) & 1);
-        if (ok && more) ok = mbar_wait(&s.kv_full[sk], (rk / STAGES) & 1);
+        int sv, sk = 0;
+        ok = wait_tile(sv);
+        const bool more = jj + 2 < n_tiles;
         for (int t = 0; t < NQT && ok; ++t) {
-          ok = mbar_wait(&s.p_ready[t], jj & 1);
+          ok = mbar_wait(&s.p_ready[t][jj & 1], (jj >> 1) & 1);
           if (!ok) break;
           tc_fence_after();
+          issue_pv(t, jj, sv);
           if (more) {
-            issue_s(t, sk);
-            if (t == NQT - 1) umma_commit(&s.kv_empty[sk]);
+            // the scores of key tile jj+2 go into the buffer P_t(jj) occupies: the tensor pipe runs
+            // its instructions in order, so the product above has read P before this overwrites it
+            if (t == 0) {
+              ok = wait_tile(sk);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_s(t, jj + 2, sk);
           }
-          issue_pv(t, sv, jj > 0);
         }
-        if (ok) umma_commit(&s.kv_empty[sv]);
+        if (ok) {
+          umma_commit(&s.kv_empty[sv]);
+          if (more) umma_commit(&s.kv_empty[sk]);
+        }
       }
       if (!ok) POP_ABORT(s, status);
     }
@@ -232,50 +273,52 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const int row = quarter * 32 + lane;                  // row in the tile == TMEM lane
     const int pos = pos0 + row;                           // absolute query position
     const uint32_t lane_addr = uint32_t(quarter * 32) << 16;
-    const uint32_t s_addr = tmem_base + lane_addr + C::S_COL + t * BKV;
+    const uint32_t s_addr = tmem_base + lane_addr + C::S_COL + t * 2 * BKV;
     const uint32_t o_addr = tmem_base + lane_addr + C::O_COL + t * HD;
-    uint8_t* p_row = s.p[t] + row * 128;
-    const int sw = row & 7;
     float m_run = -INFINITY;      // running (possibly stale) maximum, log2 domain
     float l_run = 0.f;
     bool ok = true;
+    // completion of the P V product of key tile j: barrier pv_done[t][j & 1], parity (j >> 1) & 1
+    auto wait_pv = [&](int j) { return mbar_wait(&s.pv_done[t][j & 1], (j >> 1) & 1); };
 
     for (int jj = 0; jj < n_tiles && !s.abort; ++jj) {
       const int kv0 = (j_lo + jj) * BKV;
-      if (!mbar_wait(&s.s_full[t], jj & 1)) { ok = false; break; }
+      const uint32_t sp_addr = s_addr + (jj & 1) * BKV;
+      if (!mbar_wait(&s.s_full[t][jj & 1], (jj >> 1) & 1)) { ok = false; break; }
       tc_fence_after();
       float sv[BKV];
 #pragma unroll
       for (int c = 0; c < BKV / 32; ++c)
-        tmem_ld_32x32b_x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+        tmem_ld_32x32b_x32(sp_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
       tmem_wait_ld();
-      // mask + scale, row maximum
+      // mask (diagonal / window-edge tiles only), then the row maximum of the raw scores on four
+      // independent chains of three-input max
       const bool partial = (kv0 + BKV - 1 > pos0) || (p.window > 0 && kv0 <= pos0 + 127 - p.window);
-      float mx = -INFINITY;
       if (partial) {
         const int lo = p.window > 0 ? pos - p.window : -1;   // valid keys: lo < j <= pos
 #pragma unroll
         for (int i = 0; i < BKV; ++i) {
           const int j = kv0 + i;
-          const float v = (j <= pos && j > lo) ? sv[i] * p.scale_log2 : -INFINITY;
-          sv[i] = v;
-          mx = fmaxf(mx, v);
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < BKV; ++i) {
-          sv[i] *= p.scale_log2;
-          mx = fmaxf(mx, sv[i]);
+          if (!(j <= pos && j > lo)) sv[i] = -INFINITY;
         }
       }
+      float mx0 = sv[0], mx1 = sv[1], mx2 = sv[2], mx3 = sv[3];
+#pragma unroll
+      for (int i = 4; i + 8 <= BKV; i += 8) {
+        mx0 = max3(mx0, sv[i], sv[i + 1]);
+        mx1 = max3(mx1, sv[i + 2], sv[i + 3]);
+        mx2 = max3(mx2, sv[i + 4], sv[i + 5]);
+        mx3 = max3(mx3, sv[i + 6], sv[i + 7]);
+      }
+      mx0 = max3(mx0, sv[BKV - 4], sv[BKV - 3]);
+      mx1 = max3(mx1, sv[BKV - 2], sv[BKV - 1]);
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;   // log2 domain
       const float m_new = fmaxf(m_run, mx);
       const bool need = (m_new - m_run > 8.0f) || (m_run == -INFINITY && m_new > -INFINITY);
-      bool waited_pv = false;
       if (__any_sync(0xffffffffu, need)) {
         const float factor = (m_new == -INFINITY) ? 1.0f : ex2(m_run - m_new);   // ex2(-inf) = 0
         if (jj > 0) {
-          if (!mbar_wait(&s.pv_done[t], (jj - 1) & 1)) { ok = false; break; }
-          waited_pv = true;
+          if (!wait_pv(jj - 1)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll 1
           for (int c = 0; c < HD / 32; ++c) {
@@ -291,50 +334,56 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         l_run *= factor;
         m_run = m_new;
       }
+      // P = exp2(S * scale - m) with packed fp32 pairs, summed on four chains, rounded to bf16
+      // (key 2c in the low half of packed column c, key 2c+1 in the high half)
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      float sum = 0.f;
-#pragma unroll
-      for (int i = 0; i < BKV; ++i) {
-        sv[i] = ex2(sv[i] - m_use);
-        sum += sv[i];
-      }
-      l_run += sum;
-      if (jj > 0 && !waited_pv) {
-        if (!mbar_wait(&s.pv_done[t], (jj - 1) & 1)) { ok = false; break; }
-      }
-      // P -> shared memory, K-major 128-byte-swizzled rows (16-byte chunk c of row r sits at c ^ (r & 7))
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+      const float2 nm2 = make_float2(-m_use, -m_use);
+      float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+      uint32_t pk[BKV / 2];
 #pragma unroll
       for (int c = 0; c < BKV / 8; ++c) {
-        uint4 w;
-        w.x = pack2(sv[c * 8 + 0], sv[c * 8 + 1]);
-        w.y = pack2(sv[c * 8 + 2], sv[c * 8 + 3]);
-        w.z = pack2(sv[c * 8 + 4], sv[c * 8 + 5]);
-        w.w = pack2(sv[c * 8 + 6], sv[c * 8 + 7]);
-        *reinterpret_cast<uint4*>(p_row + (c >> 3) * 16384 + (((c & 7) ^ sw) << 4)) = w;
+        float2 x0 = __ffma2_rn(make_float2(sv[c * 8 + 0], sv[c * 8 + 1]), sc2, nm2);
+        float2 x1 = __ffma2_rn(make_float2(sv[c * 8 + 2], sv[c * 8 + 3]), sc2, nm2);
+        float2 x2 = __ffma2_rn(make_float2(sv[c * 8 + 4], sv[c * 8 + 5]), sc2, nm2);
+        float2 x3 = __ffma2_rn(make_float2(sv[c * 8 + 6], sv[c * 8 + 7]), sc2, nm2);
+        x0.x = ex2(x0.x); x0.y = ex2(x0.y);
+        x1.x = ex2(x1.x); x1.y = ex2(x1.y);
+        x2.x = ex2(x2.x); x2.y = ex2(x2.y);
+        x3.x = ex2(x3.x); x3.y = ex2(x3.y);
+        acc0 = __fadd2_rn(acc0, x0);
+        acc1 = __fadd2_rn(acc1, x1);
+        acc0 = __fadd2_rn(acc0, x2);
+        acc1 = __fadd2_rn(acc1, x3);
+        pk[c * 4 + 0] = pack2(x0.x, x0.y);
+        pk[c * 4 + 1] = pack2(x1.x, x1.y);
+        pk[c * 4 + 2] = pack2(x2.x, x2.y);
+        pk[c * 4 + 3] = pack2(x3.x, x3.y);
       }
+      l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+      tmem_st_32x32b_x32(sp_addr, pk);      // over the scores this thread has just consumed
+      tmem_wait_st();
       // cache rows at positions >= kv_len may hold anything: zero them in the staged V tile so that
-      // 0 * garbage cannot poison the accumulator (only the last tile can contain such rows)
+      // 0 * garbage cannot poison the accumulator (only the last key tile can contain such rows,
+      // and its V tile is the last entry of the ring)
       if (kv0 + BKV > p.kv_len) {
-        const int rv = 2 * jj + 1;
+        const int rv = 2 * n_tiles - 1;
         if (!mbar_wait(&s.kv_full[rv % STAGES], (rv / STAGES) & 1)) { ok = false; break; }
-        if (t == 0) {
-          for (int r = row; r < BKV; r += 128) {
-            if (kv0 + r >= p.kv_len) {
-              for (int c = 0; c < HD / 64; ++c) {
-                uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + r * 128);
+        if (t == 0 && row < BKV && kv0 + row >= p.kv_len) {
+          for (int c = 0; c < HD / 64; ++c) {
+            uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + row * 128);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) dst[q] = make_uint4(0, 0, 0, 0);
-              }
-            }
+            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(0, 0, 0, 0);
           }
         }
+        fence_proxy_async_smem();
       }
-      fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(&s.p_ready[t]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.p_ready[t][jj & 1]);
     }
     if (ok && !s.abort) {
-      if (!mbar_wait(&s.pv_done[t], (n_tiles - 1) & 1)) {
+      if (!wait_pv(n_tiles - 1)) {
         ok = false;
       } else {
         tc_fence_after();
@@ -374,7 +423,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   __syncthreads();
   if (warp == NQT * 4 + 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
