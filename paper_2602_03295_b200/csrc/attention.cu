@@ -171,7 +171,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int stage = ring % STAGES;
         const uint32_t phase = (ring / STAGES) & 1;
         ++ring;
-        if (!mbar_wait(&s.kv_empty[stage], phase ^ 1)) {
+        if (!mbar_wait_relaxed(&s.kv_empty[stage], phase ^ 1)) {
           POP_ABORT(s, status);
           ok = false;
           return;
@@ -201,26 +201,32 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(128, BKV, 0, 0);
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, HD, 0, 1);
+      // Operand descriptors are built once; per instruction only the 16-byte-granular start address
+      // in the low bits moves (all shared-memory offsets here stay far below the field's 256 KB).
+      uint64_t q_desc[NQT];
+      for (int t = 0; t < NQT; ++t) q_desc[t] = umma_smem_desc(smem_u32(s.q[t]), 16, 1024);
+      const uint64_t k_desc0 = umma_smem_desc(smem_u32(s.kv[0]), 16, 1024);                 // K-major
+      const uint64_t v_desc0 = umma_smem_desc(smem_u32(s.kv[0]), C::KV_SUB_BYTES, 1024);    // MN-major
       auto issue_s = [&](int t, int j, int stage) {
-        const uint32_t qa = smem_u32(s.q[t]);
-        const uint32_t ka = smem_u32(s.kv[stage]);
+        const uint64_t qd = q_desc[t];
+        const uint64_t kd = k_desc0 + uint64_t(stage * (C::KV_TILE_BYTES >> 4));
+        const uint32_t d = tmem_base + C::S_COL + (t * 2 + (j & 1)) * BKV;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint64_t ad = umma_smem_desc(qa + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
-          const uint64_t bd = umma_smem_desc(ka + (kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32, 16, 1024);
-          umma_bf16_ss(tmem_base + C::S_COL + (t * 2 + (j & 1)) * BKV, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+          const uint64_t ad = qd + uint64_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          const uint64_t bd = kd + uint64_t(((kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32) >> 4);
+          umma_bf16_ss(d, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(&s.s_full[t][j & 1]);
       };
       auto issue_pv = [&](int t, int j, int stage) {
         // A operand = P_t in TMEM: 16 keys are 8 packed 32-bit columns; B = V tile, MN-major
         const uint32_t pa = tmem_base + C::S_COL + (t * 2 + (j & 1)) * BKV;
-        const uint32_t va = smem_u32(s.kv[stage]);
+        const uint64_t vd = v_desc0 + uint64_t(stage * (C::KV_TILE_BYTES >> 4));
+        const uint32_t d = tmem_base + C::O_COL + t * HD;
 #pragma unroll
-        for (int kk = 0; kk < BKV / 16; ++kk) {
-          const uint64_t bd = umma_smem_desc(va + kk * 2048, C::KV_SUB_BYTES, 1024);
-          umma_bf16_ts(tmem_base + C::O_COL + t * HD, pa + kk * 8, bd, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
-        }
+        for (int kk = 0; kk < BKV / 16; ++kk)
+          umma_bf16_ts(d, pa + kk * 8, vd + uint64_t((kk * 2048) >> 4), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
         umma_commit(&s.pv_done[t][j & 1]);
       };
       int ring = 0;
@@ -228,9 +234,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         stage = ring % STAGES;
         const uint32_t phase = (ring / STAGES) & 1;
         ++ring;
-        return mbar_wait(&s.kv_full[stage], phase);
+        return mbar_wait_relaxed(&s.kv_full[stage], phase);
       };
-      bool ok = mbar_wait(&s.q_full, 0);
+      bool ok = mbar_wait_relaxed(&s.q_full, 0);
       for (int j = 0; j < 2 && j < n_tiles && ok; ++j) {
         int sk;
         ok = wait_tile(sk);
@@ -244,7 +250,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         ok = wait_tile(sv);
         const bool more = jj + 2 < n_tiles;
         for (int t = 0; t < NQT && ok; ++t) {
-          ok = mbar_wait(&s.p_ready[t][jj & 1], (jj >> 1) & 1);
+          ok = mbar_wait_relaxed(&s.p_ready[t][jj & 1], (jj >> 1) & 1);
           if (!ok) break;
           tc_fence_after();
           issue_pv(t, jj, sv);

@@ -61,6 +61,30 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   }
 }
 
+// The same bounded wait for single-thread roles (TMA producer, MMA issuer) that share a scheduler
+// with working warps: between polls the thread sleeps, so its spinning does not take issue slots
+// and shared-memory bandwidth from them.
+#ifndef POP_RELAX_NS
+#define POP_RELAX_NS 32
+#endif
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+  for (int i = 0; i < 4096; ++i) {
+    if (POP_RELAX_NS > 0) __nanosleep(POP_RELAX_NS);
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 1024; ++i) {
+      if (POP_RELAX_NS > 0) __nanosleep(POP_RELAX_NS);
+      if (mbar_try_wait(bar, parity)) return true;
+    }
+    if (clock64() - t0 > kWaitLimitCycles) return false;
+  }
+}
+
 // A kernel of this library does nothing once the status word is raised: after one kernel gave up
 // on a wait, the launches queued behind it return at once instead of each running into its own
 // limit. Thread 0 samples the word, so every thread of the CTA takes the same branch.
