@@ -1,0 +1,120 @@
+"""Parity at the full benchmark sizes (configs 2-4), in the launch configuration bench.py times
+(batch 1, page size 128, the workload's own L_keep), where the whole oracle is too slow to run.
+
+What is checked instead:
+  * sampled outputs the oracle computes one by one: layer 1's K and V at sampled positions depend
+    only on the embedding row of that position (Eq. 2), so the oracle's kv_generation gives them
+    directly;
+  * properties that hold at any size:
+      - keeping all layers is bitwise the full-depth prefill, and the kept layers' cache of the
+        pruned prefill is bitwise the full prefill's (Eq. 1-3 untouched for l <= L_keep);
+      - the first pruned layer's entries equal the full model's (its input is exact), positions < N-1;
+      - Eq. 14 / Eq. 15: every pruned layer projects the SAME state H. With unit norm gains (the
+        benchmark recipe) LN_l(H[i]) is one vector h for all pruned layers, so the V entries of
+        some pruned layers determine h by least squares (fp64, the oracle's weights), and h then
+        predicts the K entries (per-head K norm, RoPE by the oracle) and the remaining V entries of
+        the other pruned layers.  A pruned layer fed a different state, the wrong layer's weights,
+        a wrong position in RoPE or a misplaced cache row fails this.
+Tolerance: per tensor max|err| / max|ref| <= 2e-2, as everywhere for bf16 cache entries.
+"""
+import pytest
+import torch
+
+import pop_synth as ps
+from oracle import pop_oracle as po
+from tests.gpu_util import rel_err
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+KV_TOL = 2e-2
+
+
+def _sample_positions(n, count, seed):
+    g = torch.Generator().manual_seed(seed)
+    fixed = [0, 1, 63, 64, 127, 128, 129, n // 2 - 1, n // 2, n - 130, n - 129, n - 3, n - 2]
+    rnd = torch.randint(0, n - 1, (count,), generator=g).tolist()
+    return sorted({p for p in fixed + rnd if 0 <= p < n - 1})
+
+
+def _run(wl):
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    cfg = wl.model
+    tokens, embeds = ps.make_prompt(wl)
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
+    t = tokens.to(DEV)
+    e = None if embeds is None else embeds.to(DEV)
+    cp = KVCache(cfg, wl.batch, wl.seq_len, 128, fill=float("nan"))
+    lp = model.prefill(t, e, wl.l_keep, cp)
+    assert model.last_status() == 0
+    cf = KVCache(cfg, wl.batch, wl.seq_len, 128, fill=float("nan"))
+    lf = model.full_prefill(t, e, cf)
+    assert model.last_status() == 0
+    ca = KVCache(cfg, wl.batch, wl.seq_len, 128, fill=float("nan"))
+    la = model.prefill(t, e, cfg.n_layers, ca)
+    assert model.last_status() == 0
+    return tokens, embeds, (lp, cp), (lf, cf), (la, ca)
+
+
+@pytest.mark.parametrize("key", ["c2", "c3", "c4"])
+def test_full_size_config(key):
+    wl = ps.WORKLOADS[key]
+    cfg, N, Lk, L = wl.model, wl.seq_len, wl.l_keep, wl.model.n_layers
+    tokens, embeds, (lp, cp), (lf, cf), (la, ca) = _run(wl)
+    for lg in (lp, lf, la):
+        assert torch.isfinite(lg).all()
+
+    # L_keep = L is the full prefill, bit for bit (logits and every cache entry of the prompt)
+    assert not cfg.distinct_gains
+    assert torch.equal(la, lf)
+    for l in range(L):
+        ka, va = ca.gather(l)
+        kf, vf = cf.gather(l)
+        assert torch.equal(ka, kf) and torch.equal(va, vf), f"layer {l + 1}"
+    del ca, la
+    # kept layers: identical kernels on identical inputs
+    for l in range(Lk):
+        kp, vp = cp.gather(l)
+        kf, vf = cf.gather(l)
+        assert torch.equal(kp, kf) and torch.equal(vp, vf), f"kept layer {l + 1}"
+        assert torch.isfinite(kp.float()).all() and torch.isfinite(vp.float()).all()
+    # first pruned layer: its input is exact, so Eq. 14 gives the full model's entries (positions < N-1
+    # through the batched projection; position N-1 through the boundary path)
+    kp, vp = cp.gather(Lk)
+    kf, vf = cf.gather(Lk)
+    assert rel_err(kp, kf) <= 1e-2 and rel_err(vp, vf) <= 1e-2
+    # deeper pruned layers hold something else than the full model's entries (they see H, not x_l)
+    kp, _ = cp.gather(L - 1)
+    kf, _ = cf.gather(L - 1)
+    assert rel_err(kp[:, :-1], kf[:, :-1]) > 5e-2
+    del cf
+
+    # ---- layer 1 at sampled positions, by the oracle (fp64)
+    w = ps.SynthWeights(cfg)
+    pos = torch.tensor(_sample_positions(N, 24, 5) + [N - 1])
+    x1 = po.embed(cfg, w, tokens[0, pos], None if embeds is None else embeds[0, pos], torch.float64)
+    k_ref, v_ref = po.kv_generation(cfg, w, 1, x1, pos, torch.float64, "exact")
+    k1, v1 = cp.gather(0)
+    assert rel_err(k1[0, pos], k_ref) <= KV_TOL
+    assert rel_err(v1[0, pos], v_ref) <= KV_TOL
+
+    # ---- pruned layers project one common state (Eq. 14-15), at sampled positions < N-1
+    pos = torch.tensor(_sample_positions(N, 12, 6))
+    pruned = list(range(Lk + 1, L + 1))                       # 1-based
+    n_fit = min(len(pruned) - 1, -(-2 * cfg.d_model // cfg.kv_dim))   # >= 2x over-determined if possible
+    fit, rest = pruned[:n_fit], pruned[n_fit:]
+    assert n_fit * cfg.kv_dim > cfg.d_model and rest
+    A = torch.cat([w.get("wv", l).double() for l in fit])     # [n_fit * kv_dim, d]
+    Bv = torch.cat([cp.gather(l - 1)[1][0, pos].reshape(len(pos), -1).cpu().double() for l in fit], dim=1)
+    h = torch.linalg.lstsq(A, Bv.T).solution.T                # [S, d] ~ LN(H[i]) (unit gains)
+    fit_res = ((h @ A.T) - Bv).abs().max() / Bv.abs().max()
+    assert fit_res <= KV_TOL, f"V entries of the fit layers are not projections of one state: {fit_res}"
+    for l in pruned:
+        k_gpu, v_gpu = cp.gather(l - 1)
+        k_pre = (h @ w.get("wk", l).double().T).reshape(len(pos), cfg.n_kv_heads, cfg.head_dim)
+        if cfg.qk_norm:
+            k_pre = po.rmsnorm(k_pre, w.get("k_norm", l).double(), cfg.rms_eps)
+        k_pred = po.rope(k_pre, pos, cfg.rope_theta)
+        assert rel_err(k_gpu[0, pos], k_pred) <= KV_TOL, f"K of pruned layer {l}"
+        if l in rest:
+            v_pred = (h @ w.get("wv", l).double().T).reshape(len(pos), cfg.n_kv_heads, cfg.head_dim)
+            assert rel_err(v_gpu[0, pos], v_pred) <= KV_TOL, f"V of pruned layer {l}"
