@@ -52,58 +52,72 @@ struct GemvDev {
 };
 
 // Each warp owns GEMV_R weight rows (mode 3: GEMV_R gate rows and their up rows) and streams them
-// once with 16-byte loads; the few activation rows come through L1.
+// once with 16-byte loads, GEMV_U k-steps (8 or 16 loads per lane) in flight at a time; the few
+// activation rows come through L1. NB = activation rows handled (1, 2, 4 or 8).
+constexpr int GEMV_U = 4;
+
 template <bool X_F32>
+__device__ __forceinline__ void load_x8(const void* x, int64_t off, float (&xf)[8]) {
+  if (X_F32) {
+    const float* xp = reinterpret_cast<const float*>(x) + off;
+    const float4 a = *reinterpret_cast<const float4*>(xp);
+    const float4 c = *reinterpret_cast<const float4*>(xp + 4);
+    xf[0] = a.x; xf[1] = a.y; xf[2] = a.z; xf[3] = a.w;
+    xf[4] = c.x; xf[5] = c.y; xf[6] = c.z; xf[7] = c.w;
+  } else {
+    unpack8(*reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(x) + off), xf);
+  }
+}
+
+template <bool X_F32, int NB, bool GATED>
 __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  const bool gated = p.mode == 3;
   constexpr int R = GEMV_R;
-  const int n_out = gated ? p.N / 2 : p.N;        // logical output rows
+  constexpr int RW = GATED ? 2 * R : R;           // weight rows streamed per warp
+  const int n_out = GATED ? p.N / 2 : p.N;        // logical output rows
   const int o0 = warp * R;
   if (o0 >= n_out) return;
   // weight rows for output o: plain -> o; gated -> gate row (o/128)*256 + o%128, up row +128
-  const bf16* wr[R * 2];
+  const bf16* wr[RW];
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const int o = min(o0 + r, n_out - 1);
-    const int64_t row = gated ? (int64_t)(o >> 7) * 256 + (o & 127) : o;
+    const int64_t row = GATED ? (int64_t)(o >> 7) * 256 + (o & 127) : o;
     wr[r] = p.w + row * p.ldw;
-    wr[R + r] = p.w + (row + 128) * p.ldw;
+    if (GATED) wr[R + r] = p.w + (row + 128) * p.ldw;
   }
-  float acc[R * 2][GEMV_MAXB];
+  float acc[RW][NB];
 #pragma unroll
-  for (int r = 0; r < R * 2; ++r)
+  for (int r = 0; r < RW; ++r)
 #pragma unroll
-    for (int b = 0; b < GEMV_MAXB; ++b) acc[r][b] = 0.f;
+    for (int b = 0; b < NB; ++b) acc[r][b] = 0.f;
 
-  for (int k = lane * 8; k < p.K; k += 256) {
-    float wf[R * 2][8];
+  for (int k0 = lane * 8; k0 < p.K; k0 += 256 * GEMV_U) {
+    uint4 wraw[GEMV_U][RW];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-      unpack8(ld_stream(wr[r] + k), wf[r]);
-      if (gated) unpack8(ld_stream(wr[R + r] + k), wf[R + r]);
+    for (int u = 0; u < GEMV_U; ++u) {
+      const int k = k0 + u * 256;
+#pragma unroll
+      for (int r = 0; r < RW; ++r)
+        wraw[u][r] = (k < p.K) ? ld_stream(wr[r] + k) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
-    for (int b = 0; b < GEMV_MAXB; ++b) {
-      if (b < p.B) {
-        float xf[8];
-        if (X_F32) {
-          const float* xp = reinterpret_cast<const float*>(p.x) + (int64_t)b * p.ldx + k;
-          const float4 a = *reinterpret_cast<const float4*>(xp);
-          const float4 c = *reinterpret_cast<const float4*>(xp + 4);
-          xf[0] = a.x; xf[1] = a.y; xf[2] = a.z; xf[3] = a.w;
-          xf[4] = c.x; xf[5] = c.y; xf[6] = c.z; xf[7] = c.w;
-        } else {
-          unpack8(*reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(p.x) + (int64_t)b * p.ldx + k), xf);
-        }
+    for (int u = 0; u < GEMV_U; ++u) {
+      const int k = k0 + u * 256;
+      if (k < p.K) {
+        float wf[RW][8];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
+        for (int r = 0; r < RW; ++r) unpack8(wraw[u][r], wf[r]);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[r][b] = fmaf(wf[r][e], xf[e], acc[r][b]);
-          if (gated) {
+        for (int b = 0; b < NB; ++b) {
+          if (b < p.B) {
+            float xf[8];
+            load_x8<X_F32>(p.x, (int64_t)b * p.ldx + k, xf);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[R + r][b] = fmaf(wf[R + r][e], xf[e], acc[R + r][b]);
+            for (int r = 0; r < RW; ++r)
+#pragma unroll
+              for (int e = 0; e < 8; ++e) acc[r][b] = fmaf(wf[r][e], xf[e], acc[r][b]);
           }
         }
       }
@@ -112,10 +126,10 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 #pragma unroll
   for (int r = 0; r < R; ++r) {
 #pragma unroll
-    for (int b = 0; b < GEMV_MAXB; ++b) {
+    for (int b = 0; b < NB; ++b) {
       if (b < p.B) {
         float v = warp_sum(acc[r][b]);
-        float u = gated ? warp_sum(acc[R + r][b]) : 0.f;
+        float u = GATED ? warp_sum(acc[GATED ? R + r : r][b]) : 0.f;
         const int o = o0 + r;
         if (lane == 0 && o < n_out) {
           if (p.mode == 0) {
@@ -129,6 +143,14 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
       }
     }
   }
+}
+
+template <bool X_F32, bool GATED>
+void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
+  if (p.B <= 1) gemv_kernel<X_F32, 1, GATED><<<blocks, 256, 0, s>>>(p);
+  else if (p.B <= 2) gemv_kernel<X_F32, 2, GATED><<<blocks, 256, 0, s>>>(p);
+  else if (p.B <= 4) gemv_kernel<X_F32, 4, GATED><<<blocks, 256, 0, s>>>(p);
+  else gemv_kernel<X_F32, 8, GATED><<<blocks, 256, 0, s>>>(p);
 }
 
 // ------------------------------------------------------------------------------ decode attention
@@ -146,83 +168,137 @@ struct DecAttnDev {
 };
 
 constexpr int DEC_MAXG = 8;
+constexpr int DEC_UNROLL = 4;     // keys per lane group whose K and V loads are in flight together
 
 template <int HD>
-__global__ void __launch_bounds__(128) dec_attn_kernel(const DecAttnDev p) {
-  constexpr int PER = HD / 32;             // elements per lane
+struct DecCfg {
+  static constexpr int LPK = HD / 8;                   // lanes per key: each lane holds 8 elements (16 bytes)
+  static constexpr int KPW = 32 / LPK;                 // keys per warp per pass
+  static constexpr int WARPS = (HD == 256) ? 4 : 8;
+};
+
+template <int HD, int GMAX>
+__global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const DecAttnDev p) {
+  using C = DecCfg<HD>;
+  constexpr int LPK = C::LPK, KPW = C::KPW, WARPS = C::WARPS;
   const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
-  const int G = p.n_q / p.n_kv;
+  const int G = p.n_q / p.n_kv;   // <= GMAX
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPK;                          // which key of the pass this lane group reads
+  const int e0 = (lane % LPK) * 8;                     // first head_dim element of this lane
   const int lo = p.window > 0 ? max(0, p.kv_len - p.window) : 0;
   const int span = p.kv_len - lo;
   const int chunk = (span + p.splits - 1) / p.splits;
   const int j0 = lo + split * chunk;
   const int j1 = min(p.kv_len, j0 + chunk);
 
-  float qv[DEC_MAXG][PER];
+  float qv[GMAX][8];
 #pragma unroll
-  for (int g = 0; g < DEC_MAXG; ++g)
+  for (int g = 0; g < GMAX; ++g)
     if (g < G) {
-      const bf16* qp = p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + g) * HD + lane * PER;
+      float t[8];
+      unpack8(*reinterpret_cast<const uint4*>(p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + g) * HD + e0), t);
 #pragma unroll
-      for (int e = 0; e < PER; ++e) qv[g][e] = __bfloat162float(qp[e]) * p.scale_log2;
+      for (int e = 0; e < 8; ++e) qv[g][e] = t[e] * p.scale_log2;
     }
-  float m[DEC_MAXG], l[DEC_MAXG], o[DEC_MAXG][PER];
+  float m[GMAX], l[GMAX], o[GMAX][8];
 #pragma unroll
-  for (int g = 0; g < DEC_MAXG; ++g) {
+  for (int g = 0; g < GMAX; ++g) {
     m[g] = -INFINITY;
     l[g] = 0.f;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) o[g][e] = 0.f;
+    for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
   }
   const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
-  for (int j = j0 + warp; j < j1; j += 4) {
-    const int page = bt[j / p.page_size];
-    const int64_t off = (((int64_t)page * p.page_size + j % p.page_size) * p.n_kv + kvh) * HD + lane * PER;
-    float kf[PER], vf[PER];
+  constexpr int STRIDE = WARPS * KPW;                  // keys the CTA covers per pass
+  // the trip count depends on the warp only, never on the lane: every lane reaches the shuffles
+  for (int jw = j0 + warp * KPW; jw < j1; jw += STRIDE * DEC_UNROLL) {
+    const int jb = jw + sub;
+    uint4 kraw[DEC_UNROLL], vraw[DEC_UNROLL];
 #pragma unroll
-    for (int e = 0; e < PER; ++e) {
-      kf[e] = __bfloat162float(p.k_pool[off + e]);
-      vf[e] = __bfloat162float(p.v_pool[off + e]);
+    for (int u = 0; u < DEC_UNROLL; ++u) {
+      const int j = jb + u * STRIDE;
+      kraw[u] = make_uint4(0, 0, 0, 0);
+      vraw[u] = make_uint4(0, 0, 0, 0);
+      if (j < j1) {
+        const int page = bt[j / p.page_size];
+        const int64_t off = (((int64_t)page * p.page_size + j % p.page_size) * p.n_kv + kvh) * HD + e0;
+        kraw[u] = ld_stream(p.k_pool + off);
+        vraw[u] = ld_stream(p.v_pool + off);
+      }
     }
 #pragma unroll
-    for (int g = 0; g < DEC_MAXG; ++g)
-      if (g < G) {
-        float s = 0.f;
+    for (int u = 0; u < DEC_UNROLL; ++u) {
+      const bool valid = jb + u * STRIDE < j1;   // uniform within a lane group
+      {
+        float kf[8], vf[8];
+        unpack8(kraw[u], kf);
+        unpack8(vraw[u], vf);
 #pragma unroll
-        for (int e = 0; e < PER; ++e) s = fmaf(qv[g][e], kf[e], s);
-        s = warp_sum(s);
-        const float mn = fmaxf(m[g], s);
-        const float f = exp2f(m[g] - mn);      // exp2f(-inf) = 0 on the first key
-        const float pj = exp2f(s - mn);
-        // the probability meets V as bf16, as it does in the prefill kernel's P.V product
-        const float pr = __bfloat162float(__float2bfloat16_rn(pj));
-        l[g] = l[g] * f + pj;
+        for (int g = 0; g < GMAX; ++g)
+          if (g < G) {
+            float sc = 0.f;
 #pragma unroll
-        for (int e = 0; e < PER; ++e) o[g][e] = fmaf(pr, vf[e], o[g][e] * f);
+            for (int e = 0; e < 8; ++e) sc = fmaf(qv[g][e], kf[e], sc);
+#pragma unroll
+            for (int w = LPK / 2; w > 0; w >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, w);
+            if (!valid) sc = -INFINITY;            // a key past the chunk contributes nothing
+            const float mn = fmaxf(m[g], sc);
+            if (mn == -INFINITY) continue;         // nothing seen yet by this lane group
+            const float f = exp2f(m[g] - mn);      // exp2f(-inf) = 0 on the first key
+            const float pj = exp2f(sc - mn);
+            // the probability meets V as bf16, as it does in the prefill kernel's P.V product
+            const float pr = __bfloat162float(__float2bfloat16_rn(pj));
+            l[g] = l[g] * f + pj;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pr, vf[e], o[g][e] * f);
+            m[g] = mn;
+          }
+      }
+    }
+  }
+  __syncwarp();
+  // merge the lane groups of a warp (they walked different keys), then the warps through shared memory
+#pragma unroll
+  for (int g = 0; g < GMAX; ++g)
+    if (g < G) {
+#pragma unroll
+      for (int w = LPK; w < 32; w <<= 1) {
+        const float mo = __shfl_xor_sync(0xffffffffu, m[g], w);
+        const float lo2 = __shfl_xor_sync(0xffffffffu, l[g], w);
+        const float mn = fmaxf(m[g], mo);
+        const float fa = (m[g] == -INFINITY) ? 0.f : exp2f(m[g] - mn);
+        const float fb = (mo == -INFINITY) ? 0.f : exp2f(mo - mn);
+        l[g] = l[g] * fa + lo2 * fb;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float oo = __shfl_xor_sync(0xffffffffu, o[g][e], w);
+          o[g][e] = o[g][e] * fa + oo * fb;
+        }
         m[g] = mn;
       }
-  }
-  // merge the 4 warps of the CTA through shared memory
-  __shared__ float sm_m[4][DEC_MAXG], sm_l[4][DEC_MAXG];
-  __shared__ float sm_o[4][DEC_MAXG][HD];
+    }
+  __shared__ float sm_m[WARPS][GMAX], sm_l[WARPS][GMAX];
+  __shared__ float sm_o[WARPS][GMAX][HD];
 #pragma unroll
-  for (int g = 0; g < DEC_MAXG; ++g)
+  for (int g = 0; g < GMAX; ++g)
     if (g < G) {
       if (lane == 0) {
         sm_m[warp][g] = m[g];
         sm_l[warp][g] = l[g];
       }
+      if (sub == 0) {
 #pragma unroll
-      for (int e = 0; e < PER; ++e) sm_o[warp][g][lane * PER + e] = o[g][e];
+        for (int e = 0; e < 8; ++e) sm_o[warp][g][e0 + e] = o[g][e];
+      }
     }
   __syncthreads();
   for (int idx = threadIdx.x; idx < G * HD; idx += blockDim.x) {
     const int g = idx / HD, e = idx - g * HD;
     float mm = -INFINITY;
-    for (int w = 0; w < 4; ++w) mm = fmaxf(mm, sm_m[w][g]);
+    for (int w = 0; w < WARPS; ++w) mm = fmaxf(mm, sm_m[w][g]);
     float ll = 0.f, oo = 0.f;
-    for (int w = 0; w < 4; ++w) {
+    for (int w = 0; w < WARPS; ++w) {
       const float f = (sm_m[w][g] == -INFINITY) ? 0.f : exp2f(sm_m[w][g] - mm);
       ll += sm_l[w][g] * f;
       oo += sm_o[w][g][e] * f;
@@ -237,23 +313,45 @@ __global__ void __launch_bounds__(128) dec_attn_kernel(const DecAttnDev p) {
 }
 
 template <int HD>
+void launch_dec_attn(const DecAttnDev& p, dim3 grid, int G, cudaStream_t s) {
+  constexpr int T = DecCfg<HD>::WARPS * 32;
+  if (G <= 1) dec_attn_kernel<HD, 1><<<grid, T, 0, s>>>(p);
+  else if (G <= 2) dec_attn_kernel<HD, 2><<<grid, T, 0, s>>>(p);
+  else if (G <= 4) dec_attn_kernel<HD, 4><<<grid, T, 0, s>>>(p);
+  else dec_attn_kernel<HD, 8><<<grid, T, 0, s>>>(p);
+}
+
+template <int HD>
 __global__ void dec_combine_kernel(const DecAttnDev p) {
+  // one CTA per (head, sequence); splits <= 64. The split weights exp2(m_s - max m) are computed
+  // once (thread s handles split s), then every thread sums its output elements over the splits
+  // with independent loads.
+  __shared__ float wgt[64];
+  __shared__ float inv_l;
   const int h = blockIdx.x, b = blockIdx.y;
   const float* src = p.partial + ((int64_t)b * p.n_q + h) * p.splits * (HD + 2);
-  float mm = -INFINITY;
-  for (int s = 0; s < p.splits; ++s) mm = fmaxf(mm, src[s * (HD + 2)]);
-  float ll = 0.f;
-  for (int s = 0; s < p.splits; ++s) {
-    const float ms = src[s * (HD + 2)];
-    if (ms > -INFINITY) ll += src[s * (HD + 2) + 1] * exp2f(ms - mm);
+  if (threadIdx.x < 32) {
+    const int s0 = threadIdx.x, s1 = threadIdx.x + 32;
+    const float m0 = s0 < p.splits ? src[s0 * (HD + 2)] : -INFINITY;
+    const float m1 = s1 < p.splits ? src[s1 * (HD + 2)] : -INFINITY;
+    const float l0 = s0 < p.splits ? src[s0 * (HD + 2) + 1] : 0.f;
+    const float l1 = s1 < p.splits ? src[s1 * (HD + 2) + 1] : 0.f;
+    float mm = fmaxf(m0, m1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+    const float w0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mm);
+    const float w1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
+    wgt[s0] = w0;
+    wgt[s1] = w1;
+    const float ll = warp_sum(l0 * w0 + l1 * w1);
+    if (threadIdx.x == 0) inv_l = 1.0f / ll;
   }
+  __syncthreads();
   for (int e = threadIdx.x; e < HD; e += blockDim.x) {
     float oo = 0.f;
-    for (int s = 0; s < p.splits; ++s) {
-      const float ms = src[s * (HD + 2)];
-      if (ms > -INFINITY) oo += src[s * (HD + 2) + 2 + e] * exp2f(ms - mm);
-    }
-    p.out[(int64_t)b * p.ldo + (int64_t)h * HD + e] = __float2bfloat16_rn(oo / ll);
+#pragma unroll 8
+    for (int s = 0; s < p.splits; ++s) oo = fmaf(src[s * (HD + 2) + 2 + e], wgt[s], oo);
+    p.out[(int64_t)b * p.ldo + (int64_t)h * HD + e] = __float2bfloat16_rn(oo * inv_l);
   }
 }
 
@@ -277,8 +375,13 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
     p.B = a.B - b0 < GEMV_MAXB ? a.B - b0 : GEMV_MAXB;
     p.N = a.N; p.K = a.K; p.mode = a.mode; p.act = a.act; p.n_valid = a.n_valid;
     ProfScope prof(PROF_GEMV, (double)a.N * a.K * 2, s);
-    if (a.x_f32) gemv_kernel<true><<<blocks, 256, 0, s>>>(p);
-    else gemv_kernel<false><<<blocks, 256, 0, s>>>(p);
+    if (a.mode == 3) {
+      if (a.x_f32) launch_gemv_nb<true, true>(p, blocks, s);
+      else launch_gemv_nb<false, true>(p, blocks, s);
+    } else {
+      if (a.x_f32) launch_gemv_nb<true, false>(p, blocks, s);
+      else launch_gemv_nb<false, false>(p, blocks, s);
+    }
     count_launch();
   }
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
@@ -306,15 +409,15 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   ProfScope prof(PROF_DECODE_ATTN, (double)a.batch * span * a.n_kv * a.head_dim * 4, s);
   switch (a.head_dim) {
     case 64:
-      dec_attn_kernel<64><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<64>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
       break;
     case 128:
-      dec_attn_kernel<128><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<128>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
       break;
     case 256:
-      dec_attn_kernel<256><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<256>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<256><<<grid2, 128, 0, s>>>(p);
       break;
     default: return POP_E_INVALID;
@@ -394,15 +497,15 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   dim3 grid(n_kv, p.splits, batch), grid2(n_q, batch);
   switch (head_dim) {
     case 64:
-      dec_attn_kernel<64><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<64>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
       break;
     case 128:
-      dec_attn_kernel<128><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<128>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
       break;
     default:
-      dec_attn_kernel<256><<<grid, 128, 0, s>>>(p);
+      launch_dec_attn<256>(p, grid, p.n_q / p.n_kv, s);
       dec_combine_kernel<256><<<grid2, 128, 0, s>>>(p);
       break;
   }
