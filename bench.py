@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--l-keep", type=int, default=0)
     ap.add_argument("--page-size", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="config-5 sweep on the workload's model shape: prompt length x batch x L_keep/L, one "
+                         "JSON line per point (POP vs full-depth prefill, tokens/s, TTFT, path TFLOP/s)")
     ap.add_argument("--kernel", default="", choices=[""] + KERNELS,
                     help="time ONE kernel of the path alone, at the workload's per-layer shape, through its "
                          "kernel-level C-ABI entry point (a small case for profiling)")
@@ -475,10 +478,62 @@ def run_kernel(a, wl):
                       "clocks": clocks}), flush=True)
 
 
+def run_sweep(a, wl0):
+    """Prompt length {512, 2048, 8192, 32768} x batch {1, 4, 8} (at most 64K tokens in total) x
+    L_keep/L in {1, 0.875, 0.75, 0.625} on one loaded model. Every point: 3 warm-up calls, then
+    `--steps` calls between CUDA events. Weights (2 bytes per parameter, far larger than L2) stream
+    on every call."""
+    from oracle import pop_oracle as po   # FLOP model only
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = wl0.model
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+    peaks = load_peaks()
+    L = cfg.n_layers
+    for n in (512, 2048, 8192, 32768):
+        for bsz in (1, 4, 8):
+            if n * bsz > 65536:
+                continue
+            tokens = ps.uniform_tokens(ps.DEFAULT_SEED + 1, bsz, n, cfg.vocab).to(dev)
+            cache = KVCache(cfg, bsz, n, a.page_size, device=dev)
+            logits = torch.empty(bsz, cfg.vocab, dtype=torch.float32, device=dev)
+            full_ms = None
+            for ratio in (1.0, 0.875, 0.75, 0.625):
+                lk = int(round(L * ratio))
+
+                def step():
+                    model.prefill(tokens, None, lk, cache, logits)
+                for _ in range(3):
+                    step()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(a.steps):
+                    step()
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / a.steps
+                assert model.last_status() == 0
+                if ratio == 1.0:
+                    full_ms = ms
+                flops = po.prefill_flops(cfg, bsz, n, lk)
+                print(json.dumps({
+                    "sweep": wl0.key, "seq_len": n, "batch": bsz, "l_keep": lk, "keep_ratio": ratio,
+                    "ttft_ms": ms, "tokens_per_s": bsz * n / (ms * 1e-3),
+                    "speedup_vs_full_depth": full_ms / ms,
+                    "speedup_ceiling_flop_ratio": po.prefill_flops(cfg, bsz, n, None) / flops,
+                    "path_tflops": flops / (ms * 1e-3) / 1e12,
+                    "frac_of_measured_burst_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}), flush=True)
+            del cache, tokens, logits
+
+
 def main():
     a = parse_args()
     wl = resolve_workload(a)
-    if a.kernel:
+    if a.sweep:
+        run_sweep(a, wl)
+    elif a.kernel:
         run_kernel(a, wl)
     elif a.impl == "reference":
         run_reference(a, wl)
