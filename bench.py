@@ -180,9 +180,12 @@ class _CachedWeights:
         return self.w.embedding_rows(ids)
 
 
-def oracle_layer_sample(wl: ps.Workload, sample_tokens: int, repeats: int, warmup: int):
-    """Times the oracle's full decoder layer (layer 1, fp32) on the first `sample_tokens`
-    positions of the workload's first sequence. Returns the list of timed durations in s."""
+def oracle_sample(wl: ps.Workload, sample_tokens: int, repeats: int, warmup: int):
+    """Times the oracle, as it stands (fp32, torch CPU ops), on a bounded slice of the workload: one
+    full decoder layer (layer 1) and one pruned layer's K/V generation (Eq. 14) on the first
+    `sample_tokens` positions of the first sequence, and the output head on one position. Returns
+    (per-step seconds for the slice extrapolated over the depth, n, parts): a "step" is
+    L_keep x layer + P x kv-projection + head."""
     from oracle import pop_oracle as po
     cfg = wl.model
     tokens, embeds = ps.make_prompt(wl)
@@ -191,27 +194,42 @@ def oracle_layer_sample(wl: ps.Workload, sample_tokens: int, repeats: int, warmu
     x = po.embed(cfg, w, tokens[0, :n], None if embeds is None else embeds[0, :n], torch.float32)
     for name in ps.layer_tensor_shapes(cfg):
         w.get(name, 1)
+    w.get("lm_head", 0), w.get("final_norm", 0)
     pos = torch.arange(n)
-    times = []
+    P = cfg.n_layers - wl.l_keep
+    steps = []
+    parts = {}
     for i in range(warmup + repeats):
         t0 = time.perf_counter()
         po.layer_forward(cfg, w, 1, x, pos, None, None, torch.float32, "exact")
+        t1 = time.perf_counter()
+        po.kv_generation(cfg, w, 1, x, pos, torch.float32, "exact")
+        t2 = time.perf_counter()
+        po.lm_logits(cfg, w, x[-1], torch.float32)
+        t3 = time.perf_counter()
         if i >= warmup:
-            times.append(time.perf_counter() - t0)
-    return times, n
+            steps.append(wl.l_keep * (t1 - t0) + P * (t2 - t1) + (t3 - t2))
+            parts = {"layer_s": t1 - t0, "kv_projection_s": t2 - t1, "head_s": t3 - t2}
+    return steps, n, parts
+
+
+def oracle_sample_text(wl, n, parts):
+    P = wl.model.n_layers - wl.l_keep
+    return (f"oracle (fp32, torch CPU ops) on the first {n} of {wl.seq_len} positions: one full decoder layer "
+            f"{parts['layer_s']:.2f} s, one pruned layer's K/V generation {parts['kv_projection_s']:.2f} s, output head "
+            f"{parts['head_s']:.3f} s; tokens/s = {n} x batch / (L_keep={wl.l_keep} x layer + {P} x kv + head), "
+            f"extrapolated over the depth from that slice (boundary-token pass not included)")
 
 
 def run_reference(a, wl):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    sample = min(wl.seq_len, 2048)
-    times, n = oracle_layer_sample(wl, sample, a.steps, a.warmup)
-    t = sum(times) / len(times)
-    value = n * wl.batch / (wl.l_keep * t) / 1.0
+    steps, n, parts = oracle_sample(wl, min(wl.seq_len, 2048), a.steps, min(a.warmup, 1))
+    t = sum(steps) / len(steps)
+    value = n * wl.batch / t
     cores = torch.get_num_threads()
-    desc = (f"oracle full decoder layer (fp32, torch CPU ops) on the first {n} of {wl.seq_len} positions; "
-            f"tokens/s = {n} / (L_keep={wl.l_keep} x layer time): kept stack only, extrapolated from one layer")
+    desc = oracle_sample_text(wl, n, parts)
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": a.gpus,
            "steps": a.steps, "warmup": a.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -342,12 +360,10 @@ def run_ours(a, wl):
                         "traffic_launch": GEMM_TRAFFIC["launch"]},
            "kernel_breakdown": breakdown}
     if rank == 0 and world == 1 and not a.no_cpu_baseline:
-        times, n = oracle_layer_sample(wl, min(wl.seq_len, 4096), 1, 0)
-        t = times[0]
-        out["cpu_baseline"] = {
-            "value": n * wl.batch / (wl.l_keep * t), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": f"one full decoder layer of the oracle (fp32) on the first {n} of {wl.seq_len} positions "
-                      f"took {t:.2f} s; tokens/s = {n} / (L_keep={wl.l_keep} x that): kept stack only, extrapolated"}
+        steps, n, parts = oracle_sample(wl, min(wl.seq_len, 4096), 3, 1)
+        t = sum(steps) / len(steps)
+        out["cpu_baseline"] = {"value": n * wl.batch / t, "unit": UNIT, "cores": torch.get_num_threads(),
+                               "kind": "oracle", "sample": oracle_sample_text(wl, n, parts)}
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
