@@ -198,7 +198,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     }
   } else if (warp == NQT * 4 + 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {
+      // the whole warp walks this role; one elected lane issues the tensor-core instructions
+      const uint32_t leader = elect_one();
       constexpr uint32_t idesc_s = umma_idesc_bf16(128, BKV, 0, 0);
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, HD, 0, 1);
       // Operand descriptors are built once; per instruction only the 16-byte-granular start address
@@ -215,9 +217,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         for (int kk = 0; kk < HD / 16; ++kk) {
           const uint64_t ad = qd + uint64_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
           const uint64_t bd = kd + uint64_t(((kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32) >> 4);
-          umma_bf16_ss(d, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+          umma_bf16_ss_w(leader, d, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
         }
-        umma_commit(&s.s_full[t][j & 1]);
+        umma_commit_w(leader, &s.s_full[t][j & 1]);
       };
       auto issue_pv = [&](int t, int j, int stage) {
         // A operand = P_t in TMEM: 16 keys are 8 packed 32-bit columns; B = V tile, MN-major
@@ -226,8 +228,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const uint32_t d = tmem_base + C::O_COL + t * HD;
 #pragma unroll
         for (int kk = 0; kk < BKV / 16; ++kk)
-          umma_bf16_ts(d, pa + kk * 8, vd + uint64_t((kk * 2048) >> 4), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
-        umma_commit(&s.pv_done[t][j & 1]);
+          umma_bf16_ts_w(leader, d, pa + kk * 8, vd + uint64_t((kk * 2048) >> 4), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        umma_commit_w(leader, &s.pv_done[t][j & 1]);
       };
       int ring = 0;
       auto wait_tile = [&](int& stage) {      // next ring entry, in the producer's order
@@ -243,7 +245,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         if (!ok) break;
         tc_fence_after();
         for (int t = 0; t < NQT; ++t) issue_s(t, j, sk);
-        umma_commit(&s.kv_empty[sk]);
+        umma_commit_w(leader, &s.kv_empty[sk]);
       }
       for (int jj = 0; jj < n_tiles && ok && !s.abort; ++jj) {
         int sv, sk = 0;
@@ -266,8 +268,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           }
         }
         if (ok) {
-          umma_commit(&s.kv_empty[sv]);
-          if (more) umma_commit(&s.kv_empty[sk]);
+          umma_commit_w(leader, &s.kv_empty[sv]);
+          if (more) umma_commit_w(leader, &s.kv_empty[sk]);
         }
       }
       if (!ok) POP_ABORT(s, status);
