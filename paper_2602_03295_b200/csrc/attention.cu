@@ -20,6 +20,8 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#include <type_traits>
+
 namespace pop {
 namespace {
 
@@ -435,9 +437,372 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Variant for head_dim <= 128: the scores of TWO consecutive 64-key tiles are produced by one set of
+// 128-wide tensor-core instructions (a 64-wide instruction occupies the pipe as long as a 128-wide
+// one), into the two adjacent score buffers of the tile. The softmax and the P V products still
+// work on 64 keys at a time, so P V of the first half runs while the second half is in the softmax.
+// K and V travel in 128-key stages. The next pair's scores can only be issued once both halves'
+// P have been consumed; the other query tile's work fills the tensor pipe in the meantime.
 template <int HD, int NQT>
+struct PC {
+  static constexpr int BKV = 64;                       // softmax / P V granularity
+  static constexpr int PKV = 128;                      // keys per stage and per score instruction set
+  static constexpr int KV_TILE_BYTES = PKV * HD * 2;
+  static constexpr int KV_SUB_BYTES = PKV * 128;       // one 64-wide slice of head_dim
+  static constexpr int Q_TILE_BYTES = 128 * HD * 2;
+  static constexpr int RING_BYTES = kSmemLimit - 3 * 1024 - NQT * Q_TILE_BYTES;
+  static constexpr int STAGES = RING_BYTES / KV_TILE_BYTES < 8 ? RING_BYTES / KV_TILE_BYTES : 8;
+  static constexpr int THREADS = NQT * 128 + 64;
+  static constexpr int S_COL = 0;                      // S_t[h] at (t * 2 + h) * 64, h = half of the pair
+  static constexpr int O_COL = NQT * 2 * BKV;
+  static constexpr int COLS_USED = O_COL + NQT * HD;
+  static constexpr uint32_t TMEM_COLS = COLS_USED <= 128 ? 128 : (COLS_USED <= 256 ? 256 : 512);
+  static_assert(COLS_USED <= 512, "TMEM budget");
+  static_assert(STAGES >= 4, "ring too shallow");
+};
+
+template <int HD, int NQT>
+struct __align__(1024) PairSmem {
+  using C = PC<HD, NQT>;
+  uint8_t q[NQT][C::Q_TILE_BYTES];
+  uint8_t kv[C::STAGES][C::KV_TILE_BYTES];
+  uint64_t q_full;
+  uint64_t kv_full[C::STAGES];
+  uint64_t kv_empty[C::STAGES];
+  uint64_t s_full[NQT];         // both halves' scores of a pair complete; phase = pair
+  uint64_t p_ready[NQT][2];     // P of half h written over its scores; phase = pair
+  uint64_t pv_done[NQT][2];     // O_t += P_t[h] V complete; phase = pair
+  uint32_t tmem_base;
+  uint32_t raised;
+  volatile uint32_t abort;
+};
+
+template <int HD, int NQT>
+__global__ void __launch_bounds__(PC<HD, NQT>::THREADS, 1)
+attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const AttnDev p, int* __restrict__ status) {
+  using C = PC<HD, NQT>;
+  constexpr int BKV = C::BKV, PKV = C::PKV;
+  constexpr int STAGES = C::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  PairSmem<HD, NQT>& s =
+      *reinterpret_cast<PairSmem<HD, NQT>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  const int q_tile = p.q_tiles - 1 - (int)blockIdx.x;    // heaviest query tiles first
+  const int head0 = blockIdx.y * NQT;
+  const int b = blockIdx.z;
+  const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
+  const int q_row0 = q_tile * 128;
+  const int pos0 = p.q_pos0 + q_row0;
+  const int last_pos = min(pos0 + 127, p.q_pos0 + p.seq_len - 1);
+  const int j_hi = min(last_pos, p.kv_len - 1) / BKV;
+  const int j_lo = p.window > 0 ? max(0, pos0 - p.window + 1) / BKV : 0;
+  const int n_tiles = j_hi - j_lo + 1;                   // 64-key tiles
+  const int n_pairs = (n_tiles + 1) >> 1;
+
+  if (status_raised(status, &s.raised)) return;
+  if (threadIdx.x == 0) {
+    mbar_init(&s.q_full, 1);
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(&s.kv_full[i], 1);
+      mbar_init(&s.kv_empty[i], 1);
+    }
+    for (int t = 0; t < NQT; ++t) {
+      mbar_init(&s.s_full[t], 1);
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&s.p_ready[t][i], 4);
+        mbar_init(&s.pv_done[t][i], 1);
+      }
+    }
+    s.abort = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+  }
+  if (warp == NQT * 4 + 1) {
+    tmem_alloc(&s.tmem_base, C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s.tmem_base;
+
+  if (warp == NQT * 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(&s.q_full, NQT * C::Q_TILE_BYTES);
+      for (int t = 0; t < NQT; ++t)
+        for (int c = 0; c < HD / 64; ++c)
+          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, b * p.seq_len + q_row0);
+      const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
+      const int loads_per_tile = PKV / p.rows_per_load;
+      // ring order: K_0, V_0, K_1, V_1, ... (128-key stages)
+      bool ok = true;
+      for (int ring = 0; ring < 2 * n_pairs && ok && !s.abort; ++ring) {
+        const int J = ring >> 1;
+        const CUtensorMap* tm = (ring & 1) ? &tmV : &tmK;
+        const int kv0 = (j_lo + 2 * J) * BKV;
+        const int stage = ring % STAGES;
+        const uint32_t phase = (ring / STAGES) & 1;
+        if (!mbar_wait_relaxed(&s.kv_empty[stage], phase ^ 1)) {
+          POP_ABORT(s, status);
+          ok = false;
+          break;
+        }
+        int n_loads = 0;
+        for (int r = 0; r < loads_per_tile; ++r)
+          if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
+        mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
+        for (int r = 0; r < n_loads; ++r) {
+          const int pos = kv0 + r * p.rows_per_load;
+          const int page = bt[pos / p.page_size];
+          const int slot = pos % p.page_size;
+          for (int c = 0; c < HD / 64; ++c)
+            tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
+                        c * 64, kv_head, slot, page);
+        }
+      }
+    }
+  } else if (warp == NQT * 4 + 1) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp, elected lane)
+    const uint32_t leader = elect_one();
+    constexpr uint32_t idesc_s = umma_idesc_bf16(128, PKV, 0, 0);
+    constexpr uint32_t idesc_o = umma_idesc_bf16(128, HD, 0, 1);
+    uint64_t q_desc[NQT];
+    for (int t = 0; t < NQT; ++t) q_desc[t] = umma_smem_desc(smem_u32(s.q[t]), 16, 1024);
+    const uint64_t k_desc0 = umma_smem_desc(smem_u32(s.kv[0]), 16, 1024);                 // K-major
+    const uint64_t v_desc0 = umma_smem_desc(smem_u32(s.kv[0]), C::KV_SUB_BYTES, 1024);    // MN-major
+    auto issue_s = [&](int t, int stage) {               // 128 keys -> both score buffers of tile t
+      const uint64_t qd = q_desc[t];
+      const uint64_t kd = k_desc0 + uint64_t(stage * (C::KV_TILE_BYTES >> 4));
+      const uint32_t d = tmem_base + C::S_COL + t * 2 * BKV;
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const uint64_t ad = qd + uint64_t(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+        const uint64_t bd = kd + uint64_t(((kk >> 2) * C::KV_SUB_BYTES + (kk & 3) * 32) >> 4);
+        umma_bf16_ss_w(leader, d, ad, bd, idesc_s, kk > 0 ? 1u : 0u);
+      }
+      umma_commit_w(leader, &s.s_full[t]);
+    };
+    auto issue_pv = [&](int t, int jj, int stage) {      // 64 keys: half jj & 1 of the pair's V stage
+      const int h = jj & 1;
+      const uint32_t pa = tmem_base + C::S_COL + (t * 2 + h) * BKV;
+      const uint64_t vd = v_desc0 + uint64_t((stage * C::KV_TILE_BYTES + h * BKV * 128) >> 4);
+      const uint32_t d = tmem_base + C::O_COL + t * HD;
+#pragma unroll
+      for (int kk = 0; kk < BKV / 16; ++kk)
+        umma_bf16_ts_w(leader, d, pa + kk * 8, vd + uint64_t((kk * 2048) >> 4), idesc_o,
+                       (jj > 0 || kk > 0) ? 1u : 0u);
+      umma_commit_w(leader, &s.pv_done[t][h]);
+    };
+    bool ok = mbar_wait_relaxed(&s.q_full, 0);
+    if (ok) ok = mbar_wait_relaxed(&s.kv_full[0], 0);
+    if (ok) {
+      tc_fence_after();
+      for (int t = 0; t < NQT; ++t) issue_s(t, 0);
+      umma_commit_w(leader, &s.kv_empty[0]);
+    }
+    for (int J = 0; J < n_pairs && ok && !s.abort; ++J) {
+      const int rv = 2 * J + 1, rk = 2 * J + 2;
+      const int sv = rv % STAGES, sk = rk % STAGES;
+      const bool more = J + 1 < n_pairs;
+      ok = mbar_wait_relaxed(&s.kv_full[sv], (rv / STAGES) & 1);
+      bool k_ready = false;
+      for (int h = 0; h < 2 && ok; ++h) {
+        const int jj = 2 * J + h;
+        if (jj >= n_tiles) break;
+        const bool last_half = (h == 1) || (jj + 1 >= n_tiles);
+        for (int t = 0; t < NQT && ok; ++t) {
+          ok = mbar_wait_relaxed(&s.p_ready[t][h], J & 1);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, jj, sv);
+          if (last_half && more) {
+            // both score buffers of tile t are consumed (the pipe runs in order): next pair's scores
+            if (!k_ready) {
+              ok = mbar_wait_relaxed(&s.kv_full[sk], (rk / STAGES) & 1);
+              if (!ok) break;
+              tc_fence_after();
+              k_ready = true;
+            }
+            issue_s(t, sk);
+          }
+        }
+      }
+      if (ok) {
+        umma_commit_w(leader, &s.kv_empty[sv]);
+        if (more) umma_commit_w(leader, &s.kv_empty[sk]);
+      }
+    }
+    if (!ok) POP_ABORT(s, status);
+  } else {
+    // ------------------------------------------------------------------ softmax warpgroups
+    const int t = warp >> 2;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int pos = pos0 + row;
+    const uint32_t lane_addr = uint32_t(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + lane_addr + C::S_COL + t * 2 * BKV;
+    const uint32_t o_addr = tmem_base + lane_addr + C::O_COL + t * HD;
+    float m_run = -INFINITY;
+    float l_run = 0.f;
+    bool ok = true;
+    // P V product of 64-key tile j: barrier pv_done[t][j & 1], phase = pair j >> 1
+    auto wait_pv = [&](int j) { return mbar_wait(&s.pv_done[t][j & 1], (j >> 1) & 1); };
+
+    for (int jj = 0; jj < n_tiles && !s.abort; ++jj) {
+      const int J = jj >> 1, h = jj & 1;
+      const int kv0 = (j_lo + jj) * BKV;
+      const uint32_t sp_addr = s_addr + h * BKV;
+      if (h == 0) {
+        if (!mbar_wait(&s.s_full[t], J & 1)) { ok = false; break; }
+        tc_fence_after();
+      }
+      float sv[BKV];
+#pragma unroll
+      for (int c = 0; c < BKV / 32; ++c)
+        tmem_ld_32x32b_x32(sp_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+      tmem_wait_ld();
+      const bool partial = (kv0 + BKV - 1 > pos0) || (p.window > 0 && kv0 <= pos0 + 127 - p.window);
+      if (partial) {
+        const int lo = p.window > 0 ? pos - p.window : -1;   // valid keys: lo < j <= pos
+#pragma unroll
+        for (int i = 0; i < BKV; ++i) {
+          const int j = kv0 + i;
+          if (!(j <= pos && j > lo)) sv[i] = -INFINITY;
+        }
+      }
+      float mx0 = sv[0], mx1 = sv[1], mx2 = sv[2], mx3 = sv[3];
+#pragma unroll
+      for (int i = 4; i + 8 <= BKV; i += 8) {
+        mx0 = max3(mx0, sv[i], sv[i + 1]);
+        mx1 = max3(mx1, sv[i + 2], sv[i + 3]);
+        mx2 = max3(mx2, sv[i + 4], sv[i + 5]);
+        mx3 = max3(mx3, sv[i + 6], sv[i + 7]);
+      }
+      mx0 = max3(mx0, sv[BKV - 4], sv[BKV - 3]);
+      mx1 = max3(mx1, sv[BKV - 2], sv[BKV - 1]);
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;   // log2 domain
+      const float m_new = fmaxf(m_run, mx);
+      const bool need = (m_new - m_run > 8.0f) || (m_run == -INFINITY && m_new > -INFINITY);
+      if (__any_sync(0xffffffffu, need)) {
+        const float factor = (m_new == -INFINITY) ? 1.0f : ex2(m_run - m_new);   // ex2(-inf) = 0
+        if (jj > 0) {
+          if (!wait_pv(jj - 1)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld_32x32b_x32(o_addr + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+            tmem_st_32x32b_x32(o_addr + c * 32, o);
+          }
+          tmem_wait_st();
+        }
+        l_run *= factor;
+        m_run = m_new;
+      }
+      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+      const float2 nm2 = make_float2(-m_use, -m_use);
+      float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+      uint32_t pk[BKV / 2];
+#pragma unroll
+      for (int c = 0; c < BKV / 8; ++c) {
+        float2 x0 = __ffma2_rn(make_float2(sv[c * 8 + 0], sv[c * 8 + 1]), sc2, nm2);
+        float2 x1 = __ffma2_rn(make_float2(sv[c * 8 + 2], sv[c * 8 + 3]), sc2, nm2);
+        float2 x2 = __ffma2_rn(make_float2(sv[c * 8 + 4], sv[c * 8 + 5]), sc2, nm2);
+        float2 x3 = __ffma2_rn(make_float2(sv[c * 8 + 6], sv[c * 8 + 7]), sc2, nm2);
+        x0.x = ex2(x0.x); x0.y = ex2(x0.y);
+        x1.x = ex2(x1.x); x1.y = ex2(x1.y);
+        x2.x = ex2(x2.x); x2.y = ex2(x2.y);
+        x3.x = ex2(x3.x); x3.y = ex2(x3.y);
+        acc0 = __fadd2_rn(acc0, x0);
+        acc1 = __fadd2_rn(acc1, x1);
+        acc0 = __fadd2_rn(acc0, x2);
+        acc1 = __fadd2_rn(acc1, x3);
+        pk[c * 4 + 0] = pack2(x0.x, x0.y);
+        pk[c * 4 + 1] = pack2(x1.x, x1.y);
+        pk[c * 4 + 2] = pack2(x2.x, x2.y);
+        pk[c * 4 + 3] = pack2(x3.x, x3.y);
+      }
+      l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+      tmem_st_32x32b_x32(sp_addr, pk);      // over the scores this thread has just consumed
+      tmem_wait_st();
+      // cache rows at positions >= kv_len may hold anything: zero them in the pair's staged V tile
+      // (128 rows, one per thread of warpgroup 0) before either half's product can read them
+      const int pair_kv0 = (j_lo + 2 * J) * BKV;
+      if (pair_kv0 + PKV > p.kv_len) {
+        const int rv = 2 * J + 1;
+        if (!mbar_wait(&s.kv_full[rv % STAGES], (rv / STAGES) & 1)) { ok = false; break; }
+        if (t == 0 && pair_kv0 + row >= p.kv_len) {
+          for (int c = 0; c < HD / 64; ++c) {
+            uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + row * 128);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) dst[q] = make_uint4(0, 0, 0, 0);
+          }
+        }
+        fence_proxy_async_smem();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.p_ready[t][h]);
+    }
+    if (ok && !s.abort) {
+      if (!wait_pv(n_tiles - 1)) {
+        ok = false;
+      } else {
+        tc_fence_after();
+        const float inv = 1.0f / l_run;
+        const int seq_row = q_row0 + row;
+        const bool store = seq_row < p.seq_len;
+        bf16* out = p.out + ((int64_t)b * p.seq_len + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
+#pragma unroll 1
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld_32x32b_x32(o_addr + c * 32, o);
+          tmem_wait_ld();
+          if (store) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 w;
+              w.x = pack2(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
+              w.y = pack2(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
+              w.z = pack2(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
+              w.w = pack2(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
+              *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
+            }
+          }
+        }
+      }
+    }
+    if (!ok) POP_ABORT(s, status);
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (s.abort && threadIdx.x == 0) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let in-flight bulk copies land
+  }
+  __syncthreads();
+  if (warp == NQT * 4 + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+template <int HD, int NQT, bool PAIR>
 int launch_t(const AttnArgs& a, cudaStream_t stream) {
-  using C = AC<HD, NQT>;
+  using C = typename std::conditional<PAIR, PC<HD, NQT>, AC<HD, NQT>>::type;
   AttnDev p;
   p.out = a.out;
   p.ldo = a.ldo;
@@ -475,10 +840,14 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
     rc = make_tmap_bf16_nd(&tv, a.v_pool, 4, dims, str, box);
     if (rc) return rc;
   }
-  const size_t smem = sizeof(AttnSmem<HD, NQT>) + 1024;
+  using Smem = typename std::conditional<PAIR, PairSmem<HD, NQT>, AttnSmem<HD, NQT>>::type;
+  const size_t smem = sizeof(Smem) + 1024;
+  void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, AttnDev, int*);
+  if constexpr (PAIR) kernel = attn_pair_kernel<HD, NQT>;
+  else kernel = attn_kernel<HD, NQT>;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(attn_kernel<HD, NQT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return POP_E_CUDA;
     configured = true;
@@ -495,7 +864,7 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
   int* status = status_word();
   if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_ATTENTION, 4.0 * HD * pairs * a.n_q_heads * a.batch, stream);
-  attn_kernel<HD, NQT><<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status);
+  kernel<<<grid, C::THREADS, smem, stream>>>(tq, tk, tv, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -511,9 +880,9 @@ int launch_attention(const AttnArgs& a, cudaStream_t stream) {
   if ((int64_t)ceil_div(a.kv_len, a.page_size) > a.max_pages_per_seq) return POP_E_NOSPACE;
   const bool pair = (a.n_q_heads / a.n_kv_heads) % 2 == 0;
   switch (a.head_dim) {
-    case 64: return pair ? launch_t<64, 2>(a, stream) : launch_t<64, 1>(a, stream);
-    case 128: return pair ? launch_t<128, 2>(a, stream) : launch_t<128, 1>(a, stream);
-    case 256: return launch_t<256, 1>(a, stream);
+    case 64: return pair ? launch_t<64, 2, true>(a, stream) : launch_t<64, 1, true>(a, stream);
+    case 128: return pair ? launch_t<128, 2, true>(a, stream) : launch_t<128, 1, true>(a, stream);
+    case 256: return launch_t<256, 1, false>(a, stream);
   }
   return POP_E_INVALID;
 }
