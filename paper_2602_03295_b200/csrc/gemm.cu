@@ -128,8 +128,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks this role with identical values; one elected lane issues.
+    {
+      const uint32_t leader = elect_one();
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      const uint64_t a_desc0 = umma_smem_desc(smem_u32(s.a[0]), 16, 1024);
+      const uint64_t b_desc0 = umma_smem_desc(smem_u32(s.b[0]), 16, 1024);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -150,15 +154,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(s.a[stage]);
-          const uint32_t b_addr = smem_u32(s.b[stage]);
+          // only the 16-byte-granular start address in the descriptor's low bits moves
+          const uint64_t ad0 = a_desc0 + uint64_t(stage * (A_BYTES >> 4));
+          const uint64_t bd0 = b_desc0 + uint64_t(stage * (B_BYTES >> 4));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t ad = umma_smem_desc(a_addr + k * 32, 16, 1024);
-            const uint64_t bd = umma_smem_desc(b_addr + k * 32, 16, 1024);
-            umma_bf16_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
-          }
-          umma_commit(&s.empty[stage]);
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16_ss_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
+                           (kb | k) != 0 ? 1u : 0u);
+          umma_commit_w(leader, &s.empty[stage]);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1;
@@ -169,7 +172,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
           break;
         }
-        umma_commit(&s.tfull[buf]);
+        umma_commit_w(leader, &s.tfull[buf]);
       }
     }
   } else {
