@@ -117,8 +117,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int lane = threadIdx.x & 31;
 
   // heaviest query tiles (latest positions) first
-  const int q_tile = p.q_tiles - 1 - (int)blockIdx.x;
-  const int head0 = blockIdx.y * NQT;
+  const int q_tile = p.q_tiles - 1 - (int)blockIdx.y;
+  const int head0 = blockIdx.x * NQT;
   const int b = blockIdx.z;
   const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
   const int q_row0 = q_tile * 128;                       // row within the sequence
@@ -491,8 +491,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  const int q_tile = p.q_tiles - 1 - (int)blockIdx.x;    // heaviest query tiles first
-  const int head0 = blockIdx.y * NQT;
+  const int q_tile = p.q_tiles - 1 - (int)blockIdx.y;    // heaviest query tiles first
+  const int head0 = blockIdx.x * NQT;
   const int b = blockIdx.z;
   const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
   const int q_row0 = q_tile * 128;
@@ -852,7 +852,9 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
       return POP_E_CUDA;
     configured = true;
   }
-  dim3 grid(p.q_tiles, a.n_q_heads / NQT, a.batch);
+  // CTAs are handed out in blockIdx order, x fastest: all heads of the heaviest query tile first, so the
+  // lightest tiles form the tail of the launch
+  dim3 grid(a.n_q_heads / NQT, p.q_tiles, a.batch);
   // algorithmic work: 4 * hd flops per unmasked (query, key) pair and query head
   double pairs = 0;
   if (prof_enabled()) {
