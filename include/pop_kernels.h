@@ -26,6 +26,20 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
                int64_t ldo, int64_t o_bs, int32_t M, int32_t N, int32_t K, int32_t batch, int32_t epilogue,
                int32_t act, int32_t n_valid, void* stream);
 
+/* The fused form of the QKV projection and pop_k_rope_cache (paper Eq. 2-3; Eq. 14 for pruned
+ * layers): D[g] = A[g] W[g]^T with W's rows ordered [q heads | k heads | v heads] * hd, and in the
+ * GEMM's epilogue the optional per-head RMSNorm (q, k), RoPE (q, k), rounding to bf16, q -> q_out
+ * [M][ldq] (n_q may be 0: no query, as for pruned layers), k and v -> cache layer layer0 + g.
+ * A bf16 [batch][M][lda] (batch stride a_bs, 0 = packed), W bf16 [batch][(n_q+2 n_kv) hd][ldw].
+ * Row / position / cache conventions and the remaining arguments are those of pop_k_rope_cache;
+ * M must be a multiple of rows_per_seq. Nothing of the fp32 projection goes through memory. */
+int pop_k_gemm_qkv_rope(const void* A, int64_t lda, int64_t a_bs, const void* W, int64_t ldw, int64_t w_bs, int32_t M,
+                        int32_t K, int32_t batch, void* q_out, int64_t ldq, void* k_pool, void* v_pool,
+                        int64_t pool_layer_stride, int32_t layer0, const int32_t* block_table,
+                        int32_t max_pages_per_seq, int32_t page_size, const float* q_gain, const float* k_gain,
+                        int64_t gain_gs, const void* table, int32_t n_q, int32_t n_kv, int32_t head_dim,
+                        int32_t rows_per_seq, int32_t rows_written, int32_t pos0, float eps, void* stream);
+
 /* Causal GQA attention of a decoder layer over the paged cache (paper Eq. 1, Attn(x_l, K, V) after
  * the append of Eq. 3): for sequence b, query row i (absolute position q_pos0 + i) and head h,
  *   out[b][i][h] = sum_j softmax_j(q[b][i][h] . k[b][j][g] / sqrt(hd)) v[b][j][g],  g = h*n_kv/n_q,

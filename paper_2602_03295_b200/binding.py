@@ -67,6 +67,8 @@ SIGNATURES = {
     "pop_strerror": (C.c_char_p, [C.c_int]),
     "pop_k_gemm": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _I32, _I32, _I32,
                              _I32, _P]),
+    "pop_k_gemm_qkv_rope": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _P, _I64, _P, _P, _I64, _I32,
+                                      _P, _I32, _I32, _P, _P, _I64, _P] + [_I32] * 6 + [_F, _P]),
     "pop_k_attention": (C.c_int, [_P, _I64, _P, _P, _P, _P, _I64] + [_I32] * 11 + [_P]),
     "pop_k_rmsnorm": (C.c_int, [_P, _I64, _P, _I64, _P, _I64, _I64, _I32, _I32, _I32, _F, _I32, _P]),
     "pop_k_rope_table": (C.c_int, [_P, _I32, _I32, _F, _P]),
@@ -154,6 +156,23 @@ class PopLibrary:
         self.check(code, "pop_k_gemm")
         return out
 
+
+    def gemm_qkv_rope(self, A, W, q_out, k_pool, v_pool, layer0, block_table, page_size, q_gain, k_gain, table,
+                      n_q, n_kv, hd, rows_per_seq, rows_written, pos0, eps, stream=None):
+        """Fused QKV projection + per-head norm + RoPE + cache write. A [M,K] or [G,M,K] bf16; W
+        [(n_q+2 n_kv) hd, K] or [G, ..., K] bf16; pools [layers, pages, page_size, n_kv, hd]."""
+        if A.dim() == 2:
+            A, W = A.unsqueeze(0), W.unsqueeze(0)
+        G, M, K = A.shape
+        gain_gs = 0 if (k_gain is None or k_gain.dim() == 1) else k_gain.stride(0)
+        code = self.dll.pop_k_gemm_qkv_rope(A.data_ptr(), A.stride(1), A.stride(0) if G > 1 else 0, W.data_ptr(),
+                                            W.stride(1), W.stride(0) if G > 1 else 0, M, K, G, _ptr(q_out),
+                                            0 if q_out is None else q_out.stride(0), k_pool.data_ptr(),
+                                            v_pool.data_ptr(), k_pool.stride(0), layer0, block_table.data_ptr(),
+                                            block_table.shape[1], page_size, _ptr(q_gain), _ptr(k_gain), gain_gs,
+                                            table.data_ptr(), n_q, n_kv, hd, rows_per_seq, rows_written, pos0, eps,
+                                            _stream_ptr(stream))
+        self.check(code, "pop_k_gemm_qkv_rope")
 
     def attention(self, q, k_pool, v_pool, block_table, out, batch, seq_len, kv_len, n_q, n_kv, hd, page_size,
                   window=0, q_pos0=0, stream=None):

@@ -18,6 +18,30 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
   return launch_gemm(a, static_cast<cudaStream_t>(stream));
 }
 
+int pop_k_gemm_qkv_rope(const void* A, int64_t lda, int64_t a_bs, const void* W, int64_t ldw, int64_t w_bs, int32_t M,
+                        int32_t K, int32_t batch, void* q_out, int64_t ldq, void* k_pool, void* v_pool,
+                        int64_t pool_layer_stride, int32_t layer0, const int32_t* block_table,
+                        int32_t max_pages_per_seq, int32_t page_size, const float* q_gain, const float* k_gain,
+                        int64_t gain_gs, const void* table, int32_t n_q, int32_t n_kv, int32_t head_dim,
+                        int32_t rows_per_seq, int32_t rows_written, int32_t pos0, float eps, void* stream) {
+  RopeArgs r{};
+  r.q_out = static_cast<bf16*>(q_out); r.ldq = ldq;
+  r.k_pool = static_cast<bf16*>(k_pool); r.v_pool = static_cast<bf16*>(v_pool);
+  r.pool_layer_stride = pool_layer_stride; r.layer0 = layer0;
+  r.block_table = block_table; r.max_pages_per_seq = max_pages_per_seq; r.page_size = page_size;
+  r.q_gain = q_gain; r.k_gain = k_gain; r.gain_group_stride = gain_gs;
+  r.table = static_cast<const float2*>(table);
+  r.n_q = n_q; r.n_kv = n_kv; r.hd = head_dim;
+  r.rows = M; r.rows_per_seq = rows_per_seq; r.rows_written = rows_written; r.pos0 = pos0; r.groups = batch;
+  r.eps = eps;
+  GemmArgs a{};
+  a.A = static_cast<const bf16*>(A); a.lda = lda; a.a_batch_stride = a_bs;
+  a.B = static_cast<const bf16*>(W); a.ldb = ldw; a.b_batch_stride = w_bs;
+  a.M = M; a.N = (n_q + 2 * n_kv) * head_dim; a.K = K; a.batch = batch;
+  a.epilogue = EPI_QKV_ROPE; a.rope = &r;
+  return launch_gemm(a, static_cast<cudaStream_t>(stream));
+}
+
 int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool, const int32_t* block_table,
                     void* out, int64_t ldo, int32_t batch, int32_t seq_len, int32_t q_pos0, int32_t kv_len,
                     int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t page_size, int32_t num_pages,

@@ -56,9 +56,12 @@ enum GemmEpilogue {
   EPI_STORE_BF16 = 0,   // out bf16 [M][ldo]
   EPI_STORE_F32 = 1,    // out fp32 [M][ldo]
   EPI_ADD_F32 = 2,      // out fp32 [M][ldo] += D  (residual add)
-  EPI_GATED_BF16 = 3    // B rows come in blocks of 256: 128 gate rows then the matching 128 up rows;
+  EPI_GATED_BF16 = 3,   // B rows come in blocks of 256: 128 gate rows then the matching 128 up rows;
                         // out bf16 [M][ldo], column f = act(gate_f) * up_f, for f < n_valid
+  EPI_QKV_ROPE = 4      // columns are heads [q heads | k heads | v heads] * hd: per-head norm, RoPE and the
+                        // paged-cache write happen in the epilogue (GemmArgs::rope describes where to)
 };
+struct RopeArgs;
 struct GemmArgs {
   const bf16* A; int64_t lda; int64_t a_batch_stride;   // elements
   const bf16* B; int64_t ldb; int64_t b_batch_stride;
@@ -67,6 +70,7 @@ struct GemmArgs {
   int epilogue;
   int act;          // EPI_GATED_BF16: 0 SiLU, 1 tanh-GELU
   int n_valid;      // EPI_GATED_BF16: number of valid output columns (d_ffn); others: ignored
+  const RopeArgs* rope;   // EPI_QKV_ROPE only (its in / ld_in fields are unused; groups == batch)
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t stream);
 

@@ -35,7 +35,21 @@ struct __align__(1024) GemmSmem {
   volatile uint32_t abort;
 };
 
+// where the QKV epilogue writes: q rows, and k / v rows into the paged cache
+struct RopeEpi {
+  bf16* q_out; int64_t ldq;
+  bf16* k_pool; bf16* v_pool; int64_t pool_layer_stride;
+  int layer0;
+  const int32_t* block_table; int max_pages_per_seq; int page_size;
+  const float* q_gain; const float* k_gain; int64_t gain_group_stride;
+  const float2* table;
+  int n_q, n_kv;
+  int rows_per_seq, rows_written, pos0;
+  float eps;
+};
+
 struct GemmDev {
+  RopeEpi rope;
   void* out;
   int64_t ldo, out_batch_stride;
   int M, N, K, batch;
@@ -67,7 +81,113 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int EPI>
+// Epilogue of the fused QKV projection (paper Eq. 2-3; Eq. 14 for pruned layers): the thread owns one
+// token row of the 128 x 256 accumulator tile, which holds 256 / HD whole heads. q and k heads get
+// the optional per-head RMSNorm and RoPE (pair (j, j + HD/2), so two 32-column chunks of TMEM are
+// processed together), everything is rounded to bf16; q goes to its row buffer, k and v straight
+// into the token's slot of the paged cache. All tcgen05.ld are executed by every lane.
+template <int HD>
+__device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t taddr, int g, int n, int row,
+                                                  bool row_ok) {
+  const RopeEpi& r = p.rope;
+  constexpr int HALF_CHUNKS = HD / 64;                   // 32-column chunks per half head
+  const int total_heads = r.n_q + 2 * r.n_kv;
+  const int b = row / r.rows_per_seq;
+  const int i = row - b * r.rows_per_seq;
+  const bool active = row_ok && i < r.rows_written;
+  const int pos = r.pos0 + i;
+  int64_t cache_row = 0;
+  if (active) {
+    const int page = r.block_table[(int64_t)b * r.max_pages_per_seq + pos / r.page_size];
+    cache_row = (int64_t)page * r.page_size + pos % r.page_size;
+  }
+  const float2* tab = r.table + (int64_t)pos * (HD / 2);
+#pragma unroll 1
+  for (int hh = 0; hh < 256 / HD; ++hh) {
+    const int head = n * (256 / HD) + hh;
+    if (head >= total_heads) break;                      // uniform: depends on the tile only
+    const uint32_t haddr = taddr + hh * HD;
+    const bool is_q = head < r.n_q;
+    const bool is_v = head >= r.n_q + r.n_kv;
+    bf16* dst;
+    if (is_q) {
+      dst = r.q_out + (int64_t)row * r.ldq + (int64_t)head * HD;
+    } else {
+      const int kvh = is_v ? head - r.n_q - r.n_kv : head - r.n_q;
+      bf16* pool = (is_v ? r.v_pool : r.k_pool) + (int64_t)(r.layer0 + g) * r.pool_layer_stride;
+      dst = pool + (cache_row * r.n_kv + kvh) * HD;
+    }
+    if (is_v) {
+#pragma unroll 1
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t x[32];
+        tmem_ld_32x32b_x32(haddr + c * 32, x);
+        tmem_wait_ld();
+        if (active) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              w[j] = pack_bf16(__uint_as_float(x[v * 8 + j * 2]), __uint_as_float(x[v * 8 + j * 2 + 1]));
+            *reinterpret_cast<uint4*>(dst + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      continue;
+    }
+    const float* gain = is_q ? r.q_gain : r.k_gain;
+    float rstd = 1.0f;
+    if (gain != nullptr) {                               // uniform
+      gain += (int64_t)g * r.gain_group_stride;
+      float ss = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t x[32];
+        tmem_ld_32x32b_x32(haddr + c * 32, x);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(x[e]), __uint_as_float(x[e]), ss);
+      }
+      rstd = rsqrtf(ss / (float)HD + r.eps);
+    }
+#pragma unroll 1
+    for (int c = 0; c < HALF_CHUNKS; ++c) {
+      uint32_t lo[32], hi[32];
+      tmem_ld_32x32b_x32(haddr + c * 32, lo);
+      tmem_ld_32x32b_x32(haddr + (c + HALF_CHUNKS) * 32, hi);
+      tmem_wait_ld();
+      if (active) {
+        float a[32], bq[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int j = c * 32 + e;
+          float x = __uint_as_float(lo[e]), y = __uint_as_float(hi[e]);
+          if (gain != nullptr) {
+            x = x * rstd * gain[j];
+            y = y * rstd * gain[j + HD / 2];
+          }
+          const float2 cs = tab[j];
+          a[e] = x * cs.x - y * cs.y;
+          bq[e] = y * cs.x + x * cs.y;
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4], z[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            w[j] = pack_bf16(a[v * 8 + j * 2], a[v * 8 + j * 2 + 1]);
+            z[j] = pack_bf16(bq[v * 8 + j * 2], bq[v * 8 + j * 2 + 1]);
+          }
+          *reinterpret_cast<uint4*>(dst + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + HD / 2 + c * 32 + v * 8) = make_uint4(z[0], z[1], z[2], z[3]);
+        }
+      }
+    }
+  }
+}
+
+template <int EPI, int HD>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p,
             int* __restrict__ status) {
@@ -194,7 +314,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int row = m * BM + row_in_tile;
       const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
-      if (EPI == EPI_GATED_BF16) {
+      if (EPI == EPI_QKV_ROPE) {
+        qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok);
+      } else if (EPI == EPI_GATED_BF16) {
         bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -280,19 +402,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
-template <int EPI>
+template <int EPI, int HD = 0>
 int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, int grid, cudaStream_t stream) {
   const size_t smem = sizeof(GemmSmem) + 1024;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_kernel<EPI, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return POP_E_CUDA;
     configured = true;
   }
   int* status = status_word();
   if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
-  gemm_kernel<EPI><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status);
+  gemm_kernel<EPI, HD><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -300,11 +422,17 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, i
 }  // namespace
 
 int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
-  if (!a.A || !a.B || !a.out || a.M < 1 || a.N < 1 || a.K < 1 || a.batch < 1) return POP_E_INVALID;
+  if (!a.A || !a.B || (!a.out && a.epilogue != EPI_QKV_ROPE) || a.M < 1 || a.N < 1 || a.K < 1 || a.batch < 1) return POP_E_INVALID;
   if (a.K % 8 || a.lda % 8 || a.ldb % 8 || a.a_batch_stride % 8 || a.b_batch_stride % 8) return POP_E_INVALID;
   if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.out)) & 15)
     return POP_E_INVALID;
-  if (a.epilogue == EPI_GATED_BF16) {
+  if (a.epilogue == EPI_QKV_ROPE) {
+    const RopeArgs* r = a.rope;
+    if (!r || !r->k_pool || !r->v_pool || !r->block_table || !r->table || (r->n_q > 0 && !r->q_out))
+      return POP_E_INVALID;
+    if ((r->hd != 64 && r->hd != 128 && r->hd != 256) || a.N != (r->n_q + 2 * r->n_kv) * r->hd) return POP_E_INVALID;
+    if (r->ldq % 8 || r->rows_per_seq < 1 || a.M % r->rows_per_seq) return POP_E_INVALID;
+  } else if (a.epilogue == EPI_GATED_BF16) {
     if (a.N % 256 || a.n_valid % 8 || a.n_valid > a.N / 2 || a.ldo % 8) return POP_E_INVALID;
   } else if (a.epilogue == EPI_STORE_BF16) {
     if (a.N % 8 || a.ldo % 8) return POP_E_INVALID;
@@ -318,7 +446,20 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
                          BN);
   if (rc) return rc;
-  GemmDev p;
+  GemmDev p{};
+  if (a.epilogue == EPI_QKV_ROPE) {
+    const RopeArgs& r = *a.rope;
+    p.rope.q_out = r.q_out; p.rope.ldq = r.ldq;
+    p.rope.k_pool = r.k_pool; p.rope.v_pool = r.v_pool; p.rope.pool_layer_stride = r.pool_layer_stride;
+    p.rope.layer0 = r.layer0;
+    p.rope.block_table = r.block_table; p.rope.max_pages_per_seq = r.max_pages_per_seq;
+    p.rope.page_size = r.page_size;
+    p.rope.q_gain = r.q_gain; p.rope.k_gain = r.k_gain; p.rope.gain_group_stride = r.gain_group_stride;
+    p.rope.table = r.table;
+    p.rope.n_q = r.n_q; p.rope.n_kv = r.n_kv;
+    p.rope.rows_per_seq = r.rows_per_seq; p.rope.rows_written = r.rows_written; p.rope.pos0 = r.pos0;
+    p.rope.eps = r.eps;
+  }
   p.out = a.out;
   p.ldo = a.ldo;
   p.out_batch_stride = a.out_batch_stride;
@@ -338,6 +479,13 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, p, grid, stream);
     case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, p, grid, stream);
     case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, p, grid, stream);
+    case EPI_QKV_ROPE:
+      switch (a.rope->hd) {
+        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, p, grid, stream);
+        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, p, grid, stream);
+        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, p, grid, stream);
+      }
+      return POP_E_INVALID;
   }
   return POP_E_INVALID;
 }

@@ -163,6 +163,54 @@ def test_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm):
     assert (kpool[0] == canary).all() and (kpool[2] == canary).all()   # other layers untouched
 
 
+@pytest.mark.parametrize("hd,n_q,n_kv,qk_norm,groups", [(64, 4, 2, 0, 1), (128, 4, 1, 1, 1), (256, 2, 2, 1, 1),
+                                                        (128, 0, 2, 1, 3), (64, 3, 3, 0, 1)])
+def test_fused_qkv_projection_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm, groups):
+    # the projection GEMM with norm, RoPE and the paged-cache write in its epilogue, against the
+    # oracle's statement of Eq. 2-3 (fp64); several m tiles with a ragged tail, several n tiles
+    B, N, K, page, theta, eps, layers = 2, 150, 136, 16, 500000.0, 1e-6, 5
+    rows, heads = B * N, n_q + 2 * n_kv
+    A = _bf((groups, rows, K), 30, 1.0)
+    W = _bf((groups, heads * hd, K), 31, 0.1)
+    table = torch.zeros(N, hd // 2, 2, dtype=torch.float32, device=DEV)
+    L.rope_table(table, N, hd, theta)
+    qg = ps.gains(1, 1, groups * hd, True).reshape(groups, hd) if qk_norm else None
+    kg = ps.gains(1, 2, groups * hd, True).reshape(groups, hd) if qk_norm else None
+    pps = (N + page - 1) // page
+    bt = torch.randperm(B * pps, generator=torch.Generator().manual_seed(2)).reshape(B, pps).int()
+    canary = -77.0
+    kpool = torch.full((layers, B * pps, page, n_kv, hd), canary, dtype=torch.bfloat16, device=DEV)
+    vpool = torch.full_like(kpool, canary)
+    q_out = torch.zeros(rows, max(n_q, 1) * hd, dtype=torch.bfloat16, device=DEV)
+    written = N - 1
+    dev = lambda t: None if t is None else t.to(DEV)
+    L.gemm_qkv_rope(A.to(DEV) if groups > 1 else A[0].to(DEV), W.to(DEV) if groups > 1 else W[0].to(DEV),
+                    q_out if n_q else None, kpool, vpool, 1, bt.to(DEV), page,
+                    dev(qg if groups > 1 or qg is None else qg[0]), dev(kg if groups > 1 or kg is None else kg[0]),
+                    table, n_q, n_kv, hd, N, written, 0, eps)
+    assert L.status() == 0
+    pos = torch.arange(N)
+    for g in range(groups):
+        x = (A[g].double() @ W[g].double().T).reshape(B, N, heads, hd)
+        q, k, v = x[:, :, :n_q], x[:, :, n_q:n_q + n_kv], x[:, :, n_q + n_kv:]
+        if qk_norm:
+            k = po.rmsnorm(k, kg[g].double(), eps)
+            if n_q:
+                q = po.rmsnorm(q, qg[g].double(), eps)
+        for b in range(B):
+            kr = po.rope(k[b], pos, theta)
+            if n_q:
+                qr = po.rope(q[b], pos, theta)
+                assert rel_err(q_out[b * N: b * N + written].reshape(written, n_q, hd), qr[:written]) < 1e-2
+            pages = bt[b, pos // page].long().to(DEV)
+            slots = (pos % page).to(DEV)
+            kg_, vg_ = kpool[1 + g][pages, slots], vpool[1 + g][pages, slots]
+            assert rel_err(kg_[:written], kr[:written]) < 1e-2
+            assert rel_err(vg_[:written], v[b, :written]) < 1e-2
+            assert (kg_[written:] == canary).all() and (vg_[written:] == canary).all()
+    assert (kpool[0] == canary).all() and (kpool[1 + groups:] == canary).all()
+
+
 @pytest.mark.parametrize("B,N,K,xf32", [(1, 1024, 4096, False), (8, 520, 688, False), (3, 1000, 256, True),
                                         (11, 64, 64, False)])
 def test_gemv_store_and_add(L, B, N, K, xf32):
