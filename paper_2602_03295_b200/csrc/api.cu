@@ -23,7 +23,7 @@ struct LayerOffsets {   // byte offsets inside one layer block of the arena
 struct Workspace {
   float* x;          // [M][d] residual stream, fp32
   bf16* hn;          // [chunk][M][d] normalised activations (GEMM operand)
-  float* qkv;        // [M][qkv_dim] fp32, or [chunk][M][2*kv_dim] for the pruned-layer pass
+  float* qkv;        // unused (kept for layout stability)
   bf16* q;           // [M][q_dim]
   bf16* ao;          // [M][q_dim] attention output
   bf16* act;         // [M][F] gated activation
@@ -116,7 +116,7 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   auto take = [&](size_t bytes) { char* r = base + o; o = align_up(o + bytes, kAlign); return r; };
   w.x = (float*)take(M * d * 4);
   w.hn = (bf16*)take((size_t)chunk * M * d * 2);
-  w.qkv = (float*)take(std::max(M * m->qkv_dim * 4, (size_t)chunk * M * 2 * m->kv_dim * 4));
+  w.qkv = nullptr;   // projections never pass through memory in fp32: the GEMM epilogue finishes them
   w.q = (bf16*)take(M * m->q_dim * 2);
   w.ao = (bf16*)take(M * m->q_dim * 2);
   w.act = (bf16*)take(M * (size_t)c.d_ffn * 2);
@@ -147,12 +147,9 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   const int M = B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
   POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_in), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
-  GemmArgs g{};
-  g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
-  g.out = w.qkv; g.ldo = m->qkv_dim; g.M = M; g.N = m->qkv_dim; g.K = d; g.batch = 1; g.epilogue = EPI_STORE_F32;
-  POP_TRY(launch_gemm(g, s));
+  // QKV projection with per-head norm, RoPE and the cache append (Eq. 2-3) in the GEMM's epilogue
   RopeArgs r{};
-  r.in = w.qkv; r.ld_in = m->qkv_dim; r.q_out = w.q; r.ldq = m->q_dim;
+  r.q_out = w.q; r.ldq = m->q_dim;
   r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
   r.layer0 = l - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
   r.page_size = kc->page_size;
@@ -160,7 +157,10 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   r.table = w.rope; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = M; r.rows_per_seq = N; r.rows_written = N; r.pos0 = 0; r.groups = 1; r.eps = c.rms_eps;
-  POP_TRY(launch_rope_cache(r, s));
+  GemmArgs g{};
+  g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
+  g.M = M; g.N = m->qkv_dim; g.K = d; g.batch = 1; g.epilogue = EPI_QKV_ROPE; g.rope = &r;
+  POP_TRY(launch_gemm(g, s));
   AttnArgs a{};
   a.q = w.q; a.ldq = m->q_dim;
   a.k_pool = (const bf16*)kc->k_pool + (int64_t)(l - 1) * pool_layer_stride;
@@ -213,15 +213,7 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
   POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l0, m->lo.ln_in), (int64_t)(m->layer_stride / 4), w.hn, d,
                          (int64_t)M * d, M, d, n, c.rms_eps, false, s));
-  GemmArgs g{};
-  g.A = w.hn; g.lda = d; g.a_batch_stride = (int64_t)M * d;
-  g.B = lp<bf16>(m, l0, m->lo.wqkv) + (int64_t)m->q_dim * d; g.ldb = d;
-  g.b_batch_stride = (int64_t)(m->layer_stride / 2);
-  g.out = w.qkv; g.ldo = 2 * m->kv_dim; g.out_batch_stride = (int64_t)M * 2 * m->kv_dim;
-  g.M = M; g.N = 2 * m->kv_dim; g.K = d; g.batch = n; g.epilogue = EPI_STORE_F32;
-  POP_TRY(launch_gemm(g, s));
   RopeArgs r{};
-  r.in = w.qkv; r.ld_in = 2 * m->kv_dim; r.in_group_stride = (int64_t)M * 2 * m->kv_dim;
   r.q_out = nullptr; r.ldq = 0;
   r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
   r.layer0 = l0 - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
@@ -231,7 +223,14 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   r.gain_group_stride = (int64_t)(m->layer_stride / 4);
   r.table = w.rope; r.n_q = 0; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = M; r.rows_per_seq = N; r.rows_written = N - 1; r.pos0 = 0; r.groups = n; r.eps = c.rms_eps;
-  return launch_rope_cache(r, s);
+  // ONE batched GEMM over the pruned layers (the layer is the batch dimension of both operands);
+  // its epilogue applies each layer's K norm and RoPE and writes the layer's cache entries
+  GemmArgs g{};
+  g.A = w.hn; g.lda = d; g.a_batch_stride = (int64_t)M * d;
+  g.B = lp<bf16>(m, l0, m->lo.wqkv) + (int64_t)m->q_dim * d; g.ldb = d;
+  g.b_batch_stride = (int64_t)(m->layer_stride / 2);
+  g.M = M; g.N = 2 * m->kv_dim; g.K = d; g.batch = n; g.epilogue = EPI_QKV_ROPE; g.rope = &r;
+  return launch_gemm(g, s);
 }
 
 // Boundary token as a decode step of layer l (paper Sec. 3.3): one row per sequence in w.xb.
