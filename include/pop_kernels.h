@@ -26,6 +26,22 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
                int64_t ldo, int64_t o_bs, int32_t M, int32_t N, int32_t K, int32_t batch, int32_t epilogue,
                int32_t act, int32_t n_valid, void* stream);
 
+/* pop_k_gemm (batch 1, epilogues 0-3) with the layer's RMSNorm (the LN of paper Eq. 1-2) folded
+ * around it, so that no separate pass over the residual stream is needed:
+ *  - producer side, epilogue 2 only, when hn_out != NULL: besides out += D the call writes
+ *    hn_out[m][n] = bf16(out_new[m][n] * gain_next[n]) (row stride ld_hn) -- the next GEMM's operand,
+ *    not yet normalised -- and ss_out[m * ss_ld + n / 256] = sum over that 256-column tile of
+ *    out_new[m][n]^2 (ss_ld >= ceil(N / 256));
+ *  - consumer side, when ss_in != NULL: every row m of D is multiplied by
+ *    rsqrt(sum_{i < ss_cnt} ss_in[m * ss_in_ld + i] / norm_d + norm_eps) before the epilogue acts
+ *    (for epilogue 3 before the activation). The partial sums are added in index order, so the
+ *    result does not depend on scheduling.
+ * Pass NULL for the side not wanted. */
+int pop_k_gemm_norm(const void* A, int64_t lda, const void* B, int64_t ldb, void* out, int64_t ldo, int32_t M,
+                    int32_t N, int32_t K, int32_t epilogue, int32_t act, int32_t n_valid, void* hn_out, int64_t ld_hn,
+                    const float* gain_next, float* ss_out, int32_t ss_ld, const float* ss_in, int32_t ss_cnt,
+                    int32_t ss_in_ld, int32_t norm_d, float norm_eps, void* stream);
+
 /* The fused form of the QKV projection and pop_k_rope_cache (paper Eq. 2-3; Eq. 14 for pruned
  * layers): D[g] = A[g] W[g]^T with W's rows ordered [q heads | k heads | v heads] * hd, and in the
  * GEMM's epilogue the optional per-head RMSNorm (q, k), RoPE (q, k), rounding to bf16, q -> q_out

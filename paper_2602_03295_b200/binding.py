@@ -67,6 +67,8 @@ SIGNATURES = {
     "pop_strerror": (C.c_char_p, [C.c_int]),
     "pop_k_gemm": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _I32, _I32, _I32,
                              _I32, _P]),
+    "pop_k_gemm_norm": (C.c_int, [_P, _I64, _P, _I64, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P, _I64, _P, _P, _I32,
+                                  _P, _I32, _I32, _I32, _F, _P]),
     "pop_k_gemm_qkv_rope": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _P, _I64, _P, _P, _I64, _I32,
                                       _P, _I32, _I32, _P, _P, _I64, _P] + [_I32] * 6 + [_F, _P]),
     "pop_k_attention": (C.c_int, [_P, _I64, _P, _P, _P, _P, _I64] + [_I32] * 11 + [_P]),
@@ -156,6 +158,22 @@ class PopLibrary:
         self.check(code, "pop_k_gemm")
         return out
 
+
+    def gemm_norm(self, A, B, out, epilogue, act=0, n_valid=0, hn_out=None, gain_next=None, ss_out=None,
+                  ss_in=None, norm_d=0, norm_eps=0.0, stream=None):
+        """pop_k_gemm_norm: 2-D operands; hn_out/gain_next/ss_out = producer side, ss_in [M, cnt] fp32 =
+        consumer side (None to leave a side out)."""
+        M, K = A.shape
+        N = B.shape[0]
+        code = self.dll.pop_k_gemm_norm(A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0), out.data_ptr(),
+                                        out.stride(0), M, N, K, epilogue, act, n_valid, _ptr(hn_out),
+                                        0 if hn_out is None else hn_out.stride(0), _ptr(gain_next), _ptr(ss_out),
+                                        0 if ss_out is None else ss_out.stride(0), _ptr(ss_in),
+                                        0 if ss_in is None else ss_in.shape[1],
+                                        0 if ss_in is None else ss_in.stride(0), norm_d, norm_eps,
+                                        _stream_ptr(stream))
+        self.check(code, "pop_k_gemm_norm")
+        return out
 
     def gemm_qkv_rope(self, A, W, q_out, k_pool, v_pool, layer0, block_table, page_size, q_gain, k_gain, table,
                       n_q, n_kv, hd, rows_per_seq, rows_written, pos0, eps, stream=None):

@@ -9,12 +9,28 @@ extern "C" {
 int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t ldb, int64_t b_bs, void* out,
                int64_t ldo, int64_t o_bs, int32_t M, int32_t N, int32_t K, int32_t batch, int32_t epilogue,
                int32_t act, int32_t n_valid, void* stream) {
-  GemmArgs a;
+  GemmArgs a{};
   a.A = static_cast<const bf16*>(A); a.lda = lda; a.a_batch_stride = a_bs;
   a.B = static_cast<const bf16*>(B); a.ldb = ldb; a.b_batch_stride = b_bs;
   a.out = out; a.ldo = ldo; a.out_batch_stride = o_bs;
   a.M = M; a.N = N; a.K = K; a.batch = batch;
   a.epilogue = epilogue; a.act = act; a.n_valid = n_valid;
+  return launch_gemm(a, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_gemm_norm(const void* A, int64_t lda, const void* B, int64_t ldb, void* out, int64_t ldo, int32_t M,
+                    int32_t N, int32_t K, int32_t epilogue, int32_t act, int32_t n_valid, void* hn_out, int64_t ld_hn,
+                    const float* gain_next, float* ss_out, int32_t ss_ld, const float* ss_in, int32_t ss_cnt,
+                    int32_t ss_in_ld, int32_t norm_d, float norm_eps, void* stream) {
+  GemmArgs a{};
+  a.A = static_cast<const bf16*>(A); a.lda = lda;
+  a.B = static_cast<const bf16*>(B); a.ldb = ldb;
+  a.out = out; a.ldo = ldo;
+  a.M = M; a.N = N; a.K = K; a.batch = 1;
+  a.epilogue = epilogue; a.act = act; a.n_valid = n_valid;
+  a.hn_out = static_cast<bf16*>(hn_out); a.ld_hn = ld_hn; a.gain_next = gain_next; a.ss_out = ss_out; a.ss_ld = ss_ld;
+  a.ss_in = ss_in; a.ss_cnt = ss_cnt; a.ss_in_ld = ss_in_ld; a.norm_d = norm_d; a.norm_eps = norm_eps;
+  if (epilogue == EPI_QKV_ROPE) return POP_E_INVALID;
   return launch_gemm(a, static_cast<cudaStream_t>(stream));
 }
 

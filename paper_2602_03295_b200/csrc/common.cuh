@@ -71,6 +71,13 @@ struct GemmArgs {
   int act;          // EPI_GATED_BF16: 0 SiLU, 1 tanh-GELU
   int n_valid;      // EPI_GATED_BF16: number of valid output columns (d_ffn); others: ignored
   const RopeArgs* rope;   // EPI_QKV_ROPE only (its in / ld_in fields are unused; groups == batch)
+  // RMSNorm folded around the GEMMs (batch == 1 only). A residual GEMM (EPI_ADD_F32) can also emit
+  // the next GEMM's operand hn = bf16(x_new * gain_next), NOT yet normalised, and per n-tile the
+  // row sums of x_new^2 (ss_out[row * ss_ld + n_tile], summed later in a fixed order, so results
+  // do not depend on timing). The consuming GEMM scales its rows by
+  // rsqrt(sum_i ss_in[row * ss_in_ld + i] / norm_d + norm_eps) before its own epilogue.
+  bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
+  const float* ss_in; int ss_cnt; int ss_in_ld; int norm_d; float norm_eps;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t stream);
 

@@ -55,6 +55,8 @@ struct GemmDev {
   int M, N, K, batch;
   int m_tiles, n_tiles;
   int act, n_valid;
+  bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
+  const float* ss_in; int ss_cnt; int ss_in_ld; float inv_d; float eps_in;
 };
 
 __device__ __forceinline__ void tile_coords(const GemmDev& p, int t, int& g, int& m, int& n) {
@@ -88,7 +90,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // into the token's slot of the paged cache. All tcgen05.ld are executed by every lane.
 template <int HD>
 __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t taddr, int g, int n, int row,
-                                                  bool row_ok) {
+                                                  bool row_ok, float rs) {
   const RopeEpi& r = p.rope;
   constexpr int HALF_CHUNKS = HD / 64;                   // 32-column chunks per half head
   const int total_heads = r.n_q + 2 * r.n_kv;
@@ -129,7 +131,7 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
             uint32_t w[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              w[j] = pack_bf16(__uint_as_float(x[v * 8 + j * 2]), __uint_as_float(x[v * 8 + j * 2 + 1]));
+              w[j] = pack_bf16(__uint_as_float(x[v * 8 + j * 2]) * rs, __uint_as_float(x[v * 8 + j * 2 + 1]) * rs);
             *reinterpret_cast<uint4*>(dst + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
@@ -147,7 +149,10 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
         tmem_ld_32x32b_x32(haddr + c * 32, x);
         tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(x[e]), __uint_as_float(x[e]), ss);
+        for (int e = 0; e < 32; ++e) {
+          const float t = __uint_as_float(x[e]) * rs;
+          ss = fmaf(t, t, ss);
+        }
       }
       rstd = rsqrtf(ss / (float)HD + r.eps);
     }
@@ -162,7 +167,7 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const int j = c * 32 + e;
-          float x = __uint_as_float(lo[e]), y = __uint_as_float(hi[e]);
+          float x = __uint_as_float(lo[e]) * rs, y = __uint_as_float(hi[e]) * rs;
           if (gain != nullptr) {
             x = x * rstd * gain[j];
             y = y * rstd * gain[j + HD / 2];
@@ -314,8 +319,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int row = m * BM + row_in_tile;
       const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+      // rows of a folded RMSNorm arrive un-normalised: their scale comes from the producer's sums
+      float rs = 1.0f;
+      if (p.ss_in != nullptr && row_ok) {
+        float sum = 0.f;
+        for (int i = 0; i < p.ss_cnt; ++i) sum += p.ss_in[(int64_t)row * p.ss_in_ld + i];
+        rs = rsqrtf(sum * p.inv_d + p.eps_in);
+      }
       if (EPI == EPI_QKV_ROPE) {
-        qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok);
+        qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok, rs);
       } else if (EPI == EPI_GATED_BF16) {
         bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
 #pragma unroll 1
@@ -333,8 +345,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   const int e = v * 8 + j * 2;
-                  const float x0 = act_fn(__uint_as_float(gr[e]), p.act) * __uint_as_float(ur[e]);
-                  const float x1 = act_fn(__uint_as_float(gr[e + 1]), p.act) * __uint_as_float(ur[e + 1]);
+                  const float x0 = act_fn(__uint_as_float(gr[e]) * rs, p.act) * (__uint_as_float(ur[e]) * rs);
+                  const float x1 = act_fn(__uint_as_float(gr[e + 1]) * rs, p.act) * (__uint_as_float(ur[e + 1]) * rs);
                   w[j] = pack_bf16(x0, x1);
                 }
                 *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -343,6 +355,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
       } else {
+        float ss = 0.f;                       // EPI_ADD_F32 with hn_out: sum of squares of this row's new values
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t r[32];
@@ -350,6 +363,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tmem_wait_ld();
           const int col0 = n * BN + c * 32;
           if (row_ok) {
+            if (EPI != EPI_ADD_F32) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * rs);
+            }
             if (EPI == EPI_STORE_BF16) {
               bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
 #pragma unroll
@@ -373,6 +390,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   if (EPI == EPI_ADD_F32) {
                     const float4 o = *dst;
                     x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
+                    if (p.hn_out != nullptr) {
+                      ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                      const float4 gn = *reinterpret_cast<const float4*>(p.gain_next + col0 + v * 4);
+                      uint2 h2;
+                      h2.x = pack_bf16(x.x * gn.x, x.y * gn.y);
+                      h2.y = pack_bf16(x.z * gn.z, x.w * gn.w);
+                      *reinterpret_cast<uint2*>(p.hn_out + (int64_t)row * p.ld_hn + col0 + v * 4) = h2;
+                    }
                   }
                   *dst = x;
                 }
@@ -380,6 +405,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           }
         }
+        if (EPI == EPI_ADD_F32 && p.hn_out != nullptr && row_ok) p.ss_out[(int64_t)row * p.ss_ld + n] = ss;
       }
       tc_fence_before();
       __syncwarp();
@@ -446,7 +472,18 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
                          BN);
   if (rc) return rc;
+  if (a.hn_out != nullptr) {
+    if (a.epilogue != EPI_ADD_F32 || a.batch != 1 || !a.gain_next || !a.ss_out || a.ld_hn % 4 ||
+        a.ss_ld < ceil_div(a.N, BN))
+      return POP_E_INVALID;
+  }
+  if (a.ss_in != nullptr && (a.batch != 1 || a.ss_cnt < 1 || a.ss_in_ld < a.ss_cnt || a.norm_d < 1))
+    return POP_E_INVALID;
   GemmDev p{};
+  p.hn_out = a.hn_out; p.ld_hn = a.ld_hn; p.gain_next = a.gain_next; p.ss_out = a.ss_out; p.ss_ld = a.ss_ld;
+  p.ss_in = a.ss_in; p.ss_cnt = a.ss_cnt; p.ss_in_ld = a.ss_in_ld;
+  p.inv_d = a.norm_d > 0 ? 1.0f / (float)a.norm_d : 0.f;
+  p.eps_in = a.norm_eps;
   if (a.epilogue == EPI_QKV_ROPE) {
     const RopeArgs& r = *a.rope;
     p.rope.q_out = r.q_out; p.rope.ldq = r.ldq;

@@ -163,6 +163,44 @@ def test_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm):
     assert (kpool[0] == canary).all() and (kpool[2] == canary).all()   # other layers untouched
 
 
+@pytest.mark.parametrize("M,d,K,F", [(300, 520, 136, 688), (129, 256, 72, 264)])
+def test_rmsnorm_folded_around_the_gemms(L, M, d, K, F):
+    # residual GEMM that also emits the next operand and row sums of squares, then a gated and a
+    # plain GEMM that consume them: together they must equal residual add -> RMSNorm -> GEMM
+    eps = 1e-5
+    A, Wo = _bf((M, K), 40), _bf((d, K), 41, 0.2)
+    x0 = _bf((M, d), 42).float()
+    gain = ps.gains(3, 11, d, True)
+    n_t = (d + 255) // 256
+    x = x0.clone().to(DEV)
+    hn = torch.zeros(M, d, dtype=torch.bfloat16, device=DEV)
+    ss = torch.full((M, n_t + 1), 1e9, dtype=torch.float32, device=DEV)
+    L.gemm_norm(A.to(DEV), Wo.to(DEV), x, 2, hn_out=hn, gain_next=gain.to(DEV), ss_out=ss)
+    assert L.status() == 0
+    x_ref = x0.double() + A.double() @ Wo.double().T
+    assert rel_err(x, x_ref) < 1e-4
+    assert rel_err(ss[:, :n_t].sum(1), x_ref.pow(2).sum(1)) < 1e-4
+    assert (ss[:, n_t] == 1e9).all()
+    assert rel_err(hn, x_ref * gain.double()) < 1e-2
+    h_ref = po.rmsnorm(x_ref, gain.double(), eps)
+    # consumer 1: gated FFN projection
+    Wg, Wu = _bf((F, d), 43, 0.1), _bf((F, d), 44, 0.1)
+    f_pad = (F + 127) // 128 * 128
+    Wgu = torch.zeros(2 * f_pad, d, dtype=torch.bfloat16)
+    for t in range(f_pad // 128):
+        n = min(128, F - t * 128)
+        Wgu[256 * t: 256 * t + n] = Wg[128 * t: 128 * t + n]
+        Wgu[256 * t + 128: 256 * t + 128 + n] = Wu[128 * t: 128 * t + n]
+    act = torch.zeros(M, F, dtype=torch.bfloat16, device=DEV)
+    L.gemm_norm(hn, Wgu.to(DEV), act, 3, act=0, n_valid=F, ss_in=ss[:, :n_t], norm_d=d, norm_eps=eps)
+    assert rel_err(act, po.gated_act(h_ref @ Wg.double().T, h_ref @ Wu.double().T, 0)) < 1e-2
+    # consumer 2: plain fp32 store
+    out = torch.zeros(M, F, dtype=torch.float32, device=DEV)
+    L.gemm_norm(hn, Wg.to(DEV), out, 1, ss_in=ss[:, :n_t], norm_d=d, norm_eps=eps)
+    assert rel_err(out, h_ref @ Wg.double().T) < 1e-2
+    assert L.status() == 0
+
+
 @pytest.mark.parametrize("hd,n_q,n_kv,qk_norm,groups", [(64, 4, 2, 0, 1), (128, 4, 1, 1, 1), (256, 2, 2, 1, 1),
                                                         (128, 0, 2, 1, 3), (64, 3, 3, 0, 1)])
 def test_fused_qkv_projection_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm, groups):
