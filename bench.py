@@ -402,9 +402,26 @@ def run_kernel(a, wl):
             out = torch.zeros(G, M, N, dtype=torch.float32, device=dev)
         work = 2.0 * G * M * N * K
 
-        def launch(i):
-            lib.gemm(A if G > 1 else A[0], B if G > 1 else B[0], out if G > 1 else out[0], epilogue=epi, act=cfg.act,
-                     n_valid=F if epi == 3 else 0)
+        if k in ("gemm_qkv", "kvproj"):
+            # as the path runs them: per-head norm, RoPE and the paged-cache write in the epilogue
+            from paper_2602_03295_b200.binding import KVCache
+            del out
+            n_q = cfg.n_q_heads if k == "gemm_qkv" else 0
+            cache = KVCache(cfg.replace(n_layers=G), wl.batch, wl.seq_len, a.page_size, device=dev)
+            table = torch.zeros(wl.seq_len, hd // 2, 2, dtype=torch.float32, device=dev)
+            lib.rope_table(table, wl.seq_len, hd, cfg.rope_theta)
+            q_out = torch.zeros(M, qd, dtype=torch.bfloat16, device=dev) if n_q else None
+            gq = torch.ones(G, hd, dtype=torch.float32, device=dev) if cfg.qk_norm else None
+
+            def launch(i):
+                lib.gemm_qkv_rope(A if G > 1 else A[0], B if G > 1 else B[0], q_out, cache.k, cache.v, 0,
+                                  cache.block_table, a.page_size, gq if (gq is None or G > 1) else gq[0],
+                                  gq if (gq is None or G > 1) else gq[0], table, n_q, cfg.n_kv_heads, hd,
+                                  wl.seq_len, wl.seq_len, 0, cfg.rms_eps)
+        else:
+            def launch(i):
+                lib.gemm(A if G > 1 else A[0], B if G > 1 else B[0], out if G > 1 else out[0], epilogue=epi,
+                         act=cfg.act, n_valid=F if epi == 3 else 0)
     elif k in ("attention", "attention_local"):
         from paper_2602_03295_b200.binding import KVCache
         window = cfg.window if k == "attention_local" else 0
