@@ -274,6 +274,27 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     return {"K": K, "V": V, "logits": logits, "H": H}
 
 
+def decode_step(cfg, weights, tokens: torch.Tensor, K, V, dtype=torch.float64, precision: str = "exact"):
+    """One decode step of the FULL model over an existing cache (Sec. 2.2, decode stage; Eq. 1-3):
+    POP prunes nothing here ("retaining the full model for decode"). tokens: int [B], the token at
+    position n = current cache length; K, V: lists (one per layer) of [B, n, n_kv, hd].
+    Returns (K', V', logits): caches with n + 1 entries and the next-token logits [B, vocab]."""
+    L = cfg.n_layers
+    B = tokens.shape[0]
+    n = K[0].shape[1]
+    K2 = [torch.empty(B, n + 1, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    V2 = [torch.empty(B, n + 1, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
+    logits = torch.empty(B, cfg.vocab, dtype=dtype)
+    pos = torch.tensor([n])
+    for b in range(B):
+        x = embed(cfg, weights, tokens[b: b + 1], None, dtype)
+        for l in range(1, L + 1):
+            x, K2[l - 1][b], V2[l - 1][b] = layer_forward(cfg, weights, l, x, pos, K[l - 1][b].to(dtype),
+                                                          V[l - 1][b].to(dtype), dtype, precision)
+        logits[b] = lm_logits(cfg, weights, x[0], dtype)
+    return K2, V2, logits
+
+
 # ---------------------------------------------------------------------------------------
 # cost model (counts of the work the method defines; no arithmetic of the method)
 # ---------------------------------------------------------------------------------------

@@ -331,6 +331,30 @@ def test_first_token_depends_on_the_projected_cache():
     assert _maxdiff(pop["logits"], popz["logits"]) > 1e-4
 
 
+@pytest.mark.parametrize("variant", list(VARIANTS))
+def test_decode_steps_reproduce_the_full_prefill_of_the_longer_prompt(variant):
+    # the decode stage is the full model on one more position over the cache (Sec. 2.2): feeding the
+    # tokens of a longer prompt one by one after a full prefill of its first part must give that
+    # longer prompt's cache and last-position logits (causality; nothing of the future is used)
+    cfg, w, tokens = _setup(variant, n=11, batch=2)
+    n0 = 7
+    ref = po.full_prefill(cfg, w, tokens)
+    part = po.full_prefill(cfg, w, tokens[:, :n0])
+    K, V = part["K"], part["V"]
+    for i in range(n0, tokens.shape[1]):
+        K, V, logits = po.decode_step(cfg, w, tokens[:, i], K, V)
+        assert K[0].shape[1] == i + 1
+    assert _maxdiff(logits, ref["logits"]) < 1e-10
+    for l in range(cfg.n_layers):
+        assert _maxdiff(K[l], ref["K"][l]) < 1e-10 and _maxdiff(V[l], ref["V"][l]) < 1e-10
+    # after a pruned prefill the decode step consumes the projected entries: the result differs
+    # from the full model's unless at most one layer was pruned
+    pop = po.pop_prefill(cfg, w, tokens[:, :n0], None, 1)
+    _, _, lg = po.decode_step(cfg, w, tokens[:, n0], pop["K"], pop["V"])
+    part2 = po.decode_step(cfg, w, tokens[:, n0], part["K"], part["V"])[2]
+    assert _maxdiff(lg, part2) > 1e-6
+
+
 def test_single_token_prompt_has_an_empty_first_phase():
     cfg, w, tokens = _setup("llama", n=1)
     pop = po.pop_prefill(cfg, w, tokens, None, 1)
