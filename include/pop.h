@@ -119,6 +119,17 @@ int pop_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq
 int pop_full_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
+/* One decode step of the FULL model over the cache a prefill left (paper Sec. 2.2, decode stage;
+ * Sec. 3: "retaining the full model for decode"): tokens is device int32 [batch], the token of
+ * each sequence at position `pos` = number of entries its cache already holds. Every layer
+ * appends its k, v at `pos` (Eq. 2-3), attends over positions 0..pos (the window in local
+ * layers), and logits_out (device fp32 [batch][vocab]) receives the next-token logits. After
+ * pop_prefill(seq_len = N) the first call uses pos = N. The cache must have room for pos + 1
+ * positions per sequence (POP_E_NOSPACE otherwise); the workspace of any earlier prefill with the
+ * same batch is large enough. Errors as pop_prefill. */
+int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,
+                    float* logits_out, void* stream);
+
 /* Synchronise `stream`, then read and clear the device status word: POP_OK, or
  * POP_E_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or POP_E_CUDA. */
 int pop_last_status(pop_model_t* m, void* stream);

@@ -61,6 +61,7 @@ SIGNATURES = {
     "pop_set_workspace": (C.c_int, [_P, _P, C.c_size_t]),
     "pop_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_full_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
+    "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_last_status": (C.c_int, [_P, _P]),
     "pop_last_launch_count": (_I64, [_P]),
     "pop_free": (None, [_P]),
@@ -402,6 +403,18 @@ class PopModel:
         code = self.lib.dll.pop_full_prefill(self.handle, C.byref(inp), N, B, C.byref(kc), logits.data_ptr(),
                                              _stream_ptr(stream))
         self.lib.check(code, "pop_full_prefill")
+        return logits
+
+    def decode_step(self, tokens, pos: int, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_decode_step: tokens int32 [B] on the device, each at position `pos` of its sequence."""
+        B = tokens.shape[0]
+        self.ensure_workspace(1, B) if self.ws is None else None
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        kc = cache.struct()
+        code = self.lib.dll.pop_decode_step(self.handle, tokens.data_ptr(), pos, B, C.byref(kc), logits.data_ptr(),
+                                            _stream_ptr(stream))
+        self.lib.check(code, "pop_decode_step")
         return logits
 
     def last_status(self, stream=None) -> int:

@@ -38,6 +38,7 @@ struct Workspace {
   bf16* ob;          // [B][q_dim]
   bf16* ab;          // [B][F]
   float* partial;    // [B][n_q][64][hd+2]
+  float2* rope1;     // [hd/2] rotary row of the one position a decode step works on
   size_t total;
 };
 
@@ -131,6 +132,7 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.ob = (bf16*)take((size_t)B * m->q_dim * 2);
   w.ab = (bf16*)take((size_t)B * c.d_ffn * 2);
   w.partial = (float*)take((size_t)B * c.n_q_heads * 64 * (c.head_dim + 2) * 4);
+  w.rope1 = (float2*)take((size_t)(c.head_dim / 2) * 8);
   w.total = o;
   return w;
 }
@@ -234,7 +236,9 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
 }
 
 // Boundary token as a decode step of layer l (paper Sec. 3.3): one row per sequence in w.xb.
-int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc, cudaStream_t s) {
+// `table` holds rotary rows starting at position `table_pos0`.
+int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc,
+                   const float2* table, int table_pos0, cudaStream_t s) {
   const pop_config_t& c = m->cfg;
   const int d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -250,7 +254,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   r.page_size = kc->page_size;
   r.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
-  r.table = w.rope; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
+  r.table = table; r.table_pos0 = table_pos0; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = B; r.rows_per_seq = 1; r.rows_written = 1; r.pos0 = N - 1; r.groups = 1; r.eps = c.rms_eps;
   POP_TRY(launch_rope_cache(r, s));
   DecAttnArgs a{};
@@ -318,11 +322,39 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
       }
     }
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
-    for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, s));
+    for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s));
   } else {
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
   }
   // final norm (kept in fp32) and output head on the last prompt position
+  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
+                         true, s));
+  GemvArgs v{};
+  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
+  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
+  POP_TRY(launch_gemv(v, s));
+  m->last_launches = launch_count() - launches0;
+  return POP_OK;
+}
+
+// One decode step of the full model (paper Sec. 2.2): every sequence's token at position `pos`
+// (= entries already in the cache) goes through all L layers as the boundary token does.
+int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache_t* kc, float* logits,
+               cudaStream_t s) {
+  if (!m || !tokens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits) return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (pos < 0 || B < 1 || pos > (1 << 24)) return POP_E_INVALID;
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(pos + 1, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
+  if ((int64_t)ceil_div(pos + 1, kc->page_size) * B > kc->num_pages) return POP_E_NOSPACE;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, 1, B);
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  const int64_t launches0 = launch_count();
+  const int d = c.d_model;
+  POP_TRY(launch_rope_table(w.rope1, 1, c.head_dim, c.rope_theta, s, pos));
+  POP_TRY(launch_embed(tokens, (const bf16*)(m->arena + m->off_embed), nullptr, w.xb, B, d, c.vocab, s));
+  for (int l = 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s));
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};
@@ -490,6 +522,11 @@ int pop_full_prefill(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int
   if (!m) return POP_E_INVALID;
   return run_prefill(m, in, seq_len, batch, m->cfg.n_layers, kv_cache_out, logits_out,
                      static_cast<cudaStream_t>(stream));
+}
+
+int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,
+                    float* logits_out, void* stream) {
+  return run_decode(m, tokens, pos, batch, kv_cache, logits_out, static_cast<cudaStream_t>(stream));
 }
 
 int pop_last_status(pop_model_t* m, void* stream) {

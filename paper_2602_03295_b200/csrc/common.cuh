@@ -106,7 +106,8 @@ int launch_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_
 int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, const float* gain, int rows, int d,
                         float eps, cudaStream_t s);
 // table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)), pos < n_pos, j < hd/2
-int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s);
+// rows for positions first_pos .. first_pos + n_pos - 1
+int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos = 0);
 struct RopeArgs {
   const float* in; int64_t ld_in; int64_t in_group_stride;   // fp32 rows [q heads | k heads | v heads] * hd
   bf16* q_out; int64_t ldq;                                  // may be null when n_q == 0
@@ -114,7 +115,7 @@ struct RopeArgs {
   int layer0;                                                // cache layer (0-based) of group 0
   const int32_t* block_table; int max_pages_per_seq; int page_size;
   const float* q_gain; const float* k_gain; int64_t gain_group_stride;   // per-head norm gains or null
-  const float2* table;
+  const float2* table; int table_pos0;                      // table row 0 holds position table_pos0
   int n_q, n_kv, hd;
   int rows, rows_per_seq, rows_written, pos0, groups;
   float eps;

@@ -113,13 +113,13 @@ __global__ void postnorm_add_kernel(float* __restrict__ x, int64_t ldx, const fl
 
 // ------------------------------------------------------------------------------ rotary table
 // table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)), evaluated in fp64, stored fp32.
-__global__ void rope_table_kernel(float2* __restrict__ table, int n_pos, int half, double theta) {
+__global__ void rope_table_kernel(float2* __restrict__ table, int n_pos, int half, double theta, int first_pos) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pos * half) return;
   const int pos = i / half, j = i - pos * half;
   const double inv = exp2(-(2.0 * j / (2.0 * half)) * log2(theta));
   double s, c;
-  sincos((double)pos * inv, &s, &c);
+  sincos((double)(first_pos + pos) * inv, &s, &c);
   table[i] = make_float2((float)c, (float)s);
 }
 
@@ -135,7 +135,7 @@ struct RopeDev {
   int layer0;                                              // cache layer of group 0
   const int32_t* block_table; int max_pages_per_seq; int page_size;
   const float* q_gain; const float* k_gain; int64_t gain_group_stride;
-  const float2* table;                                      // [pos][hd/2]
+  const float2* table; int table_pos0;                      // [pos - table_pos0][hd/2]
   int n_q, n_kv, hd;
   int rows, rows_per_seq, rows_written, pos0;
   float eps;
@@ -182,7 +182,7 @@ __global__ void rope_cache_kernel(const RopeDev p) {
     }
 #pragma unroll
     for (int u = 0; u < PER; ++u) {
-      const float2 cs = p.table[(int64_t)pos * (HD / 2) + lane + 32 * u];
+      const float2 cs = p.table[(int64_t)(pos - p.table_pos0) * (HD / 2) + lane + 32 * u];
       const float a = lo[u] * cs.x - hi[u] * cs.y;
       const float c = hi[u] * cs.x + lo[u] * cs.y;
       lo[u] = a;
@@ -249,9 +249,9 @@ int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, cons
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
 
-int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s) {
+int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos) {
   const int total = n_pos * (hd / 2);
-  rope_table_kernel<<<ceil_div(total, 256), 256, 0, s>>>(table, n_pos, hd / 2, (double)theta);
+  rope_table_kernel<<<ceil_div(total, 256), 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, first_pos);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -264,7 +264,7 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   p.layer0 = a.layer0;
   p.block_table = a.block_table; p.max_pages_per_seq = a.max_pages_per_seq; p.page_size = a.page_size;
   p.q_gain = a.q_gain; p.k_gain = a.k_gain; p.gain_group_stride = a.gain_group_stride;
-  p.table = a.table;
+  p.table = a.table; p.table_pos0 = a.table_pos0;
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.hd = a.hd;
   p.rows = a.rows; p.rows_per_seq = a.rows_per_seq; p.rows_written = a.rows_written; p.pos0 = a.pos0;
   p.eps = a.eps;
