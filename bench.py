@@ -271,7 +271,8 @@ def run_ours(a, wl):
     embeds_h = None if embeds_h is None else embeds_h.pin_memory()
     tokens = tokens_h.to(dev)
     embeds = None if embeds_h is None else embeds_h.to(dev)
-    cache = KVCache(cfg, wl.batch, wl.seq_len, a.page_size, device=dev)
+    DECODE_STEPS = 32
+    cache = KVCache(cfg, wl.batch, wl.seq_len + DECODE_STEPS, a.page_size, device=dev)   # room for the decode leg
     logits = torch.empty(wl.batch, cfg.vocab, dtype=torch.float32, device=dev)
     logits_h = torch.empty(wl.batch, cfg.vocab, dtype=torch.float32).pin_memory()
 
@@ -323,6 +324,22 @@ def run_ours(a, wl):
     step_full()
     full_ms = timed(step_full, max(2, a.steps // 2)) / max(2, a.steps // 2)
 
+    # decode stage over the cache the pruned prefill built: the full model, one position per call
+    step()
+    dec_tok = tokens[:, -1].contiguous()
+    for i in range(3):
+        model.decode_step(dec_tok, wl.seq_len + i, cache, logits)
+    barrier()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record()
+    for i in range(DECODE_STEPS):
+        model.decode_step(dec_tok, wl.seq_len + i, cache, logits)
+    d1.record()
+    barrier()
+    dec_ms = max_over_ranks(d0.elapsed_time(d1), dev) / DECODE_STEPS
+    dec_status = model.last_status()
+    weight_bytes = 2.0 * (cfg.n_layers * po.layer_params(cfg) + cfg.vocab * cfg.d_model)
+
     # per-kernel-class durations of one more step, CUDA events on the launching stream
     lib.profile(True)
     step()
@@ -351,6 +368,10 @@ def run_ours(a, wl):
            "clocks": clocks,
            "e2e": {"value": n_tok / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+           "decode": {"ms_per_step": dec_ms, "tokens_per_s": wl.batch * world / (dec_ms * 1e-3),
+                      "context": wl.seq_len, "steps": DECODE_STEPS, "device_status": dec_status,
+                      "weight_stream_gbs": weight_bytes / (dec_ms * 1e-3) / 1e9,
+                      "frac_of_measured_hbm": weight_bytes / (dec_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"]},
            "gpu_launches": int(launches * a.steps),
            "roofline": {"kernel": "gemm_kernel (tcgen05 projection GEMM, all epilogues)", "bound": "tensor",
                         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
