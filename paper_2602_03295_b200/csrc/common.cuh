@@ -40,6 +40,10 @@ int prof_summary(int kind, double* total_ms, double* total_work, int64_t* launch
 // box = [1][box1][box0]; box0 must be 64 (128 bytes).
 int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
                       uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1);
+// 3-D fp32 tensor [dim2][dim1][dim0], 128-byte swizzle, box = [1][box1][32] (32 floats = 128 bytes): the
+// GEMM's output tiles
+int make_tmap_f32_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                     uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box1);
 // rank-`rank` (3..5) bf16 tensor, dims/strides/box given innermost first (strides in elements, for
 // dims 1..rank-1), 128-byte swizzle. Used for Q and for the paged KV pools [page][slot][head][hd].
 int make_tmap_bf16_nd(CUtensorMap* out, const void* base, int rank, const uint64_t dims[5],

@@ -22,10 +22,12 @@ constexpr int B_BYTES = BN * BK * 2;
 constexpr int GEMM_THREADS = 192;
 constexpr int GROUP_M = 16;
 constexpr uint32_t TMEM_COLS = 512;
+constexpr int OUT_STAGE_BYTES = 32 * 32 * 4;
 
 struct __align__(1024) GemmSmem {
   uint8_t a[STAGES][A_BYTES];
   uint8_t b[STAGES][B_BYTES];
+  uint8_t out_stage[4][2][OUT_STAGE_BYTES];   // per epilogue warp: two 32-row x 32-float boxes for TMA stores
   uint64_t full[STAGES];
   uint64_t empty[STAGES];
   uint64_t tfull[2];
@@ -194,7 +196,8 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
 
 template <int EPI, int HD>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p,
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmO, const GemmDev p,
             int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   GemmSmem& s = *reinterpret_cast<GemmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -305,6 +308,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int quarter = warp & 3;              // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
     int it = 0;
+    uint32_t boxes_out = 0;                     // output boxes this warp has handed to the TMA engine
     for (int t = blockIdx.x; t < total_tiles && !s.abort; t += gridDim.x, ++it) {
       const int buf = it & 1;
       const uint32_t bphase = (it >> 1) & 1;
@@ -352,6 +356,41 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
               }
             }
+          }
+        }
+      } else if ((EPI == EPI_ADD_F32 || EPI == EPI_STORE_F32) && p.hn_out == nullptr) {
+        // fp32 outputs leave through shared memory: the thread writes its 32 values of the chunk as one
+        // 128-byte swizzled row of the warp's 32 x 32 box, and an elected lane hands the box to the TMA
+        // engine, which stores it or adds it to the residual at the memory side. No residual value
+        // is read by the SM, rows and columns beyond the output are clipped by the hardware.
+        const bool rows_in = m * BM + quarter * 32 < p.M;     // uniform per warp
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          if (n * BN + c * 32 >= p.N) break;                 // uniform: the rest of the tile is past the last column
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(taddr + c * 32, r);
+          tmem_wait_ld();
+          if (!rows_in) continue;
+          // boxes alternate by the count of boxes handed over, so "at most one group still reading"
+          // always means the other box
+          uint8_t* box = s.out_stage[quarter][boxes_out & 1];
+          ++boxes_out;
+          if (lane == 0) bulk_wait_read_1();
+          __syncwarp();
+          uint8_t* mine = box + lane * 128;
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                   __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+            if (EPI == EPI_STORE_F32) { x.x *= rs; x.y *= rs; x.z *= rs; x.w *= rs; }
+            *reinterpret_cast<float4*>(mine + ((v ^ (lane & 7)) << 4)) = x;
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (EPI == EPI_ADD_F32) tma_reduce_add_3d(&tmO, box, n * BN + c * 32, m * BM + quarter * 32, g);
+            else tma_store_3d(&tmO, box, n * BN + c * 32, m * BM + quarter * 32, g);
+            bulk_commit();
           }
         }
       } else {
@@ -414,6 +453,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 
   // ------------------------------------------------------------------ teardown
+  if (warp >= 2 && lane == 0) bulk_wait_all();   // this lane's output boxes have landed
   __syncwarp();
   tc_fence_before();
   __syncthreads();
@@ -429,7 +469,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 }
 
 template <int EPI, int HD = 0>
-int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, int grid, cudaStream_t stream) {
+int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p, int grid,
+               cudaStream_t stream) {
   const size_t smem = sizeof(GemmSmem) + 1024;
   static bool configured = false;
   if (!configured) {
@@ -440,7 +481,7 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const GemmDev& p, i
   int* status = status_word();
   if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
-  gemm_kernel<EPI, HD><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, p, status);
+  gemm_kernel<EPI, HD><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -479,6 +520,12 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   }
   if (a.ss_in != nullptr && (a.batch != 1 || a.ss_cnt < 1 || a.ss_in_ld < a.ss_cnt || a.norm_d < 1))
     return POP_E_INVALID;
+  CUtensorMap to = ta;   // only the fp32 epilogues use it
+  if ((a.epilogue == EPI_STORE_F32 || a.epilogue == EPI_ADD_F32) && a.hn_out == nullptr) {
+    rc = make_tmap_f32_3d(&to, a.out, a.N, a.M, a.batch, a.ldo,
+                          a.out_batch_stride ? a.out_batch_stride : a.ldo * (int64_t)a.M, 32);
+    if (rc) return rc;
+  }
   GemmDev p{};
   p.hn_out = a.hn_out; p.ld_hn = a.ld_hn; p.gain_next = a.gain_next; p.ss_out = a.ss_out; p.ss_ld = a.ss_ld;
   p.ss_in = a.ss_in; p.ss_cnt = a.ss_cnt; p.ss_in_ld = a.ss_in_ld;
@@ -512,15 +559,15 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
   const int grid = (int)(total < sms ? total : sms);
   switch (a.epilogue) {
-    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, p, grid, stream);
-    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, p, grid, stream);
-    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, p, grid, stream);
-    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, p, grid, stream);
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, stream);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, stream);
+    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, to, p, grid, stream);
+    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, to, p, grid, stream);
     case EPI_QKV_ROPE:
       switch (a.rope->hd) {
-        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, p, grid, stream);
-        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, p, grid, stream);
-        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, p, grid, stream);
+        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, to, p, grid, stream);
+        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, to, p, grid, stream);
+        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, to, p, grid, stream);
       }
       return POP_E_INVALID;
   }
