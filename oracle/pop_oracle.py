@@ -226,7 +226,7 @@ def full_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tens
 
 
 def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], l_keep: int,
-                dtype=torch.float64, precision: str = "exact"):
+                dtype=torch.float64, precision: str = "exact", skip=None):
     """POP inference up to the first generated token, in the paper's two phases (Sec. 3.3).
 
     Phase 1, pruned prefill on x_{1:N-1}: layers 1..L_keep run in full; each layer
@@ -237,10 +237,19 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     Phase 2, first decode step on x_N: one position through all L layers, each appending
     its k, v to the cache (Eq. 2-3) and attending over positions 1..N.
 
+    `skip` (a collection of 1-based layer numbers) states the pruned set S_skip of Eq. 4 / Eq. 14-15
+    explicitly instead of the deep suffix {l_keep+1..L}; it may be shallow or interleaved (the
+    layer-selection ablation of Sec. 4.4). A pruned layer projects whatever state reaches it.
+
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
-    H [B, N-1, d] (the state leaving the kept stack in phase 1)."""
+    H [B, N-1, d] (the state leaving the last layer of phase 1; for the deep-suffix set this is
+    the state leaving the kept stack)."""
     L = cfg.n_layers
-    assert 1 <= l_keep <= L
+    if skip is None:
+        assert 1 <= l_keep <= L
+        skip = set(range(l_keep + 1, L + 1))
+    skip = set(int(l) for l in skip)
+    assert all(1 <= l <= L for l in skip)
     B, N = tokens.shape
     K = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
     V = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
@@ -255,7 +264,7 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
             pos = torch.arange(N - 1)
             x = x_all[: N - 1]
             for l in range(1, L + 1):
-                if l <= l_keep:
+                if l not in skip:
                     x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, pos, None, None,
                                                             dtype, precision)
                 else:

@@ -355,6 +355,41 @@ def test_decode_steps_reproduce_the_full_prefill_of_the_longer_prompt(variant):
     assert _maxdiff(lg, part2) > 1e-6
 
 
+def test_explicit_skip_sets():
+    cfg, w, tokens = _setup("gemma", n=9, batch=2)      # 4 layers
+    L = cfg.n_layers
+    # the deep suffix given as a set is the l_keep form; the empty set is the full model
+    a = po.pop_prefill(cfg, w, tokens, None, 2)
+    b = po.pop_prefill(cfg, w, tokens, None, 0, skip={3, 4})
+    full = po.full_prefill(cfg, w, tokens)
+    none = po.pop_prefill(cfg, w, tokens, None, 0, skip=set())
+    assert _maxdiff(a["logits"], b["logits"]) == 0 and _maxdiff(none["logits"], full["logits"]) < 1e-11
+    for l in range(L):
+        assert _maxdiff(a["K"][l], b["K"][l]) == 0 and _maxdiff(none["V"][l], full["V"][l]) < 1e-11
+    # interleaved set {2, 4}: layer 1 is exact; layer 2 projects x_2 (Eq. 14) and hands it on (Eq. 15),
+    # so kept layer 3 generates its K/V from x_2 as well -- both restated here from the full model's x_2
+    r = po.pop_prefill(cfg, w, tokens, None, 0, skip={2, 4})
+    N = tokens.shape[1]
+    pos = torch.arange(N - 1)
+    for bi in range(tokens.shape[0]):
+        x1 = po.embed(cfg, w, tokens[bi], None, torch.float64)
+        x2, k1, v1 = po.layer_forward(cfg, w, 1, x1, torch.arange(N), None, None, torch.float64, "exact")
+        assert _maxdiff(r["K"][0][bi], k1) < 1e-11
+        k2, v2 = po.kv_generation(cfg, w, 2, x2[: N - 1], pos, torch.float64, "exact")
+        k3, v3 = po.kv_generation(cfg, w, 3, x2[: N - 1], pos, torch.float64, "exact")
+        assert _maxdiff(r["K"][1][bi, : N - 1], k2) < 1e-11 and _maxdiff(r["V"][1][bi, : N - 1], v2) < 1e-11
+        assert _maxdiff(r["K"][2][bi, : N - 1], k3) < 1e-11 and _maxdiff(r["V"][2][bi, : N - 1], v3) < 1e-11
+    # the boundary position runs the full stack: through layer 3 it only meets exact cache entries
+    # (layer 2 projected the exact x_2), so its entries equal the full model's; layer 3's context
+    # entries came from x_2 instead of x_3, which shows in the boundary entry of layer 4
+    for l in range(3):
+        assert _maxdiff(r["K"][l][:, N - 1], full["K"][l][:, N - 1]) < 1e-10
+    assert _maxdiff(r["K"][3][:, N - 1], full["K"][3][:, N - 1]) > 1e-6
+    # a shallow set changes the result differently from a deep set of the same size
+    sh = po.pop_prefill(cfg, w, tokens, None, 0, skip={1, 2})
+    assert _maxdiff(sh["logits"], po.pop_prefill(cfg, w, tokens, None, 2)["logits"]) > 1e-6
+
+
 def test_single_token_prompt_has_an_empty_first_phase():
     cfg, w, tokens = _setup("llama", n=1)
     pop = po.pop_prefill(cfg, w, tokens, None, 1)
