@@ -119,6 +119,16 @@ int pop_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq
 int pop_full_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
+/* pop_prefill for an explicitly given pruned set S_skip (paper Eq. 4 and Eq. 14-15; the shallow /
+ * interleaved selections of the ablation in Sec. 4.4): skip is a HOST array of n_layers bytes,
+ * skip[l-1] != 0 meaning layer l only stores its K/V projections of the state that reaches it and
+ * hands that state on unchanged. Evaluated in the paper's literal two phases (prompt positions
+ * through the layers, then the last prompt token through ALL layers as a decode step), so it costs
+ * n_layers boundary passes where pop_prefill needs n_layers - L_keep; for the deep-suffix set the
+ * two calls agree to rounding. Outputs, conventions and errors as pop_prefill. */
+int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
+                     const uint8_t* skip, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
+
 /* One decode step of the FULL model over the cache a prefill left (paper Sec. 2.2, decode stage;
  * Sec. 3: "retaining the full model for decode"): tokens is device int32 [batch], the token of
  * each sequence at position `pos` = number of entries its cache already holds. Every layer

@@ -61,6 +61,8 @@ SIGNATURES = {
     "pop_set_workspace": (C.c_int, [_P, _P, C.c_size_t]),
     "pop_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_full_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
+    "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
+                                   _P]),
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_last_status": (C.c_int, [_P, _P]),
     "pop_last_launch_count": (_I64, [_P]),
@@ -403,6 +405,19 @@ class PopModel:
         code = self.lib.dll.pop_full_prefill(self.handle, C.byref(inp), N, B, C.byref(kc), logits.data_ptr(),
                                              _stream_ptr(stream))
         self.lib.check(code, "pop_full_prefill")
+        return logits
+
+    def prefill_skip(self, tokens, embeds, skip, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_prefill_skip: `skip` is a collection of 1-based layer numbers pruned during the prefill."""
+        B, N = tokens.shape
+        self.ensure_workspace(N, B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        mask = bytes(1 if (l + 1) in set(skip) else 0 for l in range(self.cfg.n_layers))
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_prefill_skip(self.handle, C.byref(inp), N, B, mask, C.byref(kc), logits.data_ptr(),
+                                             _stream_ptr(stream))
+        self.lib.check(code, "pop_prefill_skip")
         return logits
 
     def decode_step(self, tokens, pos: int, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):

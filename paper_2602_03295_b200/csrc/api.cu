@@ -337,6 +337,46 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
   return POP_OK;
 }
 
+// POP prefill for an arbitrary pruned set S_skip (paper Eq. 4, Eq. 14-15; the layer-selection
+// ablation of Sec. 4.4), in the paper's literal two phases: phase 1 walks the layers over the
+// prompt, a kept layer in full, a pruned layer storing only its K/V projections of the state that
+// reaches it; phase 2 runs the boundary token through ALL layers as a decode step, which also
+// overwrites whatever phase 1 left at the last position of each layer's cache.
+int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const uint8_t* skip, pop_kv_cache_t* kc,
+                     float* logits, cudaStream_t s) {
+  if (!m || !in || !in->tokens || !skip || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
+    return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (N < 1 || B < 1 || (int64_t)N * B > (int64_t)1 << 24) return POP_E_INVALID;
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(N, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
+  if ((int64_t)ceil_div(N, kc->page_size) * B > kc->num_pages) return POP_E_NOSPACE;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, N, B);
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  const int64_t launches0 = launch_count();
+  const int M = B * N, d = c.d_model;
+  POP_TRY(launch_rope_table(w.rope, N, c.head_dim, c.rope_theta, s));
+  POP_TRY(launch_embed(in->tokens, (const bf16*)(m->arena + m->off_embed), (const bf16*)in->embeds, w.x, M, d,
+                       c.vocab, s));
+  POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));       // x_1 of the boundary token, kept for phase 2
+  if (N > 1) {
+    for (int l = 1; l <= c.n_layers; ++l) {
+      if (skip[l - 1]) POP_TRY(pruned_kv(m, w, l, 1, N, B, kc, s));
+      else POP_TRY(full_layer(m, w, l, N, B, kc, s));
+    }
+  }
+  for (int l = 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s));
+  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
+                         true, s));
+  GemvArgs v{};
+  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
+  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
+  POP_TRY(launch_gemv(v, s));
+  m->last_launches = launch_count() - launches0;
+  return POP_OK;
+}
+
 // One decode step of the full model (paper Sec. 2.2): every sequence's token at position `pos`
 // (= entries already in the cache) goes through all L layers as the boundary token does.
 int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache_t* kc, float* logits,
@@ -522,6 +562,11 @@ int pop_full_prefill(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int
   if (!m) return POP_E_INVALID;
   return run_prefill(m, in, seq_len, batch, m->cfg.n_layers, kv_cache_out, logits_out,
                      static_cast<cudaStream_t>(stream));
+}
+
+int pop_prefill_skip(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, const uint8_t* skip,
+                     pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
+  return run_prefill_skip(m, in, seq_len, batch, skip, kv_cache_out, logits_out, static_cast<cudaStream_t>(stream));
 }
 
 int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,

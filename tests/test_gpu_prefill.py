@@ -115,6 +115,30 @@ def test_embedding_rows_as_input():
     check_against(ref, logits, cache, cfg)
 
 
+@pytest.mark.parametrize("variant,skip", [("c1", {1}), ("qknorm", {2, 4}), ("gemma", {1, 3, 5}), ("hd128", {3, 4}),
+                                          ("hd256", set()), ("gemma", {1, 2, 3, 4, 5})])
+@pytest.mark.parametrize("B,N", [(1, 1), (2, 70)])
+def test_explicit_skip_sets(variant, skip, B, N):
+    # shallow, interleaved, deep, empty and complete pruned sets against the oracle's two phases
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS[variant]
+    tokens = ps.uniform_tokens(17, B, N, cfg.vocab)
+    ref = po.pop_prefill(cfg, ps.SynthWeights(cfg), tokens, None, 0, skip=skip)
+    model = build(cfg)
+    cache = KVCache(cfg, B, N, 16, fill=float("nan"))
+    logits = model.prefill_skip(tokens.to(DEV), None, skip, cache)
+    assert model.last_status() == 0
+    check_against(ref, logits, cache, cfg)
+    if skip and skip == set(range(min(skip), cfg.n_layers + 1)):
+        # a deep suffix: the fused form of pop_prefill computes the same function
+        cache2 = KVCache(cfg, B, N, 16, fill=float("nan"))
+        logits2 = model.prefill(tokens.to(DEV), None, min(skip) - 1, cache2) if min(skip) > 1 else None
+        if logits2 is not None:
+            assert (logits2 - logits).abs().max().item() <= 1e-2
+            for l in range(cfg.n_layers):
+                assert rel_err(cache2.gather(l)[0], cache.gather(l)[0]) <= 1e-2
+
+
 class CachedWeights:
     """Draws each synthetic tensor once (the oracle asks for a layer's weights several times)."""
 
