@@ -583,6 +583,28 @@ def run_sweep(a, wl0):
                     "speedup_ceiling_flop_ratio": po.prefill_flops(cfg, bsz, n, None) / flops,
                     "path_tflops": flops / (ms * 1e-3) / 1e12,
                     "frac_of_measured_burst_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}), flush=True)
+            if n == 8192 and bsz == 1:
+                # the same number of pruned layers chosen deep, shallow or interleaved (pop_prefill_skip)
+                P = L // 4
+                sets = {"deep": set(range(L - P + 1, L + 1)), "shallow": set(range(1, P + 1)),
+                        "interleaved": set(range(4, L + 1, 4))}
+                for name, sk in sets.items():
+                    def step_skip():
+                        model.prefill_skip(tokens, None, sk, cache, logits)
+                    for _ in range(3):
+                        step_skip()
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for _ in range(a.steps):
+                        step_skip()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ms = e0.elapsed_time(e1) / a.steps
+                    assert model.last_status() == 0
+                    print(json.dumps({"sweep": wl0.key, "seq_len": n, "batch": bsz, "skip_set": name,
+                                      "pruned_layers": sorted(sk), "ttft_ms": ms, "tokens_per_s": bsz * n / (ms * 1e-3),
+                                      "speedup_vs_full_depth": full_ms / ms}), flush=True)
             del cache, tokens, logits
 
 
