@@ -119,6 +119,16 @@ int pop_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq
 int pop_full_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
+/* pop_prefill for a batch of sequences of DIFFERENT lengths (the paper batches real prompts, Sec. 4.1 /
+ * App. C; padding is not part of the method, so none is used): the sequences are packed back to
+ * back, tokens_or_embeds->tokens is device int32 [sum of lengths] (embeds, if given, device bf16
+ * [sum of lengths][d_model]), seq_lens is a HOST array of `batch` lengths (each >= 1). Sequence b
+ * uses row b of the block table and gets seq_lens[b] cache entries in every layer; its boundary
+ * token is its own last token, and logits_out[b] are the next-token logits after it. The
+ * workspace must be sized for (max length, batch). Other conventions and errors as pop_prefill. */
+int pop_prefill_ragged(pop_model_t* m, const pop_input_t* tokens_or_embeds, const int32_t* seq_lens, int32_t batch,
+                       int32_t L_keep, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
+
 /* pop_prefill for an explicitly given pruned set S_skip (paper Eq. 4 and Eq. 14-15; the shallow /
  * interleaved selections of the ablation in Sec. 4.4): skip is a HOST array of n_layers bytes,
  * skip[l-1] != 0 meaning layer l only stores its K/V projections of the state that reaches it and

@@ -61,6 +61,8 @@ SIGNATURES = {
     "pop_set_workspace": (C.c_int, [_P, _P, C.c_size_t]),
     "pop_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_full_prefill": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
+    "pop_prefill_ragged": (C.c_int, [_P, C.POINTER(pop_input_t), C.POINTER(_I32), _I32, _I32, C.POINTER(pop_kv_cache_t),
+                                     _P, _P]),
     "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
                                    _P]),
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
@@ -405,6 +407,20 @@ class PopModel:
         code = self.lib.dll.pop_full_prefill(self.handle, C.byref(inp), N, B, C.byref(kc), logits.data_ptr(),
                                              _stream_ptr(stream))
         self.lib.check(code, "pop_full_prefill")
+        return logits
+
+    def prefill_ragged(self, tokens, embeds, seq_lens, l_keep: int, cache: KVCache,
+                       logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_prefill_ragged: tokens int32 [sum(seq_lens)] packed on the device, seq_lens a host list."""
+        B = len(seq_lens)
+        self.ensure_workspace(max(seq_lens), B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        lens = (_I32 * B)(*[int(x) for x in seq_lens])
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_prefill_ragged(self.handle, C.byref(inp), lens, B, l_keep, C.byref(kc),
+                                               logits.data_ptr(), _stream_ptr(stream))
+        self.lib.check(code, "pop_prefill_ragged")
         return logits
 
     def prefill_skip(self, tokens, embeds, skip, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):

@@ -39,6 +39,7 @@ struct Workspace {
   bf16* ab;          // [B][F]
   float* partial;    // [B][n_q][64][hd+2]
   float2* rope1;     // [hd/2] rotary row of the one position a decode step works on
+  int32_t* cu;       // [B+1] packed-row prefix sums of a ragged batch
   size_t total;
 };
 
@@ -133,6 +134,7 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.ab = (bf16*)take((size_t)B * c.d_ffn * 2);
   w.partial = (float*)take((size_t)B * c.n_q_heads * 64 * (c.head_dim + 2) * 4);
   w.rope1 = (float2*)take((size_t)(c.head_dim / 2) * 8);
+  w.cu = (int32_t*)take((size_t)(B + 1) * 4);
   w.total = o;
   return w;
 }
@@ -144,9 +146,12 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   } while (0)
 
 // one full decoder layer (paper Eq. 1-3) on all M = B*N rows of the residual stream
-int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc, cudaStream_t s) {
+// Ragged batches: `cu` (device prefix sums, B + 1 entries) and `rows` (total packed rows) replace the
+// uniform B x N layout; N is then the longest sequence.
+int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc, cudaStream_t s,
+               const int32_t* cu = nullptr, int rows = 0) {
   const pop_config_t& c = m->cfg;
-  const int M = B * N, d = c.d_model;
+  const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
   POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_in), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
   // QKV projection with per-head norm, RoPE and the cache append (Eq. 2-3) in the GEMM's epilogue
@@ -159,6 +164,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   r.table = w.rope; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = M; r.rows_per_seq = N; r.rows_written = N; r.pos0 = 0; r.groups = 1; r.eps = c.rms_eps;
+  r.cu_seqlens = cu; r.batch = B; r.skip_last = 0;
   GemmArgs g{};
   g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
   g.M = M; g.N = m->qkv_dim; g.K = d; g.batch = 1; g.epilogue = EPI_QKV_ROPE; g.rope = &r;
@@ -168,7 +174,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   a.k_pool = (const bf16*)kc->k_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.v_pool = (const bf16*)kc->v_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.block_table = kc->block_table; a.out = w.ao; a.ldo = m->q_dim;
-  a.batch = B; a.seq_len = N; a.q_pos0 = 0; a.kv_len = N;
+  a.batch = B; a.seq_len = N; a.q_pos0 = 0; a.kv_len = N; a.cu_seqlens = cu; a.total_rows = cu ? M : 0;
   a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim;
   a.page_size = kc->page_size; a.num_pages = kc->num_pages; a.max_pages_per_seq = kc->max_pages_per_seq;
   a.window = layer_window(c, l);
@@ -209,9 +215,9 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
 // Independent K/V projections of pruned layers l0..l0+n-1 (paper Eq. 14) from the state H held in
 // w.x, for positions 0..N-2 of every sequence; the state itself is left unchanged (Eq. 15).
 int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, const pop_kv_cache_t* kc,
-              cudaStream_t s) {
+              cudaStream_t s, const int32_t* cu = nullptr, int rows = 0) {
   const pop_config_t& c = m->cfg;
-  const int M = B * N, d = c.d_model;
+  const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
   POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l0, m->lo.ln_in), (int64_t)(m->layer_stride / 4), w.hn, d,
                          (int64_t)M * d, M, d, n, c.rms_eps, false, s));
@@ -225,6 +231,7 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   r.gain_group_stride = (int64_t)(m->layer_stride / 4);
   r.table = w.rope; r.n_q = 0; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = M; r.rows_per_seq = N; r.rows_written = N - 1; r.pos0 = 0; r.groups = n; r.eps = c.rms_eps;
+  r.cu_seqlens = cu; r.batch = B; r.skip_last = 1;
   // ONE batched GEMM over the pruned layers (the layer is the batch dimension of both operands);
   // its epilogue applies each layer's K norm and RoPE and writes the layer's cache entries
   GemmArgs g{};
@@ -238,7 +245,7 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
 // Boundary token as a decode step of layer l (paper Sec. 3.3): one row per sequence in w.xb.
 // `table` holds rotary rows starting at position `table_pos0`.
 int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc,
-                   const float2* table, int table_pos0, cudaStream_t s) {
+                   const float2* table, int table_pos0, cudaStream_t s, const int32_t* cu = nullptr) {
   const pop_config_t& c = m->cfg;
   const int d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -256,6 +263,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   r.table = table; r.table_pos0 = table_pos0; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = B; r.rows_per_seq = 1; r.rows_written = 1; r.pos0 = N - 1; r.groups = 1; r.eps = c.rms_eps;
+  r.cu_seqlens = cu; r.batch = B;
   POP_TRY(launch_rope_cache(r, s));
   DecAttnArgs a{};
   a.q = w.qb; a.ldq = m->q_dim;
@@ -264,6 +272,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.block_table = kc->block_table; a.max_pages_per_seq = kc->max_pages_per_seq; a.page_size = kc->page_size;
   a.partial = w.partial; a.out = w.ob; a.ldo = m->q_dim;
   a.batch = B; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads; a.head_dim = c.head_dim; a.kv_len = N;
+  a.cu_seqlens = cu;
   a.window = layer_window(c, l);
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};
@@ -327,6 +336,58 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
   }
   // final norm (kept in fp32) and output head on the last prompt position
+  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
+                         true, s));
+  GemvArgs v{};
+  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
+  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
+  POP_TRY(launch_gemv(v, s));
+  m->last_launches = launch_count() - launches0;
+  return POP_OK;
+}
+
+// pop_prefill for sequences of different lengths, packed back to back (no padding rows).
+int run_prefill_ragged(pop_model* m, const pop_input_t* in, const int32_t* seq_lens, int B, int L_keep,
+                       pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
+  if (!m || !in || !in->tokens || !seq_lens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
+    return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (B < 1 || B > 4096 || L_keep < 1 || L_keep > c.n_layers) return POP_E_INVALID;
+  std::vector<int32_t> cu(B + 1, 0);
+  int N = 0;
+  for (int b = 0; b < B; ++b) {
+    if (seq_lens[b] < 1) return POP_E_INVALID;
+    if ((int64_t)cu[b] + seq_lens[b] > (int64_t)1 << 24) return POP_E_INVALID;
+    cu[b + 1] = cu[b] + seq_lens[b];
+    N = std::max(N, (int)seq_lens[b]);
+  }
+  const int T = cu[B];
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(N, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, N, B);        // laid out for B x N rows >= T
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  const int64_t launches0 = launch_count();
+  const int d = c.d_model;
+  // the prefix sums travel through the stream like everything else (the host vector is pageable
+  // memory, which the runtime stages before returning)
+  if (cudaMemcpyAsync(w.cu, cu.data(), (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return POP_E_CUDA;
+  POP_TRY(launch_rope_table(w.rope, N, c.head_dim, c.rope_theta, s));
+  POP_TRY(launch_embed(in->tokens, (const bf16*)(m->arena + m->off_embed), (const bf16*)in->embeds, w.x, T, d,
+                       c.vocab, s));
+  for (int l = 1; l <= L_keep; ++l) POP_TRY(full_layer(m, w, l, N, B, kc, s, w.cu, T));
+  if (L_keep < c.n_layers) {
+    if (T > B) {      // some sequence has more than its boundary token
+      for (int l0 = L_keep + 1; l0 <= c.n_layers; l0 += kMaxPrunedChunk) {
+        const int n = std::min(kMaxPrunedChunk, c.n_layers - l0 + 1);
+        POP_TRY(pruned_kv(m, w, l0, n, N, B, kc, s, w.cu, T));
+      }
+    }
+    POP_TRY(launch_gather_last_rows(w.x, w.xb, B, d, w.cu, s));
+    for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s, w.cu));
+  } else {
+    POP_TRY(launch_gather_last_rows(w.x, w.xb, B, d, w.cu, s));
+  }
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};
@@ -562,6 +623,12 @@ int pop_full_prefill(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int
   if (!m) return POP_E_INVALID;
   return run_prefill(m, in, seq_len, batch, m->cfg.n_layers, kv_cache_out, logits_out,
                      static_cast<cudaStream_t>(stream));
+}
+
+int pop_prefill_ragged(pop_model_t* m, const pop_input_t* in, const int32_t* seq_lens, int32_t batch, int32_t L_keep,
+                       pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
+  return run_prefill_ragged(m, in, seq_lens, batch, L_keep, kv_cache_out, logits_out,
+                            static_cast<cudaStream_t>(stream));
 }
 
 int pop_prefill_skip(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, const uint8_t* skip,

@@ -78,6 +78,7 @@ struct AttnDev {
   int window;
   int q_tiles;
   float scale_log2;     // log2(e) / sqrt(hd)
+  const int32_t* cu;    // ragged batches: packed-row prefix sums [batch + 1], or null
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -122,9 +123,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int b = blockIdx.z;
   const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
   const int q_row0 = q_tile * 128;                       // row within the sequence
+  // a ragged batch gives every sequence its own length; query tiles past its end have nothing to do
+  const int row_base = p.cu ? p.cu[b] : b * p.seq_len;   // first packed row of the sequence
+  const int seq_len = p.cu ? p.cu[b + 1] - row_base : p.seq_len;
+  const int kv_len = p.cu ? seq_len : p.kv_len;
+  if (q_row0 >= seq_len) return;
   const int pos0 = p.q_pos0 + q_row0;                    // absolute position of row 0
-  const int last_pos = min(pos0 + 127, p.q_pos0 + p.seq_len - 1);
-  const int j_hi = min(last_pos, p.kv_len - 1) / BKV;
+  const int last_pos = min(pos0 + 127, p.q_pos0 + seq_len - 1);
+  const int j_hi = min(last_pos, kv_len - 1) / BKV;
   const int j_lo = p.window > 0 ? max(0, pos0 - p.window + 1) / BKV : 0;
   const int n_tiles = j_hi - j_lo + 1;
 
@@ -162,7 +168,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       mbar_expect_tx(&s.q_full, NQT * C::Q_TILE_BYTES);
       for (int t = 0; t < NQT; ++t)
         for (int c = 0; c < HD / 64; ++c)
-          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, b * p.seq_len + q_row0);
+          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, row_base + q_row0);
       const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
       const int loads_per_tile = BKV / p.rows_per_load;
       // ring order = the order the MMA warp consumes: K_0, K_1, then V_j, K_{j+2} for j = 0, 1, ...
@@ -180,7 +186,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         int n_loads = 0;
         for (int r = 0; r < loads_per_tile; ++r)
-          if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
+          if (kv0 + r * p.rows_per_load < kv_len) ++n_loads;
         mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
         for (int r = 0; r < n_loads; ++r) {
           const int pos = kv0 + r * p.rows_per_load;
@@ -376,10 +382,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       // cache rows at positions >= kv_len may hold anything: zero them in the staged V tile so that
       // 0 * garbage cannot poison the accumulator (only the last key tile can contain such rows,
       // and its V tile is the last entry of the ring)
-      if (kv0 + BKV > p.kv_len) {
+      if (kv0 + BKV > kv_len) {
         const int rv = 2 * n_tiles - 1;
         if (!mbar_wait(&s.kv_full[rv % STAGES], (rv / STAGES) & 1)) { ok = false; break; }
-        if (t == 0 && row < BKV && kv0 + row >= p.kv_len) {
+        if (t == 0 && row < BKV && kv0 + row >= kv_len) {
           for (int c = 0; c < HD / 64; ++c) {
             uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + row * 128);
 #pragma unroll
@@ -399,8 +405,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tc_fence_after();
         const float inv = 1.0f / l_run;
         const int seq_row = q_row0 + row;
-        const bool store = seq_row < p.seq_len;
-        bf16* out = p.out + ((int64_t)b * p.seq_len + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
+        const bool store = seq_row < seq_len;
+        bf16* out = p.out + ((int64_t)row_base + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
           uint32_t o[32];
@@ -496,9 +502,13 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int b = blockIdx.z;
   const int kv_head = head0 * p.n_kv_heads / p.n_q_heads;
   const int q_row0 = q_tile * 128;
+  const int row_base = p.cu ? p.cu[b] : b * p.seq_len;   // ragged batches: see attn_kernel
+  const int seq_len = p.cu ? p.cu[b + 1] - row_base : p.seq_len;
+  const int kv_len = p.cu ? seq_len : p.kv_len;
+  if (q_row0 >= seq_len) return;
   const int pos0 = p.q_pos0 + q_row0;
-  const int last_pos = min(pos0 + 127, p.q_pos0 + p.seq_len - 1);
-  const int j_hi = min(last_pos, p.kv_len - 1) / BKV;
+  const int last_pos = min(pos0 + 127, p.q_pos0 + seq_len - 1);
+  const int j_hi = min(last_pos, kv_len - 1) / BKV;
   const int j_lo = p.window > 0 ? max(0, pos0 - p.window + 1) / BKV : 0;
   const int n_tiles = j_hi - j_lo + 1;                   // 64-key tiles
   const int n_pairs = (n_tiles + 1) >> 1;
@@ -538,7 +548,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_expect_tx(&s.q_full, NQT * C::Q_TILE_BYTES);
       for (int t = 0; t < NQT; ++t)
         for (int c = 0; c < HD / 64; ++c)
-          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, b * p.seq_len + q_row0);
+          tma_load_3d(s.q[t] + c * 16384, &tmQ, &s.q_full, c * 64, head0 + t, row_base + q_row0);
       const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
       const int loads_per_tile = PKV / p.rows_per_load;
       // ring order: K_0, V_0, K_1, V_1, ... (128-key stages)
@@ -556,7 +566,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         int n_loads = 0;
         for (int r = 0; r < loads_per_tile; ++r)
-          if (kv0 + r * p.rows_per_load < p.kv_len) ++n_loads;
+          if (kv0 + r * p.rows_per_load < kv_len) ++n_loads;
         mbar_expect_tx(&s.kv_full[stage], n_loads * p.rows_per_load * HD * 2);
         for (int r = 0; r < n_loads; ++r) {
           const int pos = kv0 + r * p.rows_per_load;
@@ -739,10 +749,10 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // cache rows at positions >= kv_len may hold anything: zero them in the pair's staged V tile
       // (128 rows, one per thread of warpgroup 0) before either half's product can read them
       const int pair_kv0 = (j_lo + 2 * J) * BKV;
-      if (pair_kv0 + PKV > p.kv_len) {
+      if (pair_kv0 + PKV > kv_len) {
         const int rv = 2 * J + 1;
         if (!mbar_wait(&s.kv_full[rv % STAGES], (rv / STAGES) & 1)) { ok = false; break; }
-        if (t == 0 && pair_kv0 + row >= p.kv_len) {
+        if (t == 0 && pair_kv0 + row >= kv_len) {
           for (int c = 0; c < HD / 64; ++c) {
             uint4* dst = reinterpret_cast<uint4*>(s.kv[rv % STAGES] + c * C::KV_SUB_BYTES + row * 128);
 #pragma unroll
@@ -762,8 +772,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tc_fence_after();
         const float inv = 1.0f / l_run;
         const int seq_row = q_row0 + row;
-        const bool store = seq_row < p.seq_len;
-        bf16* out = p.out + ((int64_t)b * p.seq_len + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
+        const bool store = seq_row < seq_len;
+        bf16* out = p.out + ((int64_t)row_base + seq_row) * p.ldo + (int64_t)(head0 + t) * HD;
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
           uint32_t o[32];
@@ -818,14 +828,15 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
   p.window = a.window;
   p.q_tiles = ceil_div(a.seq_len, 128);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  p.cu = a.cu_seqlens;
   if (C::BKV % p.rows_per_load) return POP_E_INVALID;
 
   CUtensorMap tq, tk, tv;
   // Q [batch*seq][heads][hd] (row stride ldq)
   {
-    const uint64_t dims[5] = {(uint64_t)HD, (uint64_t)a.n_q_heads, (uint64_t)a.batch * a.seq_len, 1, 1};
-    const uint64_t str[4] = {(uint64_t)HD, (uint64_t)a.ldq, (uint64_t)a.ldq * a.batch * a.seq_len,
-                             (uint64_t)a.ldq * a.batch * a.seq_len};
+    const uint64_t rows = a.total_rows > 0 ? (uint64_t)a.total_rows : (uint64_t)a.batch * a.seq_len;
+    const uint64_t dims[5] = {(uint64_t)HD, (uint64_t)a.n_q_heads, rows, 1, 1};
+    const uint64_t str[4] = {(uint64_t)HD, (uint64_t)a.ldq, (uint64_t)a.ldq * rows, (uint64_t)a.ldq * rows};
     const uint32_t box[5] = {64, 1, 128, 1, 1};
     int rc = make_tmap_bf16_nd(&tq, a.q, 3, dims, str, box);
     if (rc) return rc;
@@ -879,6 +890,7 @@ int launch_attention(const AttnArgs& a, cudaStream_t stream) {
   if (a.n_q_heads % a.n_kv_heads || !page_size_ok(a.page_size) || a.ldq % 8 || a.ldo % 8)
     return POP_E_INVALID;
   if (a.q_pos0 + a.seq_len > a.kv_len) return POP_E_INVALID;
+  if (a.cu_seqlens != nullptr && (a.q_pos0 != 0 || a.kv_len != a.seq_len)) return POP_E_INVALID;
   if ((int64_t)ceil_div(a.kv_len, a.page_size) > a.max_pages_per_seq) return POP_E_NOSPACE;
   const bool pair = (a.n_q_heads / a.n_kv_heads) % 2 == 0;
   switch (a.head_dim) {

@@ -94,6 +94,11 @@ struct AttnArgs {
   const int32_t* block_table;            // device [batch][max_pages_per_seq]
   bf16* out; int64_t ldo;                // [batch*seq_len][ldo]
   int batch, seq_len, q_pos0, kv_len;
+  // ragged batches: device int32 [batch + 1] prefix sums of the sequence lengths over packed rows;
+  // sequence b then has cu[b+1] - cu[b] query rows and as many cache positions (seq_len / kv_len
+  // give the maximum over the batch, q_pos0 must be 0); null = every sequence has seq_len rows
+  const int32_t* cu_seqlens;
+  int total_rows;                        // rows of q / out when packed (0 = batch * seq_len)
   int n_q_heads, n_kv_heads, head_dim;
   int page_size, num_pages, max_pages_per_seq;
   int window;
@@ -123,9 +128,16 @@ struct RopeArgs {
   int n_q, n_kv, hd;
   int rows, rows_per_seq, rows_written, pos0, groups;
   float eps;
+  // ragged batches (null = uniform). In the GEMM epilogue: packed row r belongs to the sequence b with
+  // cu[b] <= r < cu[b+1], position r - cu[b]; the last `skip_last` positions of each sequence are not
+  // written. In launch_rope_cache it is only used for boundary rows (rows == batch): row b sits at
+  // position cu[b+1] - cu[b] - 1.
+  const int32_t* cu_seqlens; int batch; int skip_last;
 };
 int launch_rope_cache(const RopeArgs& a, cudaStream_t s);
 int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s);
+// dst[b][:] = src[cu[b+1] - 1][:]: the last row of every packed sequence
+int launch_gather_last_rows(const float* src, float* dst, int batch, int d, const int32_t* cu, cudaStream_t s);
 
 // ------------------------------------------------------------------------------------ boundary path
 struct GemvArgs {
@@ -142,6 +154,7 @@ struct DecAttnArgs {
   float* partial;                            // [batch][n_q][splits][hd + 2] fp32 scratch
   bf16* out; int64_t ldo;
   int batch, n_q, n_kv, head_dim, kv_len, window;
+  const int32_t* cu_seqlens;   // ragged: sequence b has cu[b+1] - cu[b] cache positions (kv_len = their maximum)
 };
 int decode_attn_splits(int kv_len, int window);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

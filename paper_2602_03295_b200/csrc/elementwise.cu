@@ -139,6 +139,7 @@ struct RopeDev {
   int n_q, n_kv, hd;
   int rows, rows_per_seq, rows_written, pos0;
   float eps;
+  const int32_t* cu;      // boundary rows of a ragged batch: row b sits at position cu[b+1] - cu[b] - 1
 };
 
 template <int HD>
@@ -155,7 +156,7 @@ __global__ void rope_cache_kernel(const RopeDev p) {
   const int b = row / p.rows_per_seq;
   const int i = row - b * p.rows_per_seq;
   if (i >= p.rows_written) return;
-  const int pos = p.pos0 + i;
+  const int pos = p.cu ? p.cu[b + 1] - p.cu[b] - 1 : p.pos0 + i;
   const float* src = p.in + (int64_t)g * p.in_group_stride + (int64_t)row * p.ld_in + (int64_t)h * HD;
   float lo[PER], hi[PER];                 // elements j and j + HD/2, j = lane + 32*u
 #pragma unroll
@@ -215,6 +216,15 @@ __global__ void gather_rows_kernel(const float* __restrict__ src, float* __restr
     *reinterpret_cast<float4*>(o + c) = *reinterpret_cast<const float4*>(s + c);
 }
 
+// dst[b][:] = src[cu[b+1] - 1][:]
+__global__ void gather_last_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int d,
+                                        const int32_t* __restrict__ cu) {
+  const float* s = src + (int64_t)(cu[blockIdx.x + 1] - 1) * d;
+  float* o = dst + (int64_t)blockIdx.x * d;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4)
+    *reinterpret_cast<float4*>(o + c) = *reinterpret_cast<const float4*>(s + c);
+}
+
 }  // namespace
 
 int launch_embed(const int32_t* tokens, const bf16* table, const bf16* embeds, float* x, int rows, int d, int vocab,
@@ -268,6 +278,8 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.hd = a.hd;
   p.rows = a.rows; p.rows_per_seq = a.rows_per_seq; p.rows_written = a.rows_written; p.pos0 = a.pos0;
   p.eps = a.eps;
+  p.cu = a.cu_seqlens;
+  if (a.cu_seqlens != nullptr && a.rows_per_seq != 1) return POP_E_INVALID;
   const int heads = a.n_q + 2 * a.n_kv;
   const int64_t items = (int64_t)a.rows * heads;
   dim3 grid((unsigned)((items + 7) / 8), a.groups);
@@ -284,6 +296,12 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
 
 int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s) {
   gather_rows_kernel<<<batch, 256, 0, s>>>(src, dst, d, rows_per_seq, row);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+int launch_gather_last_rows(const float* src, float* dst, int batch, int d, const int32_t* cu, cudaStream_t s) {
+  gather_last_rows_kernel<<<batch, 256, 0, s>>>(src, dst, d, cu);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

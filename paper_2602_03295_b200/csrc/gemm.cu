@@ -48,6 +48,7 @@ struct RopeEpi {
   int n_q, n_kv;
   int rows_per_seq, rows_written, pos0;
   float eps;
+  const int32_t* cu; int batch; int skip_last;    // ragged batches (see RopeArgs)
 };
 
 struct GemmDev {
@@ -96,9 +97,23 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
   const RopeEpi& r = p.rope;
   constexpr int HALF_CHUNKS = HD / 64;                   // 32-column chunks per half head
   const int total_heads = r.n_q + 2 * r.n_kv;
-  const int b = row / r.rows_per_seq;
-  const int i = row - b * r.rows_per_seq;
-  const bool active = row_ok && i < r.rows_written;
+  int b, i;
+  bool active;
+  if (r.cu != nullptr) {
+    // packed rows: the sequence is the last one starting at or before this row
+    int lo = 0, hi = r.batch;                            // cu[lo] <= row < cu[hi] once row < cu[batch]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (r.cu[mid] <= row) lo = mid; else hi = mid;
+    }
+    b = lo;
+    i = row - r.cu[b];
+    active = row_ok && row < r.cu[r.batch] && i < r.cu[b + 1] - r.cu[b] - r.skip_last;
+  } else {
+    b = row / r.rows_per_seq;
+    i = row - b * r.rows_per_seq;
+    active = row_ok && i < r.rows_written;
+  }
   const int pos = r.pos0 + i;
   int64_t cache_row = 0;
   if (active) {
@@ -498,7 +513,9 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     if (!r || !r->k_pool || !r->v_pool || !r->block_table || !r->table || (r->n_q > 0 && !r->q_out))
       return POP_E_INVALID;
     if ((r->hd != 64 && r->hd != 128 && r->hd != 256) || a.N != (r->n_q + 2 * r->n_kv) * r->hd) return POP_E_INVALID;
-    if (r->ldq % 8 || r->rows_per_seq < 1 || a.M % r->rows_per_seq) return POP_E_INVALID;
+    if (r->ldq % 8) return POP_E_INVALID;
+    if (r->cu_seqlens == nullptr && (r->rows_per_seq < 1 || a.M % r->rows_per_seq)) return POP_E_INVALID;
+    if (r->cu_seqlens != nullptr && (r->batch < 1 || r->skip_last < 0)) return POP_E_INVALID;
   } else if (a.epilogue == EPI_GATED_BF16) {
     if (a.N % 256 || a.n_valid % 8 || a.n_valid > a.N / 2 || a.ldo % 8) return POP_E_INVALID;
   } else if (a.epilogue == EPI_STORE_BF16) {
@@ -543,6 +560,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     p.rope.n_q = r.n_q; p.rope.n_kv = r.n_kv;
     p.rope.rows_per_seq = r.rows_per_seq; p.rope.rows_written = r.rows_written; p.rope.pos0 = r.pos0;
     p.rope.eps = r.eps;
+    p.rope.cu = r.cu_seqlens; p.rope.batch = r.batch; p.rope.skip_last = r.skip_last;
   }
   p.out = a.out;
   p.ldo = a.ldo;

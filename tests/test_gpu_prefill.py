@@ -139,6 +139,34 @@ def test_explicit_skip_sets(variant, skip, B, N):
                 assert rel_err(cache2.gather(l)[0], cache.gather(l)[0]) <= 1e-2
 
 
+@pytest.mark.parametrize("variant", list(TINY_VARIANTS))
+@pytest.mark.parametrize("lens,l_keep,page", [([1, 17, 130, 64], 2, 16), ([200], 1, 64), ([129, 1, 1, 300, 5], 3, 128)])
+def test_ragged_batch(variant, lens, l_keep, page):
+    # sequences of different lengths packed without padding: each must equal the oracle run on that
+    # sequence alone (its own boundary token, its own number of cache entries)
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS[variant]
+    l_keep = min(l_keep, cfg.n_layers)
+    w = ps.SynthWeights(cfg)
+    seqs = [ps.uniform_tokens(50 + i, 1, n, cfg.vocab) for i, n in enumerate(lens)]
+    packed = torch.cat([t[0] for t in seqs]).contiguous()
+    model = build(cfg)
+    cache = KVCache(cfg, len(lens), max(lens), page, fill=float("nan"))
+    logits = model.prefill_ragged(packed.to(DEV), None, lens, l_keep, cache)
+    assert model.last_status() == 0
+    assert not torch.isnan(logits).any()
+    for b, (t, n) in enumerate(zip(seqs, lens)):
+        ref = po.pop_prefill(cfg, w, t, None, l_keep)
+        assert (logits[b].cpu().double() - ref["logits"][0]).abs().max().item() <= LOGIT_TOL, f"seq {b}"
+        for l in range(cfg.n_layers):
+            k, v = cache.gather(l, n)
+            assert rel_err(k[b], ref["K"][l][0]) <= KV_TOL and rel_err(v[b], ref["V"][l][0]) <= KV_TOL, (b, l)
+            # nothing was written past the sequence's own length
+            if n < max(lens):
+                kk, _ = cache.gather(l, max(lens))
+                assert torch.isnan(kk[b, n:].float()).all()
+
+
 class CachedWeights:
     """Draws each synthetic tensor once (the oracle asks for a layer's weights several times)."""
 
