@@ -605,6 +605,27 @@ def run_sweep(a, wl0):
                     print(json.dumps({"sweep": wl0.key, "seq_len": n, "batch": bsz, "skip_set": name,
                                       "pruned_layers": sorted(sk), "ttft_ms": ms, "tokens_per_s": bsz * n / (ms * 1e-3),
                                       "speedup_vs_full_depth": full_ms / ms}), flush=True)
+            if n == 8192 and bsz == 8:
+                # a ragged batch of eight prompts packed without padding against the same prompts padded to 8192
+                lens = [8192, 6144, 4096, 3072, 2048, 1024, 512, 128]
+                packed = torch.cat([tokens[i, :m] for i, m in enumerate(lens)]).contiguous()
+
+                def step_ragged():
+                    model.prefill_ragged(packed, None, lens, L * 3 // 4, cache, logits)
+                for _ in range(3):
+                    step_ragged()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(a.steps):
+                    step_ragged()
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / a.steps
+                assert model.last_status() == 0
+                print(json.dumps({"sweep": wl0.key, "ragged_lens": lens, "l_keep": L * 3 // 4, "ttft_ms": ms,
+                                  "real_tokens_per_s": sum(lens) / (ms * 1e-3),
+                                  "padded_to_8192_ttft_ms_same_l_keep": "see the N 8192, B 8 row"}), flush=True)
             del cache, tokens, logits
 
 
