@@ -66,9 +66,9 @@ def resolve_workload(a) -> ps.Workload:
 
 
 # DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
-# summarised in profiles/gemm_kernel_down_proj_c2.md; valid only for the kernel source it was taken on.
+# summarised in profiles/gemm_kernel_residual_proj_c2.md; valid only for the kernel source it was taken on.
 GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
-                "gemm_cu_sha256": "55d87e9265ba3789f5865e87e4fcb2adaec5880f34312f8f26c95cf5b4affc99"}
+                "gemm_cu_sha256": "569bc6fe80dddbecdbc1b12b0b3fb7a58d2b68bd9e3695c2668d2888855c019e"}
 
 
 def gemm_traffic():
