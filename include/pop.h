@@ -150,6 +150,20 @@ int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_
 int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,
                     float* logits_out, void* stream);
 
+/* Greedy generation on the device (the decode stage of paper Sec. 2.2 run as a loop): starting from
+ * first_tokens (device int32 [batch], the token of each sequence at position pos0 -- normally the
+ * arg-max of the prefill's logits), n_steps times: one full-model decode step as pop_decode_step,
+ * then the arg-max of its logits (lowest index among equal values) becomes the next token.
+ * tokens_out (device int32 [batch][n_steps]) receives the generated tokens: tokens_out[b][i] is
+ * the token at position pos0 + i + 1. logits_scratch is device fp32 [batch][vocab] (it holds the
+ * last step's logits afterwards). One step is captured into a CUDA graph whose kernels read the
+ * position from device memory, and that graph is launched n_steps times on `stream`, so the host
+ * issues n_steps graph launches instead of n_steps x (9 n_layers + 5) kernel launches. The call
+ * creates and destroys a stream and a graph of its own (host-side objects; no device memory).
+ * Not available while pop_k_profile is on. The cache must have room for pos0 + n_steps positions. */
+int pop_generate_greedy(pop_model_t* m, const int32_t* first_tokens, int32_t pos0, int32_t n_steps, int32_t batch,
+                        pop_kv_cache_t* kv_cache, int32_t* tokens_out, float* logits_scratch, void* stream);
+
 /* Synchronise `stream`, then read and clear the device status word: POP_OK, or
  * POP_E_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or POP_E_CUDA. */
 int pop_last_status(pop_model_t* m, void* stream);

@@ -66,6 +66,7 @@ SIGNATURES = {
     "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
                                    _P]),
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
+    "pop_generate_greedy": (C.c_int, [_P, _P, _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P, _P]),
     "pop_last_status": (C.c_int, [_P, _P]),
     "pop_last_launch_count": (_I64, [_P]),
     "pop_free": (None, [_P]),
@@ -447,6 +448,21 @@ class PopModel:
                                             _stream_ptr(stream))
         self.lib.check(code, "pop_decode_step")
         return logits
+
+    def generate_greedy(self, first_tokens, pos0: int, n_steps: int, cache: KVCache,
+                        logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_generate_greedy: returns (tokens int32 [B, n_steps] on the device, last logits)."""
+        B = first_tokens.shape[0]
+        if self.ws is None:
+            self.ensure_workspace(1, B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        out = torch.full((B, n_steps), -1, dtype=torch.int32, device=self.device)
+        kc = cache.struct()
+        code = self.lib.dll.pop_generate_greedy(self.handle, first_tokens.data_ptr(), pos0, n_steps, B, C.byref(kc),
+                                                out.data_ptr(), logits.data_ptr(), _stream_ptr(stream))
+        self.lib.check(code, "pop_generate_greedy")
+        return out, logits
 
     def last_status(self, stream=None) -> int:
         return self.lib.dll.pop_last_status(self.handle, _stream_ptr(stream))

@@ -40,6 +40,8 @@ struct Workspace {
   float* partial;    // [B][n_q][64][hd+2]
   float2* rope1;     // [hd/2] rotary row of the one position a decode step works on
   int32_t* cu;       // [B+1] packed-row prefix sums of a ragged batch
+  int32_t* ctr;      // [2] device counters of the greedy loop: position, step
+  int32_t* tok;      // [B] current token of every sequence in the greedy loop
   size_t total;
 };
 
@@ -135,6 +137,8 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.partial = (float*)take((size_t)B * c.n_q_heads * 64 * (c.head_dim + 2) * 4);
   w.rope1 = (float2*)take((size_t)(c.head_dim / 2) * 8);
   w.cu = (int32_t*)take((size_t)(B + 1) * 4);
+  w.ctr = (int32_t*)take(2 * 4);
+  w.tok = (int32_t*)take((size_t)B * 4);
   w.total = o;
   return w;
 }
@@ -245,7 +249,8 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
 // Boundary token as a decode step of layer l (paper Sec. 3.3): one row per sequence in w.xb.
 // `table` holds rotary rows starting at position `table_pos0`.
 int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc,
-                   const float2* table, int table_pos0, cudaStream_t s, const int32_t* cu = nullptr) {
+                   const float2* table, int table_pos0, cudaStream_t s, const int32_t* cu = nullptr,
+                   const int32_t* pos_dev = nullptr) {
   const pop_config_t& c = m->cfg;
   const int d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -263,7 +268,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   r.table = table; r.table_pos0 = table_pos0; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
   r.rows = B; r.rows_per_seq = 1; r.rows_written = 1; r.pos0 = N - 1; r.groups = 1; r.eps = c.rms_eps;
-  r.cu_seqlens = cu; r.batch = B;
+  r.cu_seqlens = cu; r.batch = B; r.pos_dev = pos_dev;
   POP_TRY(launch_rope_cache(r, s));
   DecAttnArgs a{};
   a.q = w.qb; a.ldq = m->q_dim;
@@ -272,7 +277,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.block_table = kc->block_table; a.max_pages_per_seq = kc->max_pages_per_seq; a.page_size = kc->page_size;
   a.partial = w.partial; a.out = w.ob; a.ldo = m->q_dim;
   a.batch = B; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads; a.head_dim = c.head_dim; a.kv_len = N;
-  a.cu_seqlens = cu;
+  a.cu_seqlens = cu; a.pos_dev = pos_dev;
   a.window = layer_window(c, l);
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};
@@ -438,6 +443,24 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
   return POP_OK;
 }
 
+// The kernels of one decode step. The position comes from the host (`pos`) or, when `pos_dev` is
+// given, from device memory at run time.
+int decode_body(pop_model* m, const Workspace& w, const int32_t* tokens, int pos, const int32_t* pos_dev, int B,
+                pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
+  const pop_config_t& c = m->cfg;
+  const int d = c.d_model;
+  POP_TRY(launch_rope_table(w.rope1, 1, c.head_dim, c.rope_theta, s, pos, pos_dev));
+  POP_TRY(launch_embed(tokens, (const bf16*)(m->arena + m->off_embed), nullptr, w.xb, B, d, c.vocab, s));
+  for (int l = 1; l <= c.n_layers; ++l)
+    POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s, nullptr, pos_dev));
+  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
+                         true, s));
+  GemvArgs v{};
+  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
+  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
+  return launch_gemv(v, s);
+}
+
 // One decode step of the full model (paper Sec. 2.2): every sequence's token at position `pos`
 // (= entries already in the cache) goes through all L layers as the boundary token does.
 int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache_t* kc, float* logits,
@@ -452,18 +475,52 @@ int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache
   const Workspace w = carve(m, (char*)m->ws, 1, B);
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
   const int64_t launches0 = launch_count();
-  const int d = c.d_model;
-  POP_TRY(launch_rope_table(w.rope1, 1, c.head_dim, c.rope_theta, s, pos));
-  POP_TRY(launch_embed(tokens, (const bf16*)(m->arena + m->off_embed), nullptr, w.xb, B, d, c.vocab, s));
-  for (int l = 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s));
-  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
-                         true, s));
-  GemvArgs v{};
-  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
-  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
-  POP_TRY(launch_gemv(v, s));
+  POP_TRY(decode_body(m, w, tokens, pos, nullptr, B, kc, logits, s));
   m->last_launches = launch_count() - launches0;
   return POP_OK;
+}
+
+// Greedy generation on the device: the decode step and the arg-max that feeds the next one are
+// captured once into a CUDA graph whose kernels read the position from device memory, and the graph
+// is replayed n_steps times on the caller's stream.
+int run_generate(pop_model* m, const int32_t* first_tokens, int pos0, int n_steps, int B, pop_kv_cache_t* kc,
+                 int32_t* tokens_out, float* logits, cudaStream_t s) {
+  if (!m || !first_tokens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !tokens_out || !logits)
+    return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (pos0 < 0 || B < 1 || n_steps < 1 || (int64_t)pos0 + n_steps > (1 << 24)) return POP_E_INVALID;
+  if (prof_enabled()) return POP_E_INVALID;            // per-launch events cannot be recorded into a graph
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(pos0 + n_steps, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, 1, B);
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  const int64_t launches0 = launch_count();
+  if (cudaMemcpyAsync(w.tok, first_tokens, (size_t)B * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return POP_E_CUDA;
+  POP_TRY(launch_set_counters(w.ctr, pos0, 0, s));
+  // capture one step on a stream of the library's own
+  cudaStream_t cs = nullptr;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  if (cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) != cudaSuccess) return POP_E_CUDA;
+  int rc = POP_OK;
+  if (cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal) != cudaSuccess) rc = POP_E_CUDA;
+  if (rc == POP_OK) {
+    rc = decode_body(m, w, w.tok, 0, w.ctr, B, kc, logits, cs);
+    if (rc == POP_OK) rc = launch_argmax(logits, c.vocab, c.vocab, B, w.tok, tokens_out, n_steps, w.ctr + 1, cs);
+    if (rc == POP_OK) rc = launch_bump_counters(w.ctr, cs);
+    if (cudaStreamEndCapture(cs, &graph) != cudaSuccess || graph == nullptr) rc = rc == POP_OK ? POP_E_CUDA : rc;
+  }
+  if (rc == POP_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = POP_E_CUDA;
+  for (int i = 0; i < n_steps && rc == POP_OK; ++i)
+    if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = POP_E_CUDA;
+  // an executable graph in flight is released when its last launch has completed
+  if (exec) cudaGraphExecDestroy(exec);
+  if (graph) cudaGraphDestroy(graph);
+  cudaStreamDestroy(cs);
+  cudaGetLastError();
+  m->last_launches = launch_count() - launches0;
+  return rc;
 }
 
 struct NameRef { int layer; std::string t; };
@@ -639,6 +696,12 @@ int pop_prefill_skip(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int
 int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,
                     float* logits_out, void* stream) {
   return run_decode(m, tokens, pos, batch, kv_cache, logits_out, static_cast<cudaStream_t>(stream));
+}
+
+int pop_generate_greedy(pop_model_t* m, const int32_t* first_tokens, int32_t pos0, int32_t n_steps, int32_t batch,
+                        pop_kv_cache_t* kv_cache, int32_t* tokens_out, float* logits_scratch, void* stream) {
+  return run_generate(m, first_tokens, pos0, n_steps, batch, kv_cache, tokens_out, logits_scratch,
+                      static_cast<cudaStream_t>(stream));
 }
 
 int pop_last_status(pop_model_t* m, void* stream) {

@@ -116,7 +116,8 @@ int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, cons
                         float eps, cudaStream_t s);
 // table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)), pos < n_pos, j < hd/2
 // rows for positions first_pos .. first_pos + n_pos - 1
-int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos = 0);
+int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos = 0,
+                      const int32_t* first_pos_dev = nullptr);   // device value overrides first_pos when given
 struct RopeArgs {
   const float* in; int64_t ld_in; int64_t in_group_stride;   // fp32 rows [q heads | k heads | v heads] * hd
   bf16* q_out; int64_t ldq;                                  // may be null when n_q == 0
@@ -133,10 +134,19 @@ struct RopeArgs {
   // written. In launch_rope_cache it is only used for boundary rows (rows == batch): row b sits at
   // position cu[b+1] - cu[b] - 1.
   const int32_t* cu_seqlens; int batch; int skip_last;
+  // boundary / decode rows only: the position is read from device memory at run time (a step that is
+  // replayed from a captured graph with an advancing position); the table then holds that one row
+  const int32_t* pos_dev;
 };
 int launch_rope_cache(const RopeArgs& a, cudaStream_t s);
 int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s);
 // dst[b][:] = src[cu[b+1] - 1][:]: the last row of every packed sequence
+// tok[b] = index of the largest logit of row b (lowest index among equals), also stored at out[b * out_ld + *step]
+int launch_argmax(const float* logits, int64_t ld, int vocab, int batch, int32_t* tok, int32_t* out, int out_ld,
+                  const int32_t* step, cudaStream_t s);
+// counters[0] = a, counters[1] = b; and counters[0] += 1, counters[1] += 1
+int launch_set_counters(int32_t* counters, int a, int b, cudaStream_t s);
+int launch_bump_counters(int32_t* counters, cudaStream_t s);
 int launch_gather_last_rows(const float* src, float* dst, int batch, int d, const int32_t* cu, cudaStream_t s);
 
 // ------------------------------------------------------------------------------------ boundary path
@@ -155,6 +165,7 @@ struct DecAttnArgs {
   bf16* out; int64_t ldo;
   int batch, n_q, n_kv, head_dim, kv_len, window;
   const int32_t* cu_seqlens;   // ragged: sequence b has cu[b+1] - cu[b] cache positions (kv_len = their maximum)
+  const int32_t* pos_dev;      // run-time cache length - 1 (see RopeArgs::pos_dev); the split count is then fixed at 64
 };
 int decode_attn_splits(int kv_len, int window);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

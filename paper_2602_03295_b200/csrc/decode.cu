@@ -166,6 +166,7 @@ struct DecAttnDev {
   int n_q, n_kv, kv_len, window, splits;
   float scale_log2;
   const int32_t* cu;                       // ragged: sequence b has cu[b+1] - cu[b] cache positions
+  const int32_t* pos_dev;                  // run-time cache length - 1
 };
 
 constexpr int DEC_MAXG = 8;
@@ -187,7 +188,7 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane / LPK;                          // which key of the pass this lane group reads
   const int e0 = (lane % LPK) * 8;                     // first head_dim element of this lane
-  const int kv_len = p.cu ? p.cu[b + 1] - p.cu[b] : p.kv_len;
+  const int kv_len = p.pos_dev ? *p.pos_dev + 1 : (p.cu ? p.cu[b + 1] - p.cu[b] : p.kv_len);
   const int lo = p.window > 0 ? max(0, kv_len - p.window) : 0;
   const int span = kv_len - lo;
   const int chunk = (span + p.splits - 1) / p.splits;
@@ -405,7 +406,8 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.partial = a.partial; p.out = a.out; p.ldo = a.ldo;
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.kv_len = a.kv_len; p.window = a.window;
   p.cu = a.cu_seqlens;
-  p.splits = decode_attn_splits(a.kv_len, a.window);
+  p.pos_dev = a.pos_dev;
+  p.splits = a.pos_dev ? 64 : decode_attn_splits(a.kv_len, a.window);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)a.head_dim);
   dim3 grid(a.n_kv, p.splits, a.batch), grid2(a.n_q, a.batch);
   const int span = (a.window > 0 && a.window < a.kv_len) ? a.window : a.kv_len;
@@ -493,6 +495,7 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.out = static_cast<bf16*>(out); p.ldo = ldo;
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
   p.cu = nullptr;
+  p.pos_dev = nullptr;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // The first kernel writes every partial slot the second one reads (all splits of all heads, also

@@ -113,7 +113,9 @@ __global__ void postnorm_add_kernel(float* __restrict__ x, int64_t ldx, const fl
 
 // ------------------------------------------------------------------------------ rotary table
 // table[pos][j] = (cos, sin)(pos * theta^(-2j/hd)), evaluated in fp64, stored fp32.
-__global__ void rope_table_kernel(float2* __restrict__ table, int n_pos, int half, double theta, int first_pos) {
+__global__ void rope_table_kernel(float2* __restrict__ table, int n_pos, int half, double theta, int first_pos,
+                                  const int32_t* __restrict__ first_pos_dev) {
+  if (first_pos_dev != nullptr) first_pos = *first_pos_dev;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pos * half) return;
   const int pos = i / half, j = i - pos * half;
@@ -140,6 +142,7 @@ struct RopeDev {
   int rows, rows_per_seq, rows_written, pos0;
   float eps;
   const int32_t* cu;      // boundary rows of a ragged batch: row b sits at position cu[b+1] - cu[b] - 1
+  const int32_t* pos_dev; // run-time position of all rows; table row 0 is that position
 };
 
 template <int HD>
@@ -156,7 +159,8 @@ __global__ void rope_cache_kernel(const RopeDev p) {
   const int b = row / p.rows_per_seq;
   const int i = row - b * p.rows_per_seq;
   if (i >= p.rows_written) return;
-  const int pos = p.cu ? p.cu[b + 1] - p.cu[b] - 1 : p.pos0 + i;
+  const int pos = p.pos_dev ? *p.pos_dev : (p.cu ? p.cu[b + 1] - p.cu[b] - 1 : p.pos0 + i);
+  const int table_row = p.pos_dev ? 0 : pos - p.table_pos0;
   const float* src = p.in + (int64_t)g * p.in_group_stride + (int64_t)row * p.ld_in + (int64_t)h * HD;
   float lo[PER], hi[PER];                 // elements j and j + HD/2, j = lane + 32*u
 #pragma unroll
@@ -183,7 +187,7 @@ __global__ void rope_cache_kernel(const RopeDev p) {
     }
 #pragma unroll
     for (int u = 0; u < PER; ++u) {
-      const float2 cs = p.table[(int64_t)(pos - p.table_pos0) * (HD / 2) + lane + 32 * u];
+      const float2 cs = p.table[(int64_t)table_row * (HD / 2) + lane + 32 * u];
       const float a = lo[u] * cs.x - hi[u] * cs.y;
       const float c = hi[u] * cs.x + lo[u] * cs.y;
       lo[u] = a;
@@ -225,6 +229,44 @@ __global__ void gather_last_rows_kernel(const float* __restrict__ src, float* __
     *reinterpret_cast<float4*>(o + c) = *reinterpret_cast<const float4*>(s + c);
 }
 
+// greedy choice: index of the largest logit of a row, the lowest index among equal values
+__global__ void argmax_kernel(const float* __restrict__ logits, int64_t ld, int vocab, int32_t* __restrict__ tok,
+                              int32_t* __restrict__ out, int out_ld, const int32_t* __restrict__ step) {
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  const float* row = logits + (int64_t)blockIdx.x * ld;
+  float best = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+    const float v = row[i];
+    if (v > best || (v == best && i < idx)) { best = v; idx = i; }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = idx; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int nw = blockDim.x >> 5;
+    best = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+    idx = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+    }
+    if (threadIdx.x == 0) {
+      if (idx == 0x7fffffff) idx = 0;          // a row without any finite value
+      tok[blockIdx.x] = idx;
+      if (out != nullptr) out[(int64_t)blockIdx.x * out_ld + (step ? *step : 0)] = idx;
+    }
+  }
+}
+__global__ void set_counters_kernel(int32_t* c, int a, int b) { c[0] = a; c[1] = b; }
+__global__ void bump_counters_kernel(int32_t* c) { c[0] += 1; c[1] += 1; }
+
 }  // namespace
 
 int launch_embed(const int32_t* tokens, const bf16* table, const bf16* embeds, float* x, int rows, int d, int vocab,
@@ -259,9 +301,10 @@ int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, cons
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
 
-int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos) {
+int launch_rope_table(float2* table, int n_pos, int hd, float theta, cudaStream_t s, int first_pos,
+                      const int32_t* first_pos_dev) {
   const int total = n_pos * (hd / 2);
-  rope_table_kernel<<<ceil_div(total, 256), 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, first_pos);
+  rope_table_kernel<<<ceil_div(total, 256), 256, 0, s>>>(table, n_pos, hd / 2, (double)theta, first_pos, first_pos_dev);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -279,7 +322,8 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   p.rows = a.rows; p.rows_per_seq = a.rows_per_seq; p.rows_written = a.rows_written; p.pos0 = a.pos0;
   p.eps = a.eps;
   p.cu = a.cu_seqlens;
-  if (a.cu_seqlens != nullptr && a.rows_per_seq != 1) return POP_E_INVALID;
+  p.pos_dev = a.pos_dev;
+  if ((a.cu_seqlens != nullptr || a.pos_dev != nullptr) && a.rows_per_seq != 1) return POP_E_INVALID;
   const int heads = a.n_q + 2 * a.n_kv;
   const int64_t items = (int64_t)a.rows * heads;
   dim3 grid((unsigned)((items + 7) / 8), a.groups);
@@ -296,6 +340,23 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
 
 int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s) {
   gather_rows_kernel<<<batch, 256, 0, s>>>(src, dst, d, rows_per_seq, row);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+int launch_argmax(const float* logits, int64_t ld, int vocab, int batch, int32_t* tok, int32_t* out, int out_ld,
+                  const int32_t* step, cudaStream_t s) {
+  argmax_kernel<<<batch, 1024, 0, s>>>(logits, ld, vocab, tok, out, out_ld, step);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+int launch_set_counters(int32_t* counters, int a, int b, cudaStream_t s) {
+  set_counters_kernel<<<1, 1, 0, s>>>(counters, a, b);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+int launch_bump_counters(int32_t* counters, cudaStream_t s) {
+  bump_counters_kernel<<<1, 1, 0, s>>>(counters);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

@@ -87,3 +87,39 @@ def test_decode_step_rejects_a_full_cache():
     assert e.value.code == POP_E_INVALID
     torch.cuda.synchronize()
     assert (logits == 9.0).all()
+
+
+@pytest.mark.parametrize("variant", ["c1", "gemma", "hd256"])
+def test_graph_replayed_greedy_loop_follows_the_step_by_step_path(variant):
+    # pop_generate_greedy (one captured step replayed with a device-side position) against the same
+    # steps issued one by one with the arg-max taken on the host: every generated token must be the
+    # arg-max of the step-by-step logits for the same history (or tie with it to rounding), and the
+    # caches must agree
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS[variant]
+    B, N, T, l_keep = 3, 40, 7, 2
+    tokens = ps.uniform_tokens(77, B, N, cfg.vocab)
+    model = build(cfg)
+    ca = KVCache(cfg, B, N + T + 1, 16)
+    cb = KVCache(cfg, B, N + T + 1, 16)
+    la = model.prefill(tokens.to(DEV), None, l_keep, ca)
+    lb = model.prefill(tokens.to(DEV), None, l_keep, cb)
+    first = la.argmax(-1).to(torch.int32)
+    gen, last_logits = model.generate_greedy(first, N, T, ca)
+    assert model.last_status() == 0
+    gen = gen.cpu()
+    assert (gen >= 0).all() and (gen < cfg.vocab).all()
+    tok = first
+    for i in range(T):
+        lg = model.decode_step(tok.contiguous(), N + i, cb)
+        choice = gen[:, i].to(DEV).long()
+        picked = lg.gather(1, choice[:, None])[:, 0]
+        assert (lg.max(-1).values - picked).max().item() <= 1e-2      # the graph's token is (or ties with) the arg-max
+        tok = gen[:, i].to(DEV)
+    # (the graph path always merges 64 key splits, the step path as many as the length asks for: the
+    # attention outputs differ by bf16 roundings)
+    assert (last_logits - lg).abs().max().item() <= 1e-2
+    for l in range(cfg.n_layers):
+        ka, va = ca.gather(l, N + T)
+        kb, vb = cb.gather(l, N + T)
+        assert rel_err(ka, kb) <= 1e-2 and rel_err(va, vb) <= 1e-2
