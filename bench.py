@@ -338,6 +338,15 @@ def run_ours(a, wl):
     barrier()
     dec_ms = max_over_ranks(d0.elapsed_time(d1), dev) / DECODE_STEPS
     dec_status = model.last_status()
+    # the same steps as an on-device greedy loop: one captured step replayed per token
+    model.generate_greedy(dec_tok.to(torch.int32), wl.seq_len, 4, cache, logits)
+    barrier()
+    d0.record()
+    model.generate_greedy(dec_tok.to(torch.int32), wl.seq_len, DECODE_STEPS, cache, logits)
+    d1.record()
+    barrier()
+    gen_ms = max_over_ranks(d0.elapsed_time(d1), dev) / DECODE_STEPS
+    dec_status = dec_status or model.last_status()
     weight_bytes = 2.0 * (cfg.n_layers * po.layer_params(cfg) + cfg.vocab * cfg.d_model)
 
     # per-kernel-class durations of one more step, CUDA events on the launching stream
@@ -374,6 +383,8 @@ def run_ours(a, wl):
                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
            "decode": {"ms_per_step": dec_ms, "tokens_per_s": wl.batch * world / (dec_ms * 1e-3),
                       "context": wl.seq_len, "steps": DECODE_STEPS, "device_status": dec_status,
+                      "graph_loop_ms_per_step": gen_ms, "graph_loop_tokens_per_s": wl.batch * world / (gen_ms * 1e-3),
+                      "graph_loop_weight_stream_gbs": weight_bytes / (gen_ms * 1e-3) / 1e9,
                       "weight_stream_gbs": weight_bytes / (dec_ms * 1e-3) / 1e9,
                       "frac_of_measured_hbm": weight_bytes / (dec_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"]},
            "gpu_launches": int(launches * a.steps),
