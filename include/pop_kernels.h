@@ -97,7 +97,8 @@ int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t
                int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid, void* stream);
 
 /* Scratch floats pop_k_decode_attention needs: batch * n_q * 64 * (hd + 2). Single-query attention
- * of the boundary token (one query per sequence at position kv_len-1) over one cache layer. */
+ * of the boundary token (one query per sequence at position kv_len-1) over one cache layer.
+ * n_q / n_kv <= 8; head_dim 64, 128 or 256. */
 int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
                            const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
                            void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
@@ -113,9 +114,9 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
  * until the process ends. The call allocates and frees nothing, neither through CUDA nor any other
  * library. Arguments, layouts and results are those of pop_k_decode_attention minus `partial`.
  *  - Limit: batch * n_q * splits * (head_dim + 2) <= POP_STATIC_SCRATCH_FLOATS, where splits =
- *    ceil(span / 256) capped at 64 and span = min(kv_len, window or kv_len); a larger problem is
- *    refused with POP_E_NOSPACE and nothing is enqueued (e.g. 8 sequences x 32 heads x hd 128 at
- *    any length fit; 16 such sequences beyond 16128 positions do not).
+ *    min(64, SMs / (n_kv * batch), ceil(span / 64)), at least 1, and span = min(kv_len, window or
+ *    kv_len); a larger problem is refused with POP_E_NOSPACE and nothing is enqueued (e.g. 512
+ *    sequences x 32 heads x hd 128 fit at any length; 1024 such sequences do not).
  *  - The first call on each device looks up the array's device address (one runtime query with
  *    that device current, result kept); make that first call before starting any stream capture.
  *  - All calls share the one array, which keeps whatever the previous call left. Each call

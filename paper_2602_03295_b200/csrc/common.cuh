@@ -167,7 +167,7 @@ struct DecAttnArgs {
   const int32_t* cu_seqlens;   // ragged: sequence b has cu[b+1] - cu[b] cache positions (kv_len = their maximum)
   const int32_t* pos_dev;      // run-time cache length - 1 (see RopeArgs::pos_dev); the split count is then fixed at 64
 };
-int decode_attn_splits(int kv_len, int window);
+int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);
 
 }  // namespace pop

@@ -155,8 +155,15 @@ void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
 
 // ------------------------------------------------------------------------------ decode attention
 // One CTA per (kv head, split, sequence): the G = n_q/n_kv query heads of the group attend over a
-// contiguous chunk of cache positions; each warp walks positions, lanes split head_dim. Partials
-// (max, sum, unnormalised output) go to scratch and are merged by the combine kernel.
+// contiguous chunk of cache positions. The chunk is cut into groups of 16 keys that the four warps
+// take in turn. A warp streams the K and V rows of its groups into its own ring of shared-memory
+// stages with 16-byte asynchronous copies (several groups in flight), and computes on the warp-level
+// tensor-core path with the keys on the M side, so that no MMA row is padding:
+//     S^T [16 keys x 8 heads]  = K [16 x hd] . Q^T [hd x 8]            (hd/16 MMAs, Q^T kept in registers)
+//     O^T [hd x 8 heads]      += V^T [hd x 16 keys] . P^T [16 x 8]     (hd/16 MMAs)
+// P^T reaches the second product as bf16 (as it does in the prefill kernel), moved from the
+// accumulator layout to the B-operand layout by an 8x8 transpose across the warp. Heads G..7 are
+// zero columns. Partials (max, sum, unnormalised output) go to scratch and are merged by the combine kernel.
 struct DecAttnDev {
   const bf16* q; int64_t ldq;              // [B][n_q*hd], one query per sequence at position kv_len-1
   const bf16* k_pool; const bf16* v_pool;  // one layer: [page][slot][n_kv][hd]
@@ -169,142 +176,212 @@ struct DecAttnDev {
   const int32_t* pos_dev;                  // run-time cache length - 1
 };
 
-constexpr int DEC_MAXG = 8;
-constexpr int DEC_UNROLL = 4;     // keys per lane group whose K and V loads are in flight together
+constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of one MMA
 
 template <int HD>
 struct DecCfg {
-  static constexpr int LPK = HD / 8;                   // lanes per key: each lane holds 8 elements (16 bytes)
-  static constexpr int KPW = 32 / LPK;                 // keys per warp per pass
-  static constexpr int WARPS = (HD == 256) ? 4 : 8;
+  static constexpr int KT = 16;                        // keys per stage (the M extent of one MMA)
+  static constexpr int WARPS = 4;
+  static constexpr int ROWB = HD * 2;                  // bytes of one head's cache row
+  static constexpr int CH = ROWB / 16;                 // 16-byte chunks per row
+  static constexpr int STAGE = 2 * KT * ROWB;          // K rows, then V rows
+  static constexpr int NST = (HD == 256) ? 3 : 6;      // stages per warp
+  static constexpr int SMEM = WARPS * NST * STAGE;     // 192 KB at hd 128 and 256, 96 KB at hd 64
+  static_assert(WARPS * DEC_MAXG * (HD + 2) * 4 <= SMEM, "the merge of the warps reuses the ring");
 };
 
-template <int HD, int GMAX>
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  // src_bytes 0 writes 16 zero bytes and reads nothing
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// 8x8 transpose of 16-bit elements across the warp (thread i holds row i/4, columns 2(i%4), 2(i%4)+1)
+__device__ __forceinline__ uint32_t movm_t(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+// D[16x8] += A[16x16] . B[16x8], bf16 operands, fp32 accumulate
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int HD>
 __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const DecAttnDev p) {
   using C = DecCfg<HD>;
-  constexpr int LPK = C::LPK, KPW = C::KPW, WARPS = C::WARPS;
+  constexpr int KT = C::KT, WARPS = C::WARPS, ROWB = C::ROWB, CH = C::CH, NST = C::NST, NT = HD / 16;
+  constexpr uint32_t FULL = 0xffffffffu;
+  extern __shared__ __align__(128) uint8_t dec_smem[];
   const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
-  const int G = p.n_q / p.n_kv;   // <= GMAX
+  const int G = p.n_q / p.n_kv;   // <= DEC_MAXG
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sub = lane / LPK;                          // which key of the pass this lane group reads
-  const int e0 = (lane % LPK) * 8;                     // first head_dim element of this lane
   const int kv_len = p.pos_dev ? *p.pos_dev + 1 : (p.cu ? p.cu[b + 1] - p.cu[b] : p.kv_len);
   const int lo = p.window > 0 ? max(0, kv_len - p.window) : 0;
   const int span = kv_len - lo;
   const int chunk = (span + p.splits - 1) / p.splits;
   const int j0 = lo + split * chunk;
   const int j1 = min(kv_len, j0 + chunk);
+  // groups of KT keys; warp w takes groups w, w + WARPS, ...  (counts depend on the warp only)
+  const int n_groups = j1 > j0 ? (j1 - j0 + KT - 1) / KT : 0;
+  const int n_mine = n_groups > warp ? (n_groups - warp + WARPS - 1) / WARPS : 0;
 
-  float qv[GMAX][8];
+  // Q^T as the B operand: thread holds head lane/4, dims 16 ks + 2 (lane%4) + {0, 1} and + 8
+  uint32_t qb[NT][2];
+  {
+    const int g = lane >> 2;
+    const bf16* qrow = p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + (g < G ? g : 0)) * HD + (lane & 3) * 2;
 #pragma unroll
-  for (int g = 0; g < GMAX; ++g)
-    if (g < G) {
-      float t[8];
-      unpack8(*reinterpret_cast<const uint4*>(p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + g) * HD + e0), t);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) qv[g][e] = t[e] * p.scale_log2;
+    for (int ks = 0; ks < NT; ++ks) {
+      qb[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
+      qb[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
     }
-  float m[GMAX], l[GMAX], o[GMAX][8];
-#pragma unroll
-  for (int g = 0; g < GMAX; ++g) {
-    m[g] = -INFINITY;
-    l[g] = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
   }
+  // this thread's two heads are 2 (lane%4) and 2 (lane%4) + 1, its keys of a group lane/4 and lane/4 + 8
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  float o[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+
   const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
-  constexpr int STRIDE = WARPS * KPW;                  // keys the CTA covers per pass
-  // the trip count depends on the warp only, never on the lane: every lane reaches the shuffles
-  for (int jw = j0 + warp * KPW; jw < j1; jw += STRIDE * DEC_UNROLL) {
-    const int jb = jw + sub;
-    uint4 kraw[DEC_UNROLL], vraw[DEC_UNROLL];
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dec_smem) + warp * (NST * C::STAGE);
+
+  auto issue = [&](int it) {
+    const int jg = j0 + (warp + it * WARPS) * KT;
+    const uint32_t st = ring + (it % NST) * C::STAGE;
+    // lanes 0..15 (and again 16..31) each find the pool row of one key of the group; -1 past the chunk
+    const int jk = jg + (lane & 15);
+    int row = -1;
+    if (jk < j1) row = bt[jk / p.page_size] * p.page_size + jk % p.page_size;
 #pragma unroll
-    for (int u = 0; u < DEC_UNROLL; ++u) {
-      const int j = jb + u * STRIDE;
-      kraw[u] = make_uint4(0, 0, 0, 0);
-      vraw[u] = make_uint4(0, 0, 0, 0);
-      if (j < j1) {
-        const int page = bt[j / p.page_size];
-        const int64_t off = (((int64_t)page * p.page_size + j % p.page_size) * p.n_kv + kvh) * HD + e0;
-        kraw[u] = ld_stream(p.k_pool + off);
-        vraw[u] = ld_stream(p.v_pool + off);
+    for (int i = 0; i < KT * CH / 32; ++i) {
+      const int idx = i * 32 + lane;
+      const int key = idx / CH, ch = idx % CH;
+      const int r = __shfl_sync(FULL, row, key);
+      const int64_t off = r < 0 ? 0 : ((int64_t)r * p.n_kv + kvh) * HD + ch * 8;
+      const int nbytes = r < 0 ? 0 : 16;
+      // 16-byte chunks of a row are permuted by the key's low bits: the 8 rows one matrix load
+      // touches fall in different banks
+      const uint32_t dst = st + key * ROWB + ((ch ^ (key & 7)) << 4);
+      cp_async16(dst, p.k_pool + off, nbytes);
+      cp_async16(dst + KT * ROWB, p.v_pool + off, nbytes);
+    }
+  };
+
+#pragma unroll
+  for (int i = 0; i < NST; ++i) {
+    if (i < n_mine) issue(i);
+    cp_async_commit();
+  }
+  // matrix-load addresses of this lane (lane = 8 * matrix + row of the matrix)
+  const int mi = lane >> 3, r8 = lane & 7;
+  const uint32_t k_lane = ((mi & 1) * 8 + r8) * ROWB;          // K: matrices (keys 0-7 | 8-15) x (chunk 2ks | 2ks+1)
+  const uint32_t v_lane = KT * ROWB + ((mi >> 1) * 8 + r8) * ROWB;   // V: matrices (chunk 2t | 2t+1) x (keys 0-7 | 8-15)
+  const int kr = lane >> 2;
+
+  for (int it = 0; it < n_mine; ++it) {
+    cp_async_wait<NST - 1>();
+    __syncwarp();
+    const uint32_t st = ring + (it % NST) * C::STAGE;
+    const int jg = j0 + (warp + it * WARPS) * KT;
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < NT; ++ks) {
+      uint32_t a[4];
+      ldsm_x4(a, st + k_lane + (((2 * ks + (mi >> 1)) ^ r8) << 4));
+      mma_16816(s, a, qb[ks][0], qb[ks][1]);
+    }
+    const bool v0 = jg + kr < j1, v1 = jg + kr + 8 < j1;   // keys past the chunk contribute nothing
+    const float s0 = v0 ? s[0] * p.scale_log2 : -INFINITY, s1 = v0 ? s[1] * p.scale_log2 : -INFINITY;
+    const float s2 = v1 ? s[2] * p.scale_log2 : -INFINITY, s3 = v1 ? s[3] * p.scale_log2 : -INFINITY;
+    float x0 = fmaxf(s0, s2), x1 = fmaxf(s1, s3);
+#pragma unroll
+    for (int w = 4; w < 32; w <<= 1) {
+      x0 = fmaxf(x0, __shfl_xor_sync(FULL, x0, w));
+      x1 = fmaxf(x1, __shfl_xor_sync(FULL, x1, w));
+    }
+    // the first key of a group is always inside the chunk, so the new maxima are finite
+    const float n0 = fmaxf(m0, x0), n1 = fmaxf(m1, x1);
+    const float f0 = exp2f(m0 - n0), f1 = exp2f(m1 - n1);   // exp2f(-inf) = 0 on the first group
+    const float p0 = exp2f(s0 - n0), p1 = exp2f(s1 - n1), p2 = exp2f(s2 - n0), p3 = exp2f(s3 - n1);
+    l0 = l0 * f0 + (p0 + p2);
+    l1 = l1 * f1 + (p1 + p3);
+    m0 = n0;
+    m1 = n1;
+    if (__any_sync(FULL, f0 != 1.f || f1 != 1.f)) {
+#pragma unroll
+      for (int t = 0; t < NT; ++t) {
+        o[t][0] *= f0; o[t][1] *= f1; o[t][2] *= f0; o[t][3] *= f1;
       }
     }
+    const uint32_t pb0 = movm_t(pack_bf16x2(p0, p1));   // keys 0-7 of the group
+    const uint32_t pb1 = movm_t(pack_bf16x2(p2, p3));   // keys 8-15
 #pragma unroll
-    for (int u = 0; u < DEC_UNROLL; ++u) {
-      const bool valid = jb + u * STRIDE < j1;   // uniform within a lane group
-      {
-        float kf[8], vf[8];
-        unpack8(kraw[u], kf);
-        unpack8(vraw[u], vf);
+    for (int t = 0; t < NT; ++t) {
+      uint32_t a[4];
+      ldsm_x4_t(a, st + v_lane + (((2 * t + (mi & 1)) ^ r8) << 4));
+      mma_16816(o[t], a, pb0, pb1);
+    }
+    __syncwarp();                                         // every lane is done with the stage
+    if (it + NST < n_mine) issue(it + NST);
+    cp_async_commit();
+  }
+  cp_async_wait<0>();
 #pragma unroll
-        for (int g = 0; g < GMAX; ++g)
-          if (g < G) {
-            float sc = 0.f;
+  for (int w = 4; w < 32; w <<= 1) {
+    l0 += __shfl_xor_sync(FULL, l0, w);
+    l1 += __shfl_xor_sync(FULL, l1, w);
+  }
+  __syncthreads();                                        // all rings are idle: reuse them for the merge
+  float* sm_m = reinterpret_cast<float*>(dec_smem);       // [WARPS][8]
+  float* sm_l = sm_m + WARPS * DEC_MAXG;                  // [WARPS][8]
+  float* sm_o = sm_l + WARPS * DEC_MAXG;                  // [WARPS][8][HD]
+  {
+    const int h0 = (lane & 3) * 2;
+    if (lane < 4) {
+      sm_m[warp * DEC_MAXG + h0] = m0; sm_m[warp * DEC_MAXG + h0 + 1] = m1;
+      sm_l[warp * DEC_MAXG + h0] = l0; sm_l[warp * DEC_MAXG + h0 + 1] = l1;
+    }
+    float* so = sm_o + (warp * DEC_MAXG + h0) * HD;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sc = fmaf(qv[g][e], kf[e], sc);
-#pragma unroll
-            for (int w = LPK / 2; w > 0; w >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, w);
-            if (!valid) sc = -INFINITY;            // a key past the chunk contributes nothing
-            const float mn = fmaxf(m[g], sc);
-            if (mn == -INFINITY) continue;         // nothing seen yet by this lane group
-            const float f = exp2f(m[g] - mn);      // exp2f(-inf) = 0 on the first key
-            const float pj = exp2f(sc - mn);
-            // the probability meets V as bf16, as it does in the prefill kernel's P.V product
-            const float pr = __bfloat162float(__float2bfloat16_rn(pj));
-            l[g] = l[g] * f + pj;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pr, vf[e], o[g][e] * f);
-            m[g] = mn;
-          }
-      }
+    for (int t = 0; t < NT; ++t) {
+      so[t * 16 + kr] = o[t][0];
+      so[HD + t * 16 + kr] = o[t][1];
+      so[t * 16 + kr + 8] = o[t][2];
+      so[HD + t * 16 + kr + 8] = o[t][3];
     }
   }
-  __syncwarp();
-  // merge the lane groups of a warp (they walked different keys), then the warps through shared memory
-#pragma unroll
-  for (int g = 0; g < GMAX; ++g)
-    if (g < G) {
-#pragma unroll
-      for (int w = LPK; w < 32; w <<= 1) {
-        const float mo = __shfl_xor_sync(0xffffffffu, m[g], w);
-        const float lo2 = __shfl_xor_sync(0xffffffffu, l[g], w);
-        const float mn = fmaxf(m[g], mo);
-        const float fa = (m[g] == -INFINITY) ? 0.f : exp2f(m[g] - mn);
-        const float fb = (mo == -INFINITY) ? 0.f : exp2f(mo - mn);
-        l[g] = l[g] * fa + lo2 * fb;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float oo = __shfl_xor_sync(0xffffffffu, o[g][e], w);
-          o[g][e] = o[g][e] * fa + oo * fb;
-        }
-        m[g] = mn;
-      }
-    }
-  __shared__ float sm_m[WARPS][GMAX], sm_l[WARPS][GMAX];
-  __shared__ float sm_o[WARPS][GMAX][HD];
-#pragma unroll
-  for (int g = 0; g < GMAX; ++g)
-    if (g < G) {
-      if (lane == 0) {
-        sm_m[warp][g] = m[g];
-        sm_l[warp][g] = l[g];
-      }
-      if (sub == 0) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) sm_o[warp][g][e0 + e] = o[g][e];
-      }
-    }
   __syncthreads();
   for (int idx = threadIdx.x; idx < G * HD; idx += blockDim.x) {
     const int g = idx / HD, e = idx - g * HD;
     float mm = -INFINITY;
-    for (int w = 0; w < WARPS; ++w) mm = fmaxf(mm, sm_m[w][g]);
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) mm = fmaxf(mm, sm_m[w * DEC_MAXG + g]);
     float ll = 0.f, oo = 0.f;
+#pragma unroll
     for (int w = 0; w < WARPS; ++w) {
-      const float f = (sm_m[w][g] == -INFINITY) ? 0.f : exp2f(sm_m[w][g] - mm);
-      ll += sm_l[w][g] * f;
-      oo += sm_o[w][g][e] * f;
+      const float mw = sm_m[w * DEC_MAXG + g];
+      const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - mm);
+      ll += sm_l[w * DEC_MAXG + g] * f;
+      oo += sm_o[(w * DEC_MAXG + g) * HD + e] * f;
     }
     float* dst = p.partial + (((int64_t)b * p.n_q + kvh * G + g) * p.splits + split) * (HD + 2);
     dst[2 + e] = oo;
@@ -316,12 +393,17 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
 }
 
 template <int HD>
-void launch_dec_attn(const DecAttnDev& p, dim3 grid, int G, cudaStream_t s) {
-  constexpr int T = DecCfg<HD>::WARPS * 32;
-  if (G <= 1) dec_attn_kernel<HD, 1><<<grid, T, 0, s>>>(p);
-  else if (G <= 2) dec_attn_kernel<HD, 2><<<grid, T, 0, s>>>(p);
-  else if (G <= 4) dec_attn_kernel<HD, 4><<<grid, T, 0, s>>>(p);
-  else dec_attn_kernel<HD, 8><<<grid, T, 0, s>>>(p);
+int launch_dec_attn(const DecAttnDev& p, dim3 grid, cudaStream_t s) {
+  using C = DecCfg<HD>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(dec_attn_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) !=
+        cudaSuccess)
+      return POP_E_CUDA;
+    configured = true;
+  }
+  dec_attn_kernel<HD><<<grid, C::WARPS * 32, C::SMEM, s>>>(p);
+  return POP_OK;
 }
 
 template <int HD>
@@ -390,10 +472,49 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
 
-int decode_attn_splits(int kv_len, int window) {
-  const int span = window > 0 && window < kv_len ? window : kv_len;
-  int s = ceil_div(span, 256);
-  return s < 1 ? 1 : (s > 64 ? 64 : s);
+// Split count: as many CTAs as the GPU has SMs (one CTA fills an SM's shared memory), never more
+// than 64 (the combine kernel's limit) nor so many that a CTA gets less than one 16-key group per
+// warp. kv_len < 1 means "not known on the host" (the length is read on the device).
+int decode_attn_splits(int kv_len, int window, int n_kv, int batch) {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+    sms = n;
+  }
+  int s = sms / (n_kv * batch > 0 ? n_kv * batch : 1);
+  if (s > 64) s = 64;
+  if (kv_len >= 1) {
+    const int span = window > 0 && window < kv_len ? window : kv_len;
+    const int by_len = ceil_div(span, 64);
+    if (s > by_len) s = by_len;
+  }
+  return s < 1 ? 1 : s;
+}
+
+template <int HD>
+int launch_dec_pair(const DecAttnDev& p, int batch, cudaStream_t s) {
+  dim3 grid(p.n_kv, p.splits, batch), grid2(p.n_q, batch);
+  const int rc = launch_dec_attn<HD>(p, grid, s);
+  if (rc != POP_OK) return rc;
+  dec_combine_kernel<HD><<<grid2, HD < 128 ? HD : 128, 0, s>>>(p);
+  count_launch();
+  count_launch();
+  return POP_OK;
+}
+
+int launch_dec_by_head_dim(const DecAttnDev& p, int head_dim, int batch, cudaStream_t s) {
+  int rc = POP_E_INVALID;
+  switch (head_dim) {
+    case 64: rc = launch_dec_pair<64>(p, batch, s); break;
+    case 128: rc = launch_dec_pair<128>(p, batch, s); break;
+    case 256: rc = launch_dec_pair<256>(p, batch, s); break;
+    default: return POP_E_INVALID;
+  }
+  if (rc != POP_OK) return rc;
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
 
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
@@ -407,29 +528,11 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.kv_len = a.kv_len; p.window = a.window;
   p.cu = a.cu_seqlens;
   p.pos_dev = a.pos_dev;
-  p.splits = a.pos_dev ? 64 : decode_attn_splits(a.kv_len, a.window);
+  p.splits = decode_attn_splits(a.pos_dev ? 0 : a.kv_len, a.window, a.n_kv, a.batch);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)a.head_dim);
-  dim3 grid(a.n_kv, p.splits, a.batch), grid2(a.n_q, a.batch);
   const int span = (a.window > 0 && a.window < a.kv_len) ? a.window : a.kv_len;
   ProfScope prof(PROF_DECODE_ATTN, (double)a.batch * span * a.n_kv * a.head_dim * 4, s);
-  switch (a.head_dim) {
-    case 64:
-      launch_dec_attn<64>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
-      break;
-    case 128:
-      launch_dec_attn<128>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
-      break;
-    case 256:
-      launch_dec_attn<256>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<256><<<grid2, 128, 0, s>>>(p);
-      break;
-    default: return POP_E_INVALID;
-  }
-  count_launch();
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+  return launch_dec_by_head_dim(p, a.head_dim, a.batch, s);
 }
 
 }  // namespace pop
@@ -481,7 +584,7 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   if (head_dim != 64 && head_dim != 128 && head_dim != 256) return POP_E_INVALID;
   if ((int64_t)ceil_div(kv_len, page_size) > max_pages_per_seq) return POP_E_NOSPACE;
   DecAttnDev p;
-  p.splits = decode_attn_splits(kv_len, window);
+  p.splits = decode_attn_splits(kv_len, window, n_kv, batch);
   // every (sequence, query head, split) owns head_dim + 2 floats of the shared array
   const int64_t need = (int64_t)batch * n_q * p.splits * (head_dim + 2);
   if (need > (int64_t)POP_STATIC_SCRATCH_FLOATS) return POP_E_NOSPACE;
@@ -501,22 +604,5 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   // The first kernel writes every partial slot the second one reads (all splits of all heads, also
   // the empty ones), so nothing left in the array by an earlier call is ever consumed and no
   // clearing is needed between calls.
-  dim3 grid(n_kv, p.splits, batch), grid2(n_q, batch);
-  switch (head_dim) {
-    case 64:
-      launch_dec_attn<64>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
-      break;
-    case 128:
-      launch_dec_attn<128>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
-      break;
-    default:
-      launch_dec_attn<256>(p, grid, p.n_q / p.n_kv, s);
-      dec_combine_kernel<256><<<grid2, 128, 0, s>>>(p);
-      break;
-  }
-  count_launch();
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+  return launch_dec_by_head_dim(p, head_dim, batch, s);
 }

@@ -116,8 +116,8 @@ def test_graph_replayed_greedy_loop_follows_the_step_by_step_path(variant):
         picked = lg.gather(1, choice[:, None])[:, 0]
         assert (lg.max(-1).values - picked).max().item() <= 1e-2      # the graph's token is (or ties with) the arg-max
         tok = gen[:, i].to(DEV)
-    # (the graph path always merges 64 key splits, the step path as many as the length asks for: the
-    # attention outputs differ by bf16 roundings)
+    # (the graph path cannot size its key splits by the length, the step path does: the attention
+    # outputs differ by bf16 roundings)
     assert (last_logits - lg).abs().max().item() <= 1e-2
     for l in range(cfg.n_layers):
         ka, va = ca.gather(l, N + T)

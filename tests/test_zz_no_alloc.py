@@ -58,9 +58,9 @@ def test_static_scratch_variant_refuses_what_does_not_fit():
     import paper_2602_03295_b200 as pk
     from paper_2602_03295_b200 import PopError, POP_E_NOSPACE, POP_E_INVALID
     L = pk.lib()
-    # 64 sequences x 32 heads x 64 splits x 130 floats = 17 M floats > the 4 Mi the library holds.
+    # 1024 sequences x 32 heads x 1 split x 130 floats = 4.26 M floats > the 4 Mi the library holds.
     # The size check comes before any launch, so the (tiny, unrelated) buffers are never read.
-    B, n_q, n_kv, hd, S = 64, 32, 8, 128, 16384
+    B, n_q, n_kv, hd, S = 1024, 32, 8, 128, 16384
     q = torch.zeros(B, n_q * hd, dtype=torch.bfloat16, device=DEV)
     pool = torch.zeros(1, 128, n_kv, hd, dtype=torch.bfloat16, device=DEV)
     bt = torch.zeros(B, S // 128, dtype=torch.int32, device=DEV)
