@@ -494,10 +494,13 @@ def run_kernel(a, wl):
         q = rnd(wl.batch, qd, std=1.0)
         out = torch.zeros(wl.batch, qd, dtype=torch.bfloat16, device=dev)
         work = per_set
+        # as the decode step calls it: zeroed arrival counters, so the kernel merges its own key splits
+        ctr = torch.zeros(wl.batch * cfg.n_kv_heads, dtype=torch.int32, device=dev)
+        part = torch.empty(wl.batch * cfg.n_q_heads * 64 * (hd + 2), dtype=torch.float32, device=dev)
 
         def launch(i):
             lib.decode_attention(q, cache.k[i % sets], cache.v[i % sets], cache.block_table, out, cfg.n_q_heads,
-                                 cfg.n_kv_heads, hd, N, a.page_size, 0)
+                                 cfg.n_kv_heads, hd, N, a.page_size, 0, counters=ctr, partial=part)
     elif k == "rmsnorm":
         bound = "hbm"
         x = rnd(M, d, dtype=torch.float32)

@@ -96,13 +96,17 @@ int pop_k_rope_cache(const float* in, int64_t ld_in, int64_t in_gs, void* q_out,
 int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t ldw, void* out, int64_t ldo,
                int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid, void* stream);
 
-/* Scratch floats pop_k_decode_attention needs: batch * n_q * 64 * (hd + 2). Single-query attention
- * of the boundary token (one query per sequence at position kv_len-1) over one cache layer.
- * n_q / n_kv <= 8; head_dim 64, 128 or 256. */
+/* Single-query attention of the boundary token (paper Sec. 3.3; one query per sequence at position
+ * kv_len-1) over one cache layer, split over the keys. n_q / n_kv <= 8; head_dim 64, 128 or 256.
+ * partial: device scratch of batch * n_q * 64 * (hd + 2) floats, contents irrelevant before and after.
+ * counters: optional device int32 [batch * n_kv]. If given they must all be zero when the call's
+ * kernels start and are all zero again when they end (so one zeroed array serves any number of
+ * calls on one stream); the attention kernel then merges its own splits and the call is a single
+ * launch. Null: a second kernel merges them. Both ways give the same bits. */
 int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
                            const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
-                           void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
-                           int32_t kv_len, int32_t window, void* stream);
+                           int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
+                           int32_t head_dim, int32_t kv_len, int32_t window, void* stream);
 
 /* The same single-query attention as pop_k_decode_attention for callers that have no way to hand
  * over a scratch buffer because they cannot allocate device memory at the point of the call: code

@@ -83,7 +83,7 @@ SIGNATURES = {
     "pop_k_rope_cache": (C.c_int, [_P, _I64, _I64, _P, _I64, _P, _P, _I64, _I32, _P, _I32, _I32, _P, _P, _I64, _P]
                          + [_I32] * 8 + [_F, _P]),
     "pop_k_gemv": (C.c_int, [_P, _I64, _I32, _P, _I64, _P, _I64] + [_I32] * 6 + [_P]),
-    "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _I64] + [_I32] * 6 + [_P]),
+    "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_decode_attention_static": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_profile": (None, [_I32]),
     "pop_k_profile_summary": (C.c_int, [_I32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_I64)]),
@@ -247,12 +247,16 @@ class PopLibrary:
         return out
 
     def decode_attention(self, q, k_pool, v_pool, block_table, out, n_q, n_kv, hd, kv_len, page_size, window=0,
-                         stream=None):
+                         stream=None, counters=None, partial=None):
+        """pop_k_decode_attention. `counters`: a zeroed int32 tensor of batch * n_kv entries (left zero by
+        the call) makes it a single launch; without, a second kernel merges the key splits."""
         batch = q.shape[0]
-        partial = torch.empty(batch * n_q * 64 * (hd + 2), dtype=torch.float32, device=q.device)
+        if partial is None:
+            partial = torch.empty(batch * n_q * 64 * (hd + 2), dtype=torch.float32, device=q.device)
         code = self.dll.pop_k_decode_attention(q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(),
                                                block_table.data_ptr(), block_table.shape[1], page_size,
-                                               partial.data_ptr(), out.data_ptr(), out.stride(0), batch, n_q, n_kv,
+                                               partial.data_ptr(), 0 if counters is None else counters.data_ptr(),
+                                               out.data_ptr(), out.stride(0), batch, n_q, n_kv,
                                                hd, kv_len, window, _stream_ptr(stream))
         self.check(code, "pop_k_decode_attention")
         return out

@@ -42,6 +42,7 @@ struct Workspace {
   int32_t* cu;       // [B+1] packed-row prefix sums of a ragged batch
   int32_t* ctr;      // [2] device counters of the greedy loop: position, step
   int32_t* tok;      // [B] current token of every sequence in the greedy loop
+  int32_t* dec_ctr;  // [B][n_kv] arrival counters of the decode attention's split merge (zero between launches)
   size_t total;
 };
 
@@ -139,6 +140,7 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.cu = (int32_t*)take((size_t)(B + 1) * 4);
   w.ctr = (int32_t*)take(2 * 4);
   w.tok = (int32_t*)take((size_t)B * 4);
+  w.dec_ctr = (int32_t*)take((size_t)B * c.n_kv_heads * 4);
   w.total = o;
   return w;
 }
@@ -277,7 +279,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.block_table = kc->block_table; a.max_pages_per_seq = kc->max_pages_per_seq; a.page_size = kc->page_size;
   a.partial = w.partial; a.out = w.ob; a.ldo = m->q_dim;
   a.batch = B; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads; a.head_dim = c.head_dim; a.kv_len = N;
-  a.cu_seqlens = cu; a.pos_dev = pos_dev;
+  a.cu_seqlens = cu; a.pos_dev = pos_dev; a.counters = w.dec_ctr;
   a.window = layer_window(c, l);
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};
@@ -321,6 +323,8 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
   if (!m->ws) return POP_E_NOSPACE;
   const Workspace w = carve(m, (char*)m->ws, N, B);
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  // the workspace is the caller's between calls: the split-merge counters start from zero in every call
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
   const int M = B * N, d = c.d_model;
 
@@ -372,6 +376,8 @@ int run_prefill_ragged(pop_model* m, const pop_input_t* in, const int32_t* seq_l
   if (!m->ws) return POP_E_NOSPACE;
   const Workspace w = carve(m, (char*)m->ws, N, B);        // laid out for B x N rows >= T
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  // the workspace is the caller's between calls: the split-merge counters start from zero in every call
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
   const int d = c.d_model;
   // the prefix sums travel through the stream like everything else (the host vector is pageable
@@ -420,6 +426,8 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
   if (!m->ws) return POP_E_NOSPACE;
   const Workspace w = carve(m, (char*)m->ws, N, B);
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  // the workspace is the caller's between calls: the split-merge counters start from zero in every call
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
   const int M = B * N, d = c.d_model;
   POP_TRY(launch_rope_table(w.rope, N, c.head_dim, c.rope_theta, s));
@@ -474,6 +482,8 @@ int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache
   if (!m->ws) return POP_E_NOSPACE;
   const Workspace w = carve(m, (char*)m->ws, 1, B);
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  // the workspace is the caller's between calls: the split-merge counters start from zero in every call
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
   POP_TRY(decode_body(m, w, tokens, pos, nullptr, B, kc, logits, s));
   m->last_launches = launch_count() - launches0;
@@ -495,6 +505,8 @@ int run_generate(pop_model* m, const int32_t* first_tokens, int pos0, int n_step
   if (!m->ws) return POP_E_NOSPACE;
   const Workspace w = carve(m, (char*)m->ws, 1, B);
   if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  // the workspace is the caller's between calls: the split-merge counters start from zero in every call
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
   if (cudaMemcpyAsync(w.tok, first_tokens, (size_t)B * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return POP_E_CUDA;
   POP_TRY(launch_set_counters(w.ctr, pos0, 0, s));

@@ -115,9 +115,10 @@ int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t
 
 int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
                            const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
-                           void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv, int32_t head_dim,
-                           int32_t kv_len, int32_t window, void* stream) {
+                           int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
+                           int32_t head_dim, int32_t kv_len, int32_t window, void* stream) {
   DecAttnArgs a{};
+  a.counters = counters;
   a.q = static_cast<const bf16*>(q); a.ldq = ldq;
   a.k_pool = static_cast<const bf16*>(k_pool); a.v_pool = static_cast<const bf16*>(v_pool);
   a.block_table = block_table; a.max_pages_per_seq = max_pages_per_seq; a.page_size = page_size;

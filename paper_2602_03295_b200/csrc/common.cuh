@@ -165,7 +165,10 @@ struct DecAttnArgs {
   bf16* out; int64_t ldo;
   int batch, n_q, n_kv, head_dim, kv_len, window;
   const int32_t* cu_seqlens;   // ragged: sequence b has cu[b+1] - cu[b] cache positions (kv_len = their maximum)
-  const int32_t* pos_dev;      // run-time cache length - 1 (see RopeArgs::pos_dev); the split count is then fixed at 64
+  const int32_t* pos_dev;      // run-time cache length - 1 (see RopeArgs::pos_dev)
+  // optional [batch][n_kv] int32, all zero before the call and all zero again after it: with it the
+  // attention kernel merges its own splits (one launch); without, a second kernel does
+  int32_t* counters;
 };
 int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

@@ -155,7 +155,7 @@ void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
 
 // ------------------------------------------------------------------------------ decode attention
 // One CTA per (kv head, split, sequence): the G = n_q/n_kv query heads of the group attend over a
-// contiguous chunk of cache positions. The chunk is cut into groups of 16 keys that the four warps
+// contiguous chunk of cache positions. The chunk is cut into groups of 16 keys that the warps
 // take in turn. A warp streams the K and V rows of its groups into its own ring of shared-memory
 // stages with 16-byte asynchronous copies (several groups in flight), and computes on the warp-level
 // tensor-core path with the keys on the M side, so that no MMA row is padding:
@@ -174,6 +174,9 @@ struct DecAttnDev {
   float scale_log2;
   const int32_t* cu;                       // ragged: sequence b has cu[b+1] - cu[b] cache positions
   const int32_t* pos_dev;                  // run-time cache length - 1
+  // [B][n_kv] arrival counters, zero before the launch and zero again after it: the last CTA of a
+  // (sequence, kv head) to finish merges the splits itself. Null: the combine kernel does it.
+  unsigned int* counters;
 };
 
 constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of one MMA
@@ -181,13 +184,14 @@ constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of on
 template <int HD>
 struct DecCfg {
   static constexpr int KT = 16;                        // keys per stage (the M extent of one MMA)
-  static constexpr int WARPS = 4;
+  static constexpr int WARPS = (HD == 256) ? 4 : 8;
   static constexpr int ROWB = HD * 2;                  // bytes of one head's cache row
   static constexpr int CH = ROWB / 16;                 // 16-byte chunks per row
   static constexpr int STAGE = 2 * KT * ROWB;          // K rows, then V rows
-  static constexpr int NST = (HD == 256) ? 3 : 6;      // stages per warp
-  static constexpr int SMEM = WARPS * NST * STAGE;     // 192 KB at hd 128 and 256, 96 KB at hd 64
-  static_assert(WARPS * DEC_MAXG * (HD + 2) * 4 <= SMEM, "the merge of the warps reuses the ring");
+  static constexpr int NST = (HD == 64) ? 6 : 3;       // stages per warp
+  static constexpr int SMEM = WARPS * NST * STAGE;     // 192 KB
+  static constexpr int MERGE_FLOATS = WARPS * DEC_MAXG * (HD + 2);
+  static_assert((MERGE_FLOATS + DEC_MAXG * 65) * 4 <= SMEM, "the merge of the warps reuses the ring");
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -223,6 +227,42 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Merge of the split partials of heads h_first .. h_first + n_heads - 1 of sequence b, by all
+// threads of the CTA (splits <= 64). Per head one warp computes the split weights exp2(m_s - max m)
+// (lane s handles splits s and s + 32), then every thread sums its output elements over the splits
+// with independent loads. Partials are read past L1: other CTAs of the same launch may have written them.
+template <int HD>
+__device__ __forceinline__ void dec_combine_heads(const DecAttnDev& p, int b, int h_first, int n_heads,
+                                                  float* wgt /* [n_heads][64] */, float* inv_l /* [n_heads] */) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  for (int g = warp; g < n_heads; g += n_warps) {
+    const float* src = p.partial + ((int64_t)b * p.n_q + h_first + g) * p.splits * (HD + 2);
+    const int s0 = lane, s1 = lane + 32;
+    const float m0 = s0 < p.splits ? __ldcg(src + s0 * (HD + 2)) : -INFINITY;
+    const float m1 = s1 < p.splits ? __ldcg(src + s1 * (HD + 2)) : -INFINITY;
+    const float l0 = s0 < p.splits ? __ldcg(src + s0 * (HD + 2) + 1) : 0.f;
+    const float l1 = s1 < p.splits ? __ldcg(src + s1 * (HD + 2) + 1) : 0.f;
+    float mm = fmaxf(m0, m1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+    const float w0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mm);
+    const float w1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
+    wgt[g * 64 + s0] = w0;
+    wgt[g * 64 + s1] = w1;
+    const float ll = warp_sum(l0 * w0 + l1 * w1);
+    if (lane == 0) inv_l[g] = 1.0f / ll;
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < n_heads * HD; idx += blockDim.x) {
+    const int g = idx / HD, e = idx - g * HD;
+    const float* src = p.partial + ((int64_t)b * p.n_q + h_first + g) * p.splits * (HD + 2) + 2 + e;
+    float oo = 0.f;
+#pragma unroll 8
+    for (int sp = 0; sp < p.splits; ++sp) oo = fmaf(__ldcg(src + sp * (HD + 2)), wgt[g * 64 + sp], oo);
+    p.out[(int64_t)b * p.ldo + (int64_t)(h_first + g) * HD + e] = __float2bfloat16_rn(oo * inv_l[g]);
+  }
 }
 
 template <int HD>
@@ -302,13 +342,17 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
     __syncwarp();
     const uint32_t st = ring + (it % NST) * C::STAGE;
     const int jg = j0 + (warp + it * WARPS) * KT;
-    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};   // two chains of dependent MMAs
 #pragma unroll
-    for (int ks = 0; ks < NT; ++ks) {
-      uint32_t a[4];
+    for (int ks = 0; ks < NT; ks += 2) {
+      uint32_t a[4], a2[4];
       ldsm_x4(a, st + k_lane + (((2 * ks + (mi >> 1)) ^ r8) << 4));
+      ldsm_x4(a2, st + k_lane + (((2 * ks + 2 + (mi >> 1)) ^ r8) << 4));
       mma_16816(s, a, qb[ks][0], qb[ks][1]);
+      mma_16816(sb, a2, qb[ks + 1][0], qb[ks + 1][1]);
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] += sb[i];
     const bool v0 = jg + kr < j1, v1 = jg + kr + 8 < j1;   // keys past the chunk contribute nothing
     const float s0 = v0 ? s[0] * p.scale_log2 : -INFINITY, s1 = v0 ? s[1] * p.scale_log2 : -INFINITY;
     const float s2 = v1 ? s[2] * p.scale_log2 : -INFINITY, s3 = v1 ? s[3] * p.scale_log2 : -INFINITY;
@@ -390,6 +434,20 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
       dst[1] = ll;
     }
   }
+  if (p.counters == nullptr) return;
+  // the last CTA of this (sequence, kv head) to get here merges the splits; the counter wraps back to 0
+  __shared__ int is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int old = atomicInc(p.counters + (int64_t)b * p.n_kv + kvh, (unsigned int)p.splits - 1u);
+    is_last = old == (unsigned int)p.splits - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  float* wgt = reinterpret_cast<float*>(dec_smem) + C::MERGE_FLOATS;
+  dec_combine_heads<HD>(p, b, kvh * G, G, wgt, wgt + DEC_MAXG * 64);
 }
 
 template <int HD>
@@ -408,36 +466,10 @@ int launch_dec_attn(const DecAttnDev& p, dim3 grid, cudaStream_t s) {
 
 template <int HD>
 __global__ void dec_combine_kernel(const DecAttnDev p) {
-  // one CTA per (head, sequence); splits <= 64. The split weights exp2(m_s - max m) are computed
-  // once (thread s handles split s), then every thread sums its output elements over the splits
-  // with independent loads.
+  // one CTA per (head, sequence)
   __shared__ float wgt[64];
   __shared__ float inv_l;
-  const int h = blockIdx.x, b = blockIdx.y;
-  const float* src = p.partial + ((int64_t)b * p.n_q + h) * p.splits * (HD + 2);
-  if (threadIdx.x < 32) {
-    const int s0 = threadIdx.x, s1 = threadIdx.x + 32;
-    const float m0 = s0 < p.splits ? src[s0 * (HD + 2)] : -INFINITY;
-    const float m1 = s1 < p.splits ? src[s1 * (HD + 2)] : -INFINITY;
-    const float l0 = s0 < p.splits ? src[s0 * (HD + 2) + 1] : 0.f;
-    const float l1 = s1 < p.splits ? src[s1 * (HD + 2) + 1] : 0.f;
-    float mm = fmaxf(m0, m1);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-    const float w0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mm);
-    const float w1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mm);
-    wgt[s0] = w0;
-    wgt[s1] = w1;
-    const float ll = warp_sum(l0 * w0 + l1 * w1);
-    if (threadIdx.x == 0) inv_l = 1.0f / ll;
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < HD; e += blockDim.x) {
-    float oo = 0.f;
-#pragma unroll 8
-    for (int s = 0; s < p.splits; ++s) oo = fmaf(src[s * (HD + 2) + 2 + e], wgt[s], oo);
-    p.out[(int64_t)b * p.ldo + (int64_t)h * HD + e] = __float2bfloat16_rn(oo * inv_l);
-  }
+  dec_combine_heads<HD>(p, blockIdx.y, blockIdx.x, 1, wgt, &inv_l);
 }
 
 }  // namespace
@@ -499,9 +531,11 @@ int launch_dec_pair(const DecAttnDev& p, int batch, cudaStream_t s) {
   dim3 grid(p.n_kv, p.splits, batch), grid2(p.n_q, batch);
   const int rc = launch_dec_attn<HD>(p, grid, s);
   if (rc != POP_OK) return rc;
-  dec_combine_kernel<HD><<<grid2, HD < 128 ? HD : 128, 0, s>>>(p);
   count_launch();
-  count_launch();
+  if (p.counters == nullptr) {
+    dec_combine_kernel<HD><<<grid2, HD < 128 ? HD : 128, 0, s>>>(p);
+    count_launch();
+  }
   return POP_OK;
 }
 
@@ -528,6 +562,7 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.kv_len = a.kv_len; p.window = a.window;
   p.cu = a.cu_seqlens;
   p.pos_dev = a.pos_dev;
+  p.counters = reinterpret_cast<unsigned int*>(a.counters);
   p.splits = decode_attn_splits(a.pos_dev ? 0 : a.kv_len, a.window, a.n_kv, a.batch);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)a.head_dim);
   const int span = (a.window > 0 && a.window < a.kv_len) ? a.window : a.kv_len;
@@ -545,27 +580,36 @@ namespace pop {
 namespace {
 
 static __device__ __align__(256) float g_dec_static_scratch[POP_STATIC_SCRATCH_FLOATS];
+// arrival counters of the split merge, one per (sequence, kv head): zero when the module is loaded,
+// and every launch leaves them at zero again
+constexpr int kStaticCounters = 4096;
+static __device__ unsigned int g_dec_static_counters[kStaticCounters];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mu;
 float* g_static_ptr[kMaxDevices] = {};
+unsigned int* g_static_ctr[kMaxDevices] = {};
 
 // Device address of the scratch array on the current device. In host code the array's name is only
 // a handle for the runtime, not something a kernel can dereference, so the address is looked up
 // once per device (with that device current) and remembered.
-int static_scratch(float** out) {
+int static_scratch(float** out, unsigned int** counters) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return POP_E_CUDA;
   std::lock_guard<std::mutex> lk(g_static_mu);
   if (g_static_ptr[dev] == nullptr) {
     float* ptr = nullptr;
-    if (cudaGetSymbolAddress((void**)&ptr, g_dec_static_scratch) != cudaSuccess || ptr == nullptr) {
+    unsigned int* ctr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_dec_static_scratch) != cudaSuccess || ptr == nullptr ||
+        cudaGetSymbolAddress((void**)&ctr, g_dec_static_counters) != cudaSuccess || ctr == nullptr) {
       cudaGetLastError();
       return POP_E_CUDA;
     }
     g_static_ptr[dev] = ptr;
+    g_static_ctr[dev] = ctr;
   }
   *out = g_static_ptr[dev];
+  *counters = g_static_ctr[dev];
   return POP_OK;
 }
 
@@ -589,7 +633,8 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   const int64_t need = (int64_t)batch * n_q * p.splits * (head_dim + 2);
   if (need > (int64_t)POP_STATIC_SCRATCH_FLOATS) return POP_E_NOSPACE;
   float* scratch = nullptr;
-  const int rc = static_scratch(&scratch);
+  unsigned int* counters = nullptr;
+  const int rc = static_scratch(&scratch, &counters);
   if (rc != POP_OK) return rc;
   p.q = static_cast<const bf16*>(q); p.ldq = ldq;
   p.k_pool = static_cast<const bf16*>(k_pool); p.v_pool = static_cast<const bf16*>(v_pool);
@@ -599,10 +644,12 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
   p.cu = nullptr;
   p.pos_dev = nullptr;
+  // with a counter per (sequence, kv head) the attention kernel merges its own splits
+  p.counters = (int64_t)batch * n_kv <= kStaticCounters ? counters : nullptr;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // The first kernel writes every partial slot the second one reads (all splits of all heads, also
-  // the empty ones), so nothing left in the array by an earlier call is ever consumed and no
-  // clearing is needed between calls.
+  // Every partial slot that the merge reads is written first by this call's own CTAs (all splits of
+  // all heads, also the empty ones), so nothing left in the array by an earlier call is ever
+  // consumed and no clearing is needed between calls.
   return launch_dec_by_head_dim(p, head_dim, batch, s);
 }

@@ -291,6 +291,15 @@ def test_decode_attention(L, B, S, n_q, n_kv, hd, page, window):
                                     torch.tensor([S - 1]), window).reshape(-1) for b in range(B)])
     assert not torch.isnan(out).any()
     assert rel_err(out, ref) < 1e-2
+    # with arrival counters the attention kernel merges its own splits: same bits, counters left at zero,
+    # so the same array serves the next call
+    ctr = torch.zeros(B * n_kv, dtype=torch.int32, device=DEV)
+    for _ in range(2):
+        out2 = torch.full_like(out, float("nan"))
+        L.decode_attention(q.to(DEV), kp.to(DEV), vp.to(DEV), bt.to(DEV), out2, n_q, n_kv, hd, S, page, window,
+                           counters=ctr)
+        assert torch.equal(out2, out)
+        assert (ctr == 0).all()
 
 
 def test_generators_agree_between_cpu_and_gpu():
