@@ -69,15 +69,20 @@ __device__ __forceinline__ void load_x8(const void* x, int64_t off, float (&xf)[
   }
 }
 
-template <bool X_F32, int NB, bool GATED>
+// KS = warps of a CTA that share the same rows and split K between them (KS consecutive warps act
+// as one group of 32 KS lanes); their partial sums meet in shared memory in a fixed order. Few
+// output rows with KS = 1 would leave most of the SMs' load slots empty.
+template <bool X_F32, int NB, bool GATED, int KS>
 __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
+  const int wic = threadIdx.x >> 5;                         // warp in CTA
+  const int slice = wic % KS;
+  const int warp = blockIdx.x * (8 / KS) + wic / KS;        // row group
   constexpr int R = GEMV_R;
   constexpr int RW = GATED ? 2 * R : R;           // weight rows streamed per warp
   const int n_out = GATED ? p.N / 2 : p.N;        // logical output rows
   const int o0 = warp * R;
-  if (o0 >= n_out) return;
+  if (KS == 1 && o0 >= n_out) return;
   // weight rows for output o: plain -> o; gated -> gate row (o/128)*256 + o%128, up row +128
   const bf16* wr[RW];
 #pragma unroll
@@ -93,18 +98,18 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 #pragma unroll
     for (int b = 0; b < NB; ++b) acc[r][b] = 0.f;
 
-  for (int k0 = lane * 8; k0 < p.K; k0 += 256 * GEMV_U) {
+  for (int k0 = (slice * 32 + lane) * 8; k0 < p.K; k0 += 256 * KS * GEMV_U) {
     uint4 wraw[GEMV_U][RW];
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
-      const int k = k0 + u * 256;
+      const int k = k0 + u * 256 * KS;
 #pragma unroll
       for (int r = 0; r < RW; ++r)
         wraw[u][r] = (k < p.K) ? ld_stream(wr[r] + k) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
-      const int k = k0 + u * 256;
+      const int k = k0 + u * 256 * KS;
       if (k < p.K) {
         float wf[RW][8];
 #pragma unroll
@@ -123,13 +128,35 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
       }
     }
   }
+  if (KS > 1) {
+    // slice 0 of every group adds the other slices' sums in slice order
+    __shared__ float part[8][RW][NB];
+#pragma unroll
+    for (int r = 0; r < RW; ++r)
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+        acc[r][b] = warp_sum(acc[r][b]);
+        if (lane == 0) part[wic][r][b] = acc[r][b];
+      }
+    __syncthreads();
+    if (slice != 0 || o0 >= n_out) return;
+#pragma unroll
+    for (int r = 0; r < RW; ++r)
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+        float v = 0.f;
+#pragma unroll
+        for (int sl = 0; sl < KS; ++sl) v += part[wic + sl][r][b];
+        acc[r][b] = v;
+      }
+  }
 #pragma unroll
   for (int r = 0; r < R; ++r) {
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       if (b < p.B) {
-        float v = warp_sum(acc[r][b]);
-        float u = GATED ? warp_sum(acc[GATED ? R + r : r][b]) : 0.f;
+        float v = KS > 1 ? acc[r][b] : warp_sum(acc[r][b]);
+        float u = GATED ? (KS > 1 ? acc[GATED ? R + r : r][b] : warp_sum(acc[GATED ? R + r : r][b])) : 0.f;
         const int o = o0 + r;
         if (lane == 0 && o < n_out) {
           if (p.mode == 0) {
@@ -145,12 +172,23 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   }
 }
 
-template <bool X_F32, bool GATED>
+template <bool X_F32, bool GATED, int KS>
 void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
-  if (p.B <= 1) gemv_kernel<X_F32, 1, GATED><<<blocks, 256, 0, s>>>(p);
-  else if (p.B <= 2) gemv_kernel<X_F32, 2, GATED><<<blocks, 256, 0, s>>>(p);
-  else if (p.B <= 4) gemv_kernel<X_F32, 4, GATED><<<blocks, 256, 0, s>>>(p);
-  else gemv_kernel<X_F32, 8, GATED><<<blocks, 256, 0, s>>>(p);
+  if (p.B <= 1) gemv_kernel<X_F32, 1, GATED, KS><<<blocks, 256, 0, s>>>(p);
+  else if (p.B <= 2) gemv_kernel<X_F32, 2, GATED, KS><<<blocks, 256, 0, s>>>(p);
+  else if (p.B <= 4) gemv_kernel<X_F32, 4, GATED, KS><<<blocks, 256, 0, s>>>(p);
+  else gemv_kernel<X_F32, 8, GATED, KS><<<blocks, 256, 0, s>>>(p);
+}
+
+template <bool X_F32, bool GATED>
+void launch_gemv_ks(const GemvDev& p, int row_warps, int ks, cudaStream_t s) {
+  const int blocks = ceil_div(row_warps * ks, 8);
+  switch (ks) {
+    case 8: launch_gemv_nb<X_F32, GATED, 8>(p, blocks, s); break;
+    case 4: launch_gemv_nb<X_F32, GATED, 4>(p, blocks, s); break;
+    case 2: launch_gemv_nb<X_F32, GATED, 2>(p, blocks, s); break;
+    default: launch_gemv_nb<X_F32, GATED, 1>(p, blocks, s); break;
+  }
 }
 
 // ------------------------------------------------------------------------------ decode attention
@@ -480,7 +518,9 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
   if (a.mode == 3 && (a.N % 256 || a.n_valid > a.N / 2)) return POP_E_INVALID;
   const int n_out = a.mode == 3 ? a.N / 2 : a.N;
   const int warps = ceil_div(n_out, GEMV_R);
-  const int blocks = ceil_div(warps, 8);
+  // split K between the warps of a CTA while all warps still fit on the GPU at once (148 SMs x 64)
+  int ks = 1;
+  while (ks < 8 && warps * ks * 2 <= 148 * 64 && a.K >= 256 * ks * 2) ks *= 2;
   const int elt = a.x_f32 ? 4 : 2;
   for (int b0 = 0; b0 < a.B; b0 += GEMV_MAXB) {
     GemvDev p;
@@ -493,11 +533,11 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
     p.N = a.N; p.K = a.K; p.mode = a.mode; p.act = a.act; p.n_valid = a.n_valid;
     ProfScope prof(PROF_GEMV, (double)a.N * a.K * 2, s);
     if (a.mode == 3) {
-      if (a.x_f32) launch_gemv_nb<true, true>(p, blocks, s);
-      else launch_gemv_nb<false, true>(p, blocks, s);
+      if (a.x_f32) launch_gemv_ks<true, true>(p, warps, ks, s);
+      else launch_gemv_ks<false, true>(p, warps, ks, s);
     } else {
-      if (a.x_f32) launch_gemv_nb<true, false>(p, blocks, s);
-      else launch_gemv_nb<false, false>(p, blocks, s);
+      if (a.x_f32) launch_gemv_ks<true, false>(p, warps, ks, s);
+      else launch_gemv_ks<false, false>(p, warps, ks, s);
     }
     count_launch();
   }
