@@ -35,6 +35,36 @@ struct ProfScope {   // records the start event on construction, the end event o
 };
 int prof_summary(int kind, double* total_ms, double* total_work, int64_t* launches);   // clears that kind
 
+// Chained launches of the single-row (boundary token / decode) kernels. A kernel launched with
+// launch_chained may become resident while the kernel before it on the stream is still running;
+// it calls chain_trigger() at its top (its own successor may then be made resident) and
+// chain_wait() before it reads anything an earlier kernel wrote and before it writes anything:
+// chain_wait() returns when the preceding kernel has completed and its writes are visible. Every
+// kernel of a chain waits, so completion is transitive. Before the wait a kernel touches only data
+// that no kernel ever writes (weights, gains, block tables). A kernel launched the ordinary way
+// after a chained one is ordered after it as usual. POP_CHAINED_LAUNCH=0 in the environment turns
+// the early residency off (the kernels then run strictly one after the other).
+bool chained_launch_enabled();
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <typename... P, typename... A>
+inline cudaError_t launch_chained(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                  A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained_launch_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+#endif
+
 // Tensor-map encoding through the driver entry point (no link-time dependency on libcuda).
 // 3-D bf16 tensor [dim2][dim1][dim0] with dim0 contiguous; strides in elements; 128-byte swizzle;
 // box = [1][box1][box0]; box0 must be 64 (128 bytes).

@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   constexpr int RW = GATED ? 2 * R : R;           // weight rows streamed per warp
   const int n_out = GATED ? p.N / 2 : p.N;        // logical output rows
   const int o0 = warp * R;
+  chain_trigger();
   if (KS == 1 && o0 >= n_out) return;
   // weight rows for output o: plain -> o; gated -> gate row (o/128)*256 + o%128, up row +128
   const bf16* wr[RW];
@@ -98,8 +99,9 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 #pragma unroll
     for (int b = 0; b < NB; ++b) acc[r][b] = 0.f;
 
-  for (int k0 = (slice * 32 + lane) * 8; k0 < p.K; k0 += 256 * KS * GEMV_U) {
-    uint4 wraw[GEMV_U][RW];
+  // the first batch of weight loads goes out before the wait on the preceding kernel: weights are
+  // never written by a kernel, the activations may be
+  auto load_batch = [&](uint4 (&wraw)[GEMV_U][RW], int k0) {
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
       const int k = k0 + u * 256 * KS;
@@ -107,6 +109,12 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
       for (int r = 0; r < RW; ++r)
         wraw[u][r] = (k < p.K) ? ld_stream(wr[r] + k) : make_uint4(0, 0, 0, 0);
     }
+  };
+  int k0 = (slice * 32 + lane) * 8;
+  uint4 wraw[GEMV_U][RW];
+  if (k0 < p.K) load_batch(wraw, k0);
+  chain_wait();
+  while (k0 < p.K) {
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
       const int k = k0 + u * 256 * KS;
@@ -127,6 +135,8 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
         }
       }
     }
+    k0 += 256 * KS * GEMV_U;
+    if (k0 < p.K) load_batch(wraw, k0);
   }
   if (KS > 1) {
     // slice 0 of every group adds the other slices' sums in slice order
@@ -174,10 +184,10 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 
 template <bool X_F32, bool GATED, int KS>
 void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
-  if (p.B <= 1) gemv_kernel<X_F32, 1, GATED, KS><<<blocks, 256, 0, s>>>(p);
-  else if (p.B <= 2) gemv_kernel<X_F32, 2, GATED, KS><<<blocks, 256, 0, s>>>(p);
-  else if (p.B <= 4) gemv_kernel<X_F32, 4, GATED, KS><<<blocks, 256, 0, s>>>(p);
-  else gemv_kernel<X_F32, 8, GATED, KS><<<blocks, 256, 0, s>>>(p);
+  if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
+  else if (p.B <= 2) launch_chained(gemv_kernel<X_F32, 2, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
+  else if (p.B <= 4) launch_chained(gemv_kernel<X_F32, 4, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
+  else launch_chained(gemv_kernel<X_F32, 8, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
 }
 
 template <bool X_F32, bool GATED>
@@ -309,6 +319,8 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   constexpr int KT = C::KT, WARPS = C::WARPS, ROWB = C::ROWB, CH = C::CH, NST = C::NST, NT = HD / 16;
   constexpr uint32_t FULL = 0xffffffffu;
   extern __shared__ __align__(128) uint8_t dec_smem[];
+  chain_trigger();
+  chain_wait();   // the query, the newest cache row and the run-time length come from earlier kernels
   const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
   const int G = p.n_q / p.n_kv;   // <= DEC_MAXG
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -498,7 +510,8 @@ int launch_dec_attn(const DecAttnDev& p, dim3 grid, cudaStream_t s) {
       return POP_E_CUDA;
     configured = true;
   }
-  dec_attn_kernel<HD><<<grid, C::WARPS * 32, C::SMEM, s>>>(p);
+  if (launch_chained(dec_attn_kernel<HD>, grid, dim3(C::WARPS * 32), (size_t)C::SMEM, s, p) != cudaSuccess)
+    return POP_E_CUDA;
   return POP_OK;
 }
 
@@ -507,6 +520,8 @@ __global__ void dec_combine_kernel(const DecAttnDev p) {
   // one CTA per (head, sequence)
   __shared__ float wgt[64];
   __shared__ float inv_l;
+  chain_trigger();
+  chain_wait();
   dec_combine_heads<HD>(p, blockIdx.y, blockIdx.x, 1, wgt, &inv_l);
 }
 
@@ -573,7 +588,7 @@ int launch_dec_pair(const DecAttnDev& p, int batch, cudaStream_t s) {
   if (rc != POP_OK) return rc;
   count_launch();
   if (p.counters == nullptr) {
-    dec_combine_kernel<HD><<<grid2, HD < 128 ? HD : 128, 0, s>>>(p);
+    launch_chained(dec_combine_kernel<HD>, grid2, dim3(HD < 128 ? HD : 128), 0, s, p);
     count_launch();
   }
   return POP_OK;

@@ -58,6 +58,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, int64_t ldx, const f
                                int64_t gain_stride, void* __restrict__ out, int64_t ldo, int64_t out_group_stride,
                                int d, float eps) {
   __shared__ float red[32];
+  chain_trigger();
+  chain_wait();
   const int row = blockIdx.x;
   const float* xr = x + (int64_t)row * ldx;
   float ss = 0.f;
@@ -92,6 +94,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, int64_t ldx, const f
 __global__ void postnorm_add_kernel(float* __restrict__ x, int64_t ldx, const float* __restrict__ t, int64_t ldt,
                                     const float* __restrict__ gain, int d, float eps) {
   __shared__ float red[32];
+  chain_trigger();
+  chain_wait();
   const int row = blockIdx.x;
   const float* tr = t + (int64_t)row * ldt;
   float* xr = x + (int64_t)row * ldx;
@@ -147,6 +151,8 @@ struct RopeDev {
 
 template <int HD>
 __global__ void rope_cache_kernel(const RopeDev p) {
+  chain_trigger();
+  chain_wait();
   constexpr int PER = HD / 64;            // rotation pairs per lane
   const int warps_per_block = blockDim.x >> 5;
   const int heads = p.n_q + 2 * p.n_kv;
@@ -285,9 +291,11 @@ int launch_rmsnorm(const float* x, int64_t ldx, const float* gain, int64_t gain_
   const int threads = d >= 2048 ? 256 : 128;
   ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * (4.0 + groups * (out_f32 ? 4.0 : 2.0)), s);
   if (out_f32)
-    rmsnorm_kernel<true><<<grid, threads, 0, s>>>(x, ldx, gain, gain_stride, out, ldo, out_group_stride, d, eps);
+    launch_chained(rmsnorm_kernel<true>, grid, dim3(threads), 0, s, x, ldx, gain, gain_stride, out, ldo,
+                   out_group_stride, d, eps);
   else
-    rmsnorm_kernel<false><<<grid, threads, 0, s>>>(x, ldx, gain, gain_stride, out, ldo, out_group_stride, d, eps);
+    launch_chained(rmsnorm_kernel<false>, grid, dim3(threads), 0, s, x, ldx, gain, gain_stride, out, ldo,
+                   out_group_stride, d, eps);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -296,7 +304,7 @@ int launch_postnorm_add(float* x, int64_t ldx, const float* t, int64_t ldt, cons
                         float eps, cudaStream_t s) {
   if (d % 4 || ldx % 4 || ldt % 4) return POP_E_INVALID;
   ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 12, s);
-  postnorm_add_kernel<<<rows, d >= 2048 ? 256 : 128, 0, s>>>(x, ldx, t, ldt, gain, d, eps);
+  launch_chained(postnorm_add_kernel, dim3(rows), dim3(d >= 2048 ? 256 : 128), 0, s, x, ldx, t, ldt, gain, d, eps);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -329,9 +337,9 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   dim3 grid((unsigned)((items + 7) / 8), a.groups);
   ProfScope prof(PROF_ELEMENTWISE, (double)items * a.groups * a.hd * 6, s);
   switch (a.hd) {
-    case 64: rope_cache_kernel<64><<<grid, 256, 0, s>>>(p); break;
-    case 128: rope_cache_kernel<128><<<grid, 256, 0, s>>>(p); break;
-    case 256: rope_cache_kernel<256><<<grid, 256, 0, s>>>(p); break;
+    case 64: launch_chained(rope_cache_kernel<64>, grid, dim3(256), 0, s, p); break;
+    case 128: launch_chained(rope_cache_kernel<128>, grid, dim3(256), 0, s, p); break;
+    case 256: launch_chained(rope_cache_kernel<256>, grid, dim3(256), 0, s, p); break;
     default: return POP_E_INVALID;
   }
   count_launch();

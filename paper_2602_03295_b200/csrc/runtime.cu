@@ -2,6 +2,8 @@
 // tensor-map encoding through the driver entry point.
 #include "common.cuh"
 
+#include <cstdlib>
+
 #include <atomic>
 #include <mutex>
 #include <vector>
@@ -49,6 +51,14 @@ static std::vector<ProfRecord> g_prof[PROF_KINDS];
 
 void prof_enable(bool on) { g_prof_on.store(on); }
 bool prof_enabled() { return g_prof_on.load(std::memory_order_relaxed); }
+
+bool chained_launch_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("POP_CHAINED_LAUNCH");
+    return !(e && e[0] == '0');
+  }();
+  return on;
+}
 
 ProfScope::ProfScope(int kind_, double work_, cudaStream_t s)
     : kind(kind_), work(work_), stream(s), e0(nullptr), e1(nullptr), active(false) {
