@@ -34,7 +34,7 @@ import pop_synth as ps  # noqa: E402
 METRIC = "pop_prefill_tokens_per_s"
 UNIT = "tokens/s"
 KERNELS = ["gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down", "kvproj", "attention", "attention_local", "gemv_head",
-           "decode_attention", "rmsnorm", "rope_cache"]
+           "decode_attention", "decode_step", "rmsnorm", "rope_cache"]
 
 
 def parse_args():
@@ -501,6 +501,23 @@ def run_kernel(a, wl):
         def launch(i):
             lib.decode_attention(q, cache.k[i % sets], cache.v[i % sets], cache.block_table, out, cfg.n_q_heads,
                                  cfg.n_kv_heads, hd, N, a.page_size, 0, counters=ctr, partial=part)
+    elif k == "decode_step":
+        # one position per sequence through all layers over the cache of a full-depth prefill (the
+        # single-row kernels: GEMV, norm, RoPE + cache write, split-KV attention, output head)
+        from paper_2602_03295_b200.binding import KVCache, PopModel
+        bound = "hbm"
+        N = wl.seq_len
+        model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+        cache = KVCache(cfg, wl.batch, N + 64, a.page_size, device=dev)
+        tokens, embeds = ps.make_prompt(wl)
+        model.prefill(tokens.to(dev), None if embeds is None else embeds.to(dev), cfg.n_layers, cache)
+        tok = torch.zeros(wl.batch, dtype=torch.int32, device=dev)
+        logits = torch.zeros(wl.batch, cfg.vocab, dtype=torch.float32, device=dev)
+        per_layer = d * (qd + 2 * kvd) + qd * d + 3 * d * F
+        work = 2.0 * (cfg.n_layers * per_layer + cfg.vocab * d) + 4.0 * wl.batch * N * kvd * cfg.n_layers
+
+        def launch(i):
+            model.decode_step(tok, N + i % 64, cache, logits)
     elif k == "rmsnorm":
         bound = "hbm"
         x = rnd(M, d, dtype=torch.float32)

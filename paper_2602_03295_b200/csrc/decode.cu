@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   const int lane = threadIdx.x & 31;
   const int wic = threadIdx.x >> 5;                         // warp in CTA
   const int slice = wic % KS;
-  const int warp = blockIdx.x * (8 / KS) + wic / KS;        // row group
+  const int warp = blockIdx.x * ((blockDim.x >> 5) / KS) + wic / KS;   // row group
   constexpr int R = GEMV_R;
   constexpr int RW = GATED ? 2 * R : R;           // weight rows streamed per warp
   const int n_out = GATED ? p.N / 2 : p.N;        // logical output rows
@@ -183,21 +183,24 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 }
 
 template <bool X_F32, bool GATED, int KS>
-void launch_gemv_nb(const GemvDev& p, int blocks, cudaStream_t s) {
-  if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
-  else if (p.B <= 2) launch_chained(gemv_kernel<X_F32, 2, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
-  else if (p.B <= 4) launch_chained(gemv_kernel<X_F32, 4, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
-  else launch_chained(gemv_kernel<X_F32, 8, GATED, KS>, dim3(blocks), dim3(256), 0, s, p);
+void launch_gemv_nb(const GemvDev& p, int blocks, int threads, cudaStream_t s) {
+  if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
+  else if (p.B <= 2) launch_chained(gemv_kernel<X_F32, 2, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
+  else if (p.B <= 4) launch_chained(gemv_kernel<X_F32, 4, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
+  else launch_chained(gemv_kernel<X_F32, 8, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
 }
 
 template <bool X_F32, bool GATED>
 void launch_gemv_ks(const GemvDev& p, int row_warps, int ks, cudaStream_t s) {
-  const int blocks = ceil_div(row_warps * ks, 8);
+  // the slices of a row group sit in one CTA of 8 warps; without a K split the warps are
+  // independent and CTAs of 4 warps spread more evenly over the SMs (fewer, shorter stragglers)
+  const int wpc = ks == 1 ? 4 : 8;
+  const int blocks = ceil_div(row_warps * ks, wpc);
   switch (ks) {
-    case 8: launch_gemv_nb<X_F32, GATED, 8>(p, blocks, s); break;
-    case 4: launch_gemv_nb<X_F32, GATED, 4>(p, blocks, s); break;
-    case 2: launch_gemv_nb<X_F32, GATED, 2>(p, blocks, s); break;
-    default: launch_gemv_nb<X_F32, GATED, 1>(p, blocks, s); break;
+    case 8: launch_gemv_nb<X_F32, GATED, 8>(p, blocks, 256, s); break;
+    case 4: launch_gemv_nb<X_F32, GATED, 4>(p, blocks, 256, s); break;
+    case 2: launch_gemv_nb<X_F32, GATED, 2>(p, blocks, 256, s); break;
+    default: launch_gemv_nb<X_F32, GATED, 1>(p, blocks, wpc * 32, s); break;
   }
 }
 

@@ -57,37 +57,62 @@ template <bool OUT_F32>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ gain,
                                int64_t gain_stride, void* __restrict__ out, int64_t ldo, int64_t out_group_stride,
                                int d, float eps) {
+  // The first RN_CACHE float4 per thread of the row and of the gain stay in registers (rows up to
+  // 16 * blockDim floats are read exactly once); longer rows re-read their remainder from L1/L2.
+  constexpr int RN_CACHE = 4;
   __shared__ float red[32];
   chain_trigger();
-  chain_wait();
-  const int row = blockIdx.x;
+  const int row = blockIdx.x, g = blockIdx.y;
   const float* xr = x + (int64_t)row * ldx;
+  const float* gr = gain + (int64_t)g * gain_stride;
+  const int step = blockDim.x * 4;
+  // gains are weights, never written by a kernel: their loads go out before the wait on the producer of x
+  float4 gv[RN_CACHE];
+#pragma unroll
+  for (int i = 0; i < RN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    gv[i] = c < d ? *reinterpret_cast<const float4*>(gr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  chain_wait();
+  float4 xv[RN_CACHE];
+#pragma unroll
+  for (int i = 0; i < RN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    xv[i] = c < d ? *reinterpret_cast<const float4*>(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+#pragma unroll
+  for (int i = 0; i < RN_CACHE; ++i) {
+    const float4 v = xv[i];
+    if (threadIdx.x * 4 + i * step < d) ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  for (int c = threadIdx.x * 4 + RN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(xr + c);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, red);
   const float rstd = rsqrtf(ss / (float)d + eps);
-  for (int g = blockIdx.y; g < (int)gridDim.y; g += gridDim.y) {
-    const float* gr = gain + (int64_t)g * gain_stride;
-    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-      const float4 v = *reinterpret_cast<const float4*>(xr + c);
-      const float4 w = *reinterpret_cast<const float4*>(gr + c);
-      const float a = v.x * rstd * w.x, b = v.y * rstd * w.y, c2 = v.z * rstd * w.z, e = v.w * rstd * w.w;
-      if (OUT_F32) {
-        float* o = reinterpret_cast<float*>(out) + (int64_t)g * out_group_stride + (int64_t)row * ldo + c;
-        *reinterpret_cast<float4*>(o) = make_float4(a, b, c2, e);
-      } else {
-        bf16* o = reinterpret_cast<bf16*>(out) + (int64_t)g * out_group_stride + (int64_t)row * ldo + c;
-        __nv_bfloat162 p0 = __floats2bfloat162_rn(a, b), p1 = __floats2bfloat162_rn(c2, e);
-        uint2 w2;
-        w2.x = *reinterpret_cast<uint32_t*>(&p0);
-        w2.y = *reinterpret_cast<uint32_t*>(&p1);
-        *reinterpret_cast<uint2*>(o) = w2;
-      }
+  auto emit = [&](int c, const float4& v, const float4& w) {
+    const float a = v.x * rstd * w.x, b = v.y * rstd * w.y, c2 = v.z * rstd * w.z, e = v.w * rstd * w.w;
+    if (OUT_F32) {
+      float* o = reinterpret_cast<float*>(out) + (int64_t)g * out_group_stride + (int64_t)row * ldo + c;
+      *reinterpret_cast<float4*>(o) = make_float4(a, b, c2, e);
+    } else {
+      bf16* o = reinterpret_cast<bf16*>(out) + (int64_t)g * out_group_stride + (int64_t)row * ldo + c;
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(a, b), p1 = __floats2bfloat162_rn(c2, e);
+      uint2 w2;
+      w2.x = *reinterpret_cast<uint32_t*>(&p0);
+      w2.y = *reinterpret_cast<uint32_t*>(&p1);
+      *reinterpret_cast<uint2*>(o) = w2;
     }
+  };
+#pragma unroll
+  for (int i = 0; i < RN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    if (c < d) emit(c, xv[i], gv[i]);
   }
+  for (int c = threadIdx.x * 4 + RN_CACHE * step; c < d; c += step)
+    emit(c, *reinterpret_cast<const float4*>(xr + c), *reinterpret_cast<const float4*>(gr + c));
 }
 
 // x[row][:] += rmsnorm(t[row][:]) * gain      (post-norm models: norm of the sublayer output)
