@@ -90,14 +90,14 @@ def gated_act(gate: torch.Tensor, up: torch.Tensor, act: int) -> torch.Tensor:
 
 
 def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, q_pos: torch.Tensor,
-              window: int, precision: str = "exact") -> torch.Tensor:
+              window: int, precision: str = "exact", k_pos0: int = 0) -> torch.Tensor:
     """Attn of Eq. 1 for one sequence. q: [T, n_q, hd] at absolute positions q_pos [T];
-    k, v: [S, n_kv, hd] holding cache positions 0..S-1. Query at position i sees keys
+    k, v: [S, n_kv, hd] holding cache positions k_pos0..k_pos0+S-1. Query at position i sees keys
     j <= i, and j > i - window when window > 0. Returns [T, n_q, hd]."""
     T, n_q, hd = q.shape
     S, n_kv, _ = k.shape
     out = torch.empty_like(q)
-    kpos = torch.arange(S)
+    kpos = torch.arange(S) + k_pos0
     allowed = kpos[None, :] <= q_pos[:, None]
     if window > 0:
         allowed &= kpos[None, :] > (q_pos[:, None] - window)
@@ -152,21 +152,23 @@ def kv_generation(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
 
 def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Tensor,
                   k_past: Optional[torch.Tensor], v_past: Optional[torch.Tensor],
-                  dtype, precision: str):
+                  dtype, precision: str, k_pos0: int = 0):
     """One full decoder layer (Eq. 1-3) on the T new positions `positions` of one sequence,
-    given the cache of earlier positions. Returns x_{l+1} [T, d], K_cur, V_cur."""
+    given the cache of earlier positions (its first entry is position k_pos0; with no past
+    entries the new positions are the whole cache). Returns x_{l+1} [T, d], K_cur, V_cur."""
     k_new, v_new = kv_generation(cfg, weights, layer, x, positions, dtype, precision)
     if k_past is not None and k_past.shape[0] > 0:
         k_cur = torch.cat([k_past, k_new], dim=0)                       # Eq. 3
         v_cur = torch.cat([v_past, v_new], dim=0)
     else:
         k_cur, v_cur = k_new, v_new
+        k_pos0 = int(positions[0])
     h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
     q = (h @ _w(weights, "wq", layer, dtype).T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
     if cfg.qk_norm:
         q = rmsnorm(q, _w(weights, "q_norm", layer, dtype), cfg.rms_eps)
     q = _rnd(rope(q, positions, cfg.rope_theta), precision)
-    a = attention(q, k_cur, v_cur, positions, cfg.layer_window(layer), precision)
+    a = attention(q, k_cur, v_cur, positions, cfg.layer_window(layer), precision, k_pos0)
     a = _rnd(a.reshape(-1, cfg.q_dim), precision)
     o = a @ _w(weights, "wo", layer, dtype).T
     if cfg.post_norms:
@@ -226,7 +228,8 @@ def full_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tens
 
 
 def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], l_keep: int,
-                dtype=torch.float64, precision: str = "exact", skip=None):
+                dtype=torch.float64, precision: str = "exact", skip=None, boundary: bool = True,
+                indep_kv: bool = True):
     """POP inference up to the first generated token, in the paper's two phases (Sec. 3.3).
 
     Phase 1, pruned prefill on x_{1:N-1}: layers 1..L_keep run in full; each layer
@@ -241,9 +244,19 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     explicitly instead of the deep suffix {l_keep+1..L}; it may be shallow or interleaved (the
     layer-selection ablation of Sec. 4.4). A pruned layer projects whatever state reaches it.
 
+    The two component ablations of Sec. 4.4.1 (Table "design choices"):
+      boundary=False ("w/o Boundary Handling"): x_N is processed by the pruned prefill model like
+        every other position: phase 1 covers all N positions, there is no phase 2, and the logits
+        come from the state that leaves phase 1 at position N.
+      indep_kv=False ("w/o Indep. KV Proj."): pruned layers generate no cache entries in phase 1;
+        in phase 2 (and in later decode steps) such a layer can only attend to positions >= N.
+        Their K, V rows of positions 1..N-1 are returned as NaN ("absent").
+
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
-    H [B, N-1, d] (the state leaving the last layer of phase 1; for the deep-suffix set this is
-    the state leaving the kept stack)."""
+    H [B, N-1, d] (the state leaving the last layer of phase 1 at positions 1..N-1; for the
+    deep-suffix set this is the state leaving the kept stack), first_pos (per layer, 0-based: the
+    first cache position later decode steps may attend to: 0, or N-1 for pruned layers when
+    indep_kv is off)."""
     L = cfg.n_layers
     if skip is None:
         assert 1 <= l_keep <= L
@@ -259,34 +272,50 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
         x_all = embed(cfg, weights, tokens[b], None if embeds is None else embeds[b], dtype)
         kc = [None] * L
         vc = [None] * L
-        # ---- phase 1: pruned prefill on positions 0..N-2
-        if N > 1:
-            pos = torch.arange(N - 1)
-            x = x_all[: N - 1]
+        # ---- phase 1: pruned prefill on positions 0..N-2 (on all N positions without boundary handling)
+        n1 = N - 1 if boundary else N
+        if n1 > 0:
+            pos = torch.arange(n1)
+            x = x_all[:n1]
             for l in range(1, L + 1):
                 if l not in skip:
                     x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, pos, None, None,
                                                             dtype, precision)
-                else:
+                elif indep_kv:
                     kc[l - 1], vc[l - 1] = kv_generation(cfg, weights, l, x, pos, dtype, precision)
                     # Eq. 15: x is handed to layer l+1 unchanged
-            H[b] = x
-        # ---- phase 2: x_N as the first decode step of the full model
-        posN = torch.tensor([N - 1])
-        x = x_all[N - 1: N]
-        for l in range(1, L + 1):
-            x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1],
-                                                    dtype, precision)
+            H[b] = x[: N - 1]
+        if boundary:
+            # ---- phase 2: x_N as the first decode step of the full model
+            posN = torch.tensor([N - 1])
+            x = x_all[N - 1: N]
+            for l in range(1, L + 1):
+                x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1],
+                                                        dtype, precision)
+            x_last = x[0]
+        else:
+            x_last = x[N - 1]
         for l in range(L):
-            K[l][b], V[l][b] = kc[l], vc[l]
-        logits[b] = lm_logits(cfg, weights, x[0], dtype)
-    return {"K": K, "V": V, "logits": logits, "H": H}
+            if kc[l] is None:                    # pruned layer without cache entries, no phase 2
+                K[l][b] = float("nan")
+                V[l][b] = float("nan")
+            else:
+                absent = N - kc[l].shape[0]      # positions a pruned layer holds nothing for
+                K[l][b, :absent] = float("nan")
+                V[l][b, :absent] = float("nan")
+                K[l][b, absent:], V[l][b, absent:] = kc[l], vc[l]
+        logits[b] = lm_logits(cfg, weights, x_last, dtype)
+    first_pos = [N - 1 if (not indep_kv and (l + 1) in skip) else 0 for l in range(L)]
+    return {"K": K, "V": V, "logits": logits, "H": H, "first_pos": first_pos}
 
 
-def decode_step(cfg, weights, tokens: torch.Tensor, K, V, dtype=torch.float64, precision: str = "exact"):
+def decode_step(cfg, weights, tokens: torch.Tensor, K, V, dtype=torch.float64, precision: str = "exact",
+                first_pos=None):
     """One decode step of the FULL model over an existing cache (Sec. 2.2, decode stage; Eq. 1-3):
     POP prunes nothing here ("retaining the full model for decode"). tokens: int [B], the token at
     position n = current cache length; K, V: lists (one per layer) of [B, n, n_kv, hd].
+    first_pos (per layer, 0-based) is the first cache position a layer may attend to: positions
+    before it hold nothing (the "w/o Indep. KV Proj." ablation of Sec. 4.4.1).
     Returns (K', V', logits): caches with n + 1 entries and the next-token logits [B, vocab]."""
     L = cfg.n_layers
     B = tokens.shape[0]
@@ -298,8 +327,11 @@ def decode_step(cfg, weights, tokens: torch.Tensor, K, V, dtype=torch.float64, p
     for b in range(B):
         x = embed(cfg, weights, tokens[b: b + 1], None, dtype)
         for l in range(1, L + 1):
-            x, K2[l - 1][b], V2[l - 1][b] = layer_forward(cfg, weights, l, x, pos, K[l - 1][b].to(dtype),
-                                                          V[l - 1][b].to(dtype), dtype, precision)
+            f = 0 if first_pos is None else int(first_pos[l - 1])
+            x, k_cur, v_cur = layer_forward(cfg, weights, l, x, pos, K[l - 1][b, f:].to(dtype),
+                                            V[l - 1][b, f:].to(dtype), dtype, precision, k_pos0=f)
+            K2[l - 1][b, :f], V2[l - 1][b, :f] = K[l - 1][b, :f], V[l - 1][b, :f]
+            K2[l - 1][b, f:], V2[l - 1][b, f:] = k_cur, v_cur
         logits[b] = lm_logits(cfg, weights, x[0], dtype)
     return K2, V2, logits
 

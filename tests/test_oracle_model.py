@@ -390,6 +390,80 @@ def test_explicit_skip_sets():
     assert _maxdiff(sh["logits"], po.pop_prefill(cfg, w, tokens, None, 2)["logits"]) > 1e-6
 
 
+def test_without_boundary_handling_the_last_token_sees_the_pruned_model():
+    # Sec. 4.4.1 "w/o Boundary Handling": x_N goes through the pruned prefill model. Pruned layers pass
+    # the state on unchanged (Eq. 15), so the logits are those of the model truncated to its kept
+    # layers, and every position of a pruned layer -- the last included -- holds Eq. 14 of the kept
+    # stack's output.
+    for variant in ("llama", "gemma"):
+        cfg, w, tokens = _setup(variant, n=9, batch=2)
+        L, lk, N = cfg.n_layers, 2, tokens.shape[1]
+        r = po.pop_prefill(cfg, w, tokens, None, lk, boundary=False)
+        trunc = po.full_prefill(cfg, w, tokens, n_layers=lk)
+        assert _maxdiff(r["logits"], trunc["logits"]) < 1e-11
+        assert _maxdiff(r["logits"], po.pop_prefill(cfg, w, tokens, None, lk)["logits"]) > 1e-6
+        for l in range(lk):
+            assert _maxdiff(r["K"][l], trunc["K"][l]) < 1e-11 and _maxdiff(r["V"][l], trunc["V"][l]) < 1e-11
+        for bi in range(tokens.shape[0]):
+            for l in range(lk + 1, L + 1):
+                k, v = po.kv_generation(cfg, w, l, trunc["hidden"][bi], torch.arange(N), torch.float64, "exact")
+                assert _maxdiff(r["K"][l - 1][bi], k) < 1e-11 and _maxdiff(r["V"][l - 1][bi], v) < 1e-11
+        assert r["first_pos"] == [0] * L
+
+
+def test_without_independent_kv_a_pruned_layer_attends_to_the_last_token_only():
+    # Sec. 4.4.1 "w/o Indep. KV Proj.": pruned layers generate no cache in the prefill, so in the first
+    # decode step such a layer sees one key, its own: softmax over one score is 1 and the attention
+    # output is the token's own value vector (repeated over the query heads of a group), whatever q is.
+    cfg, w, tokens = _setup("llama", n=7, batch=2)          # 3 layers, no window, no post norms
+    L, lk, N = cfg.n_layers, 2, tokens.shape[1]
+    r = po.pop_prefill(cfg, w, tokens, None, lk, indep_kv=False)
+    ref = po.pop_prefill(cfg, w, tokens, None, lk)
+    assert r["first_pos"] == [0, 0, N - 1]
+    # kept layers are untouched; the pruned layer holds nothing before the last position
+    for l in range(lk):
+        assert _maxdiff(r["K"][l], ref["K"][l]) == 0 and _maxdiff(r["V"][l], ref["V"][l]) == 0
+    assert torch.isnan(r["K"][lk][:, : N - 1]).all() and torch.isnan(r["V"][lk][:, : N - 1]).all()
+    # its entry of the last position comes from the true state, as with boundary handling
+    assert _maxdiff(r["K"][lk][:, N - 1], ref["K"][lk][:, N - 1]) < 1e-11
+    # closed form of the pruned layer for the last token, written with plain matrix products
+    f64 = torch.float64
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    for bi in range(tokens.shape[0]):
+        full = po.full_prefill(cfg, w, tokens[bi: bi + 1], n_layers=lk)
+        x = full["hidden"][0, N - 1]                         # the last token's state entering layer lk + 1
+        v_own = r["V"][lk][bi, N - 1]                        # [n_kv, hd]
+        a = v_own.repeat_interleave(G, dim=0).reshape(-1)    # attention output = own value per query head
+        y = x + w.get("wo", lk + 1).to(f64) @ a
+        h2 = po.rmsnorm(y, w.get("ln_ffn", lk + 1).to(f64), cfg.rms_eps)
+        f = w.get("w_down", lk + 1).to(f64) @ po.gated_act(w.get("w_gate", lk + 1).to(f64) @ h2,
+                                                             w.get("w_up", lk + 1).to(f64) @ h2, cfg.act)
+        assert _maxdiff(r["logits"][bi], po.lm_logits(cfg, w, y + f, f64)) < 1e-10
+    assert _maxdiff(r["logits"], ref["logits"]) > 1e-6
+    # later decode steps keep that horizon: the pruned layer attends from position N-1 on, which is the
+    # same as handing it a cache that starts there
+    nxt = torch.tensor([5, 11])
+    K2, V2, lg = po.decode_step(cfg, w, nxt, r["K"], r["V"], first_pos=r["first_pos"])
+    Kc = [k.clone() for k in r["K"]]
+    Vc = [v.clone() for v in r["V"]]
+    for bi in range(2):
+        x = po.embed(cfg, w, nxt[bi: bi + 1], None, f64)
+        for l in range(1, L + 1):
+            f0 = r["first_pos"][l - 1]
+            x, kk, vv = po.layer_forward(cfg, w, l, x, torch.tensor([N]), Kc[l - 1][bi, f0:], Vc[l - 1][bi, f0:],
+                                         f64, "exact", k_pos0=f0)
+            assert _maxdiff(K2[l - 1][bi, f0:], kk) < 1e-12
+        assert _maxdiff(lg[bi], po.lm_logits(cfg, w, x[0], f64)) < 1e-12
+    # and the horizon matters: with the (NaN) rows before it the result would not even be finite
+    assert torch.isfinite(lg).all()
+    # a windowed model: the horizon and the window combine (keys must satisfy both)
+    cfg, w, tokens = _setup("gemma", n=9, batch=1)           # window 3 in local layers
+    r = po.pop_prefill(cfg, w, tokens, None, 2, indep_kv=False)
+    assert torch.isfinite(r["logits"]).all()
+    K2, V2, lg = po.decode_step(cfg, w, torch.tensor([3]), r["K"], r["V"], first_pos=r["first_pos"])
+    assert torch.isfinite(lg).all()
+
+
 def test_single_token_prompt_has_an_empty_first_phase():
     cfg, w, tokens = _setup("llama", n=1)
     pop = po.pop_prefill(cfg, w, tokens, None, 1)
