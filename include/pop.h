@@ -139,6 +139,33 @@ int pop_prefill_ragged(pop_model_t* m, const pop_input_t* tokens_or_embeds, cons
 int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      const uint8_t* skip, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
+/* The two component ablations of the paper's Sec. 4.4.1 ("Effectiveness of Design Choices") on top
+ * of pop_prefill_skip; flags is a combination of
+ *   POP_NO_BOUNDARY  "w/o Boundary Handling": the last prompt token is processed by the pruned
+ *                    prefill model like every other position (pruned layers store their Eq. 14
+ *                    projections for all seq_len positions, there is no full-depth pass for the last
+ *                    token) and logits_out comes from the state that leaves the pruned model there;
+ *   POP_NO_INDEP_KV  "w/o Indep. KV Proj.": pruned layers generate no cache entries for the prompt
+ *                    (their rows of positions 0..seq_len-2 are left untouched); in the last token's
+ *                    full-depth pass such a layer attends to position seq_len-1 only. Later decode
+ *                    steps must keep that horizon: use pop_decode_step_from.
+ * flags = 0 is pop_prefill_skip. Other arguments, outputs and errors as pop_prefill_skip;
+ * POP_E_INVALID for unknown flag bits. */
+#define POP_NO_BOUNDARY 1
+#define POP_NO_INDEP_KV 2
+int pop_prefill_ablation(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
+                         const uint8_t* skip, int32_t flags, pop_kv_cache_t* kv_cache_out, float* logits_out,
+                         void* stream);
+
+/* pop_decode_step with an attention horizon per layer: layer_first_pos is a HOST array of n_layers
+ * int32; layer l attends to cache positions layer_first_pos[l-1] .. pos only (and within its window,
+ * if it has one). After pop_prefill_ablation(POP_NO_INDEP_KV) on seq_len = N tokens the pruned layers
+ * take N-1 (N if POP_NO_BOUNDARY was set as well: they then hold nothing of the prompt), the others 0 (paper Sec. 4.4.1: the model "can only access the last input token and the
+ * generated tokens" in those layers). NULL = pop_decode_step. POP_E_INVALID if an entry is negative
+ * or beyond pos. */
+int pop_decode_step_from(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch,
+                         const int32_t* layer_first_pos, pop_kv_cache_t* kv_cache, float* logits_out, void* stream);
+
 /* One decode step of the FULL model over the cache a prefill left (paper Sec. 2.2, decode stage;
  * Sec. 3: "retaining the full model for decode"): tokens is device int32 [batch], the token of
  * each sequence at position `pos` = number of entries its cache already holds. Every layer

@@ -255,8 +255,8 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
     H [B, N-1, d] (the state leaving the last layer of phase 1 at positions 1..N-1; for the
     deep-suffix set this is the state leaving the kept stack), first_pos (per layer, 0-based: the
-    first cache position later decode steps may attend to: 0, or N-1 for pruned layers when
-    indep_kv is off)."""
+    first cache position later decode steps may attend to: 0, or for pruned layers when
+    indep_kv is off N-1, the entry phase 2 wrote -- N if there was no phase 2 either)."""
     L = cfg.n_layers
     if skip is None:
         assert 1 <= l_keep <= L
@@ -305,7 +305,8 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
                 V[l][b, :absent] = float("nan")
                 K[l][b, absent:], V[l][b, absent:] = kc[l], vc[l]
         logits[b] = lm_logits(cfg, weights, x_last, dtype)
-    first_pos = [N - 1 if (not indep_kv and (l + 1) in skip) else 0 for l in range(L)]
+    horizon = N - 1 if boundary else N           # without phase 2 a pruned layer holds nothing at all
+    first_pos = [horizon if (not indep_kv and (l + 1) in skip) else 0 for l in range(L)]
     return {"K": K, "V": V, "logits": logits, "H": H, "first_pos": first_pos}
 
 

@@ -53,6 +53,8 @@ class pop_input_t(C.Structure):
 
 # name -> (restype, argtypes); every symbol declared in include/*.h
 _I32, _I64, _P, _F = C.c_int32, C.c_int64, C.c_void_p, C.c_float
+POP_NO_BOUNDARY, POP_NO_INDEP_KV = 1, 2
+
 SIGNATURES = {
     "pop_weight_arena_bytes": (C.c_size_t, [C.POINTER(pop_config_t)]),
     "pop_load_weights": (C.c_int, [C.POINTER(pop_config_t), C.POINTER(pop_tensor_t), _I32, _P, C.c_size_t, _P,
@@ -65,7 +67,10 @@ SIGNATURES = {
                                      _P, _P]),
     "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
                                    _P]),
+    "pop_prefill_ablation": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, _I32,
+                                       C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
+    "pop_decode_step_from": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_I32), C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_generate_greedy": (C.c_int, [_P, _P, _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P, _P]),
     "pop_last_status": (C.c_int, [_P, _P]),
     "pop_last_launch_count": (_I64, [_P]),
@@ -441,16 +446,44 @@ class PopModel:
         self.lib.check(code, "pop_prefill_skip")
         return logits
 
-    def decode_step(self, tokens, pos: int, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None):
-        """pop_decode_step: tokens int32 [B] on the device, each at position `pos` of its sequence."""
+    def prefill_ablation(self, tokens, embeds, skip, cache: KVCache, boundary: bool = True, indep_kv: bool = True,
+                         logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_prefill_ablation: pop_prefill_skip without boundary handling and / or without the pruned
+        layers' independent KV projections. Returns (logits, layer_first_pos) where layer_first_pos is
+        what later decode_step calls must be given (None when every layer holds the whole prompt)."""
+        B, N = tokens.shape
+        self.ensure_workspace(N, B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        skip = set(skip)
+        mask = bytes(1 if (l + 1) in skip else 0 for l in range(self.cfg.n_layers))
+        flags = (0 if boundary else POP_NO_BOUNDARY) | (0 if indep_kv else POP_NO_INDEP_KV)
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_prefill_ablation(self.handle, C.byref(inp), N, B, mask, flags, C.byref(kc),
+                                                 logits.data_ptr(), _stream_ptr(stream))
+        self.lib.check(code, "pop_prefill_ablation")
+        horizon = N - 1 if boundary else N       # without the full-depth pass a pruned layer holds nothing at all
+        first = None if indep_kv else [horizon if (l + 1) in skip else 0 for l in range(self.cfg.n_layers)]
+        return logits, first
+
+    def decode_step(self, tokens, pos: int, cache: KVCache, logits: Optional[torch.Tensor] = None, stream=None,
+                    layer_first_pos=None):
+        """pop_decode_step: tokens int32 [B] on the device, each at position `pos` of its sequence.
+        layer_first_pos (n_layers ints) -> pop_decode_step_from: per-layer attention horizon."""
         B = tokens.shape[0]
         self.ensure_workspace(1, B) if self.ws is None else None
         if logits is None:
             logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
         kc = cache.struct()
-        code = self.lib.dll.pop_decode_step(self.handle, tokens.data_ptr(), pos, B, C.byref(kc), logits.data_ptr(),
-                                            _stream_ptr(stream))
-        self.lib.check(code, "pop_decode_step")
+        if layer_first_pos is None:
+            code = self.lib.dll.pop_decode_step(self.handle, tokens.data_ptr(), pos, B, C.byref(kc),
+                                                logits.data_ptr(), _stream_ptr(stream))
+            self.lib.check(code, "pop_decode_step")
+        else:
+            arr = (_I32 * self.cfg.n_layers)(*[int(v) for v in layer_first_pos])
+            code = self.lib.dll.pop_decode_step_from(self.handle, tokens.data_ptr(), pos, B, arr, C.byref(kc),
+                                                     logits.data_ptr(), _stream_ptr(stream))
+            self.lib.check(code, "pop_decode_step_from")
         return logits
 
     def generate_greedy(self, first_tokens, pos0: int, n_steps: int, cache: KVCache,

@@ -221,7 +221,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
 // Independent K/V projections of pruned layers l0..l0+n-1 (paper Eq. 14) from the state H held in
 // w.x, for positions 0..N-2 of every sequence; the state itself is left unchanged (Eq. 15).
 int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, const pop_kv_cache_t* kc,
-              cudaStream_t s, const int32_t* cu = nullptr, int rows = 0) {
+              cudaStream_t s, const int32_t* cu = nullptr, int rows = 0, bool write_last = false) {
   const pop_config_t& c = m->cfg;
   const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -236,8 +236,9 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   r.k_gain = c.qk_norm ? lp<float>(m, l0, m->lo.k_norm) : nullptr;
   r.gain_group_stride = (int64_t)(m->layer_stride / 4);
   r.table = w.rope; r.n_q = 0; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
-  r.rows = M; r.rows_per_seq = N; r.rows_written = N - 1; r.pos0 = 0; r.groups = n; r.eps = c.rms_eps;
-  r.cu_seqlens = cu; r.batch = B; r.skip_last = 1;
+  r.rows = M; r.rows_per_seq = N; r.rows_written = write_last ? N : N - 1; r.pos0 = 0; r.groups = n;
+  r.eps = c.rms_eps;
+  r.cu_seqlens = cu; r.batch = B; r.skip_last = write_last ? 0 : 1;
   // ONE batched GEMM over the pruned layers (the layer is the batch dimension of both operands);
   // its epilogue applies each layer's K norm and RoPE and writes the layer's cache entries
   GemmArgs g{};
@@ -252,7 +253,7 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
 // `table` holds rotary rows starting at position `table_pos0`.
 int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc,
                    const float2* table, int table_pos0, cudaStream_t s, const int32_t* cu = nullptr,
-                   const int32_t* pos_dev = nullptr) {
+                   const int32_t* pos_dev = nullptr, int kv_first = 0) {
   const pop_config_t& c = m->cfg;
   const int d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -280,6 +281,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.partial = w.partial; a.out = w.ob; a.ldo = m->q_dim;
   a.batch = B; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads; a.head_dim = c.head_dim; a.kv_len = N;
   a.cu_seqlens = cu; a.pos_dev = pos_dev; a.counters = w.dec_ctr;
+  a.kv_first = kv_first;
   a.window = layer_window(c, l);
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};
@@ -414,8 +416,10 @@ int run_prefill_ragged(pop_model* m, const pop_input_t* in, const int32_t* seq_l
 // prompt, a kept layer in full, a pruned layer storing only its K/V projections of the state that
 // reaches it; phase 2 runs the boundary token through ALL layers as a decode step, which also
 // overwrites whatever phase 1 left at the last position of each layer's cache.
-int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const uint8_t* skip, pop_kv_cache_t* kc,
-                     float* logits, cudaStream_t s) {
+int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const uint8_t* skip, int flags,
+                     pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
+  if (flags & ~(POP_NO_BOUNDARY | POP_NO_INDEP_KV)) return POP_E_INVALID;
+  const bool boundary = !(flags & POP_NO_BOUNDARY), indep_kv = !(flags & POP_NO_INDEP_KV);
   if (!m || !in || !in->tokens || !skip || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
     return POP_E_INVALID;
   const pop_config_t& c = m->cfg;
@@ -433,14 +437,22 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
   POP_TRY(launch_rope_table(w.rope, N, c.head_dim, c.rope_theta, s));
   POP_TRY(launch_embed(in->tokens, (const bf16*)(m->arena + m->off_embed), (const bf16*)in->embeds, w.x, M, d,
                        c.vocab, s));
-  POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));       // x_1 of the boundary token, kept for phase 2
-  if (N > 1) {
+  if (boundary) POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));   // x_1 of the boundary token, kept for phase 2
+  if (N > 1 || !boundary) {
     for (int l = 1; l <= c.n_layers; ++l) {
-      if (skip[l - 1]) POP_TRY(pruned_kv(m, w, l, 1, N, B, kc, s));
-      else POP_TRY(full_layer(m, w, l, N, B, kc, s));
+      if (!skip[l - 1]) POP_TRY(full_layer(m, w, l, N, B, kc, s));
+      else if (indep_kv) POP_TRY(pruned_kv(m, w, l, 1, N, B, kc, s, nullptr, 0, !boundary));
     }
   }
-  for (int l = 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s));
+  if (boundary) {
+    // without independent KV projections a pruned layer holds nothing before position N-1
+    for (int l = 1; l <= c.n_layers; ++l)
+      POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s, nullptr, nullptr,
+                             (!indep_kv && skip[l - 1]) ? N - 1 : 0));
+  } else {
+    // the last token went through the pruned model with all the others: its logits come from there
+    POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
+  }
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};
@@ -454,13 +466,14 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
 // The kernels of one decode step. The position comes from the host (`pos`) or, when `pos_dev` is
 // given, from device memory at run time.
 int decode_body(pop_model* m, const Workspace& w, const int32_t* tokens, int pos, const int32_t* pos_dev, int B,
-                pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
+                pop_kv_cache_t* kc, float* logits, cudaStream_t s, const int32_t* layer_first_pos = nullptr) {
   const pop_config_t& c = m->cfg;
   const int d = c.d_model;
   POP_TRY(launch_rope_table(w.rope1, 1, c.head_dim, c.rope_theta, s, pos, pos_dev));
   POP_TRY(launch_embed(tokens, (const bf16*)(m->arena + m->off_embed), nullptr, w.xb, B, d, c.vocab, s));
   for (int l = 1; l <= c.n_layers; ++l)
-    POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s, nullptr, pos_dev));
+    POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s, nullptr, pos_dev,
+                           layer_first_pos ? layer_first_pos[l - 1] : 0));
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};
@@ -472,9 +485,12 @@ int decode_body(pop_model* m, const Workspace& w, const int32_t* tokens, int pos
 // One decode step of the full model (paper Sec. 2.2): every sequence's token at position `pos`
 // (= entries already in the cache) goes through all L layers as the boundary token does.
 int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache_t* kc, float* logits,
-               cudaStream_t s) {
+               cudaStream_t s, const int32_t* layer_first_pos = nullptr) {
   if (!m || !tokens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits) return POP_E_INVALID;
   const pop_config_t& c = m->cfg;
+  if (layer_first_pos)
+    for (int l = 0; l < c.n_layers; ++l)
+      if (layer_first_pos[l] < 0 || layer_first_pos[l] > pos) return POP_E_INVALID;
   if (pos < 0 || B < 1 || pos > (1 << 24)) return POP_E_INVALID;
   if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
   if ((int64_t)ceil_div(pos + 1, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
@@ -485,7 +501,7 @@ int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache
   // the workspace is the caller's between calls: the split-merge counters start from zero in every call
   if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
   const int64_t launches0 = launch_count();
-  POP_TRY(decode_body(m, w, tokens, pos, nullptr, B, kc, logits, s));
+  POP_TRY(decode_body(m, w, tokens, pos, nullptr, B, kc, logits, s, layer_first_pos));
   m->last_launches = launch_count() - launches0;
   return POP_OK;
 }
@@ -702,7 +718,20 @@ int pop_prefill_ragged(pop_model_t* m, const pop_input_t* in, const int32_t* seq
 
 int pop_prefill_skip(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, const uint8_t* skip,
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
-  return run_prefill_skip(m, in, seq_len, batch, skip, kv_cache_out, logits_out, static_cast<cudaStream_t>(stream));
+  return run_prefill_skip(m, in, seq_len, batch, skip, 0, kv_cache_out, logits_out,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int pop_prefill_ablation(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, const uint8_t* skip,
+                         int32_t flags, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
+  return run_prefill_skip(m, in, seq_len, batch, skip, flags, kv_cache_out, logits_out,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int pop_decode_step_from(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch,
+                         const int32_t* layer_first_pos, pop_kv_cache_t* kv_cache, float* logits_out, void* stream) {
+  return run_decode(m, tokens, pos, batch, kv_cache, logits_out, static_cast<cudaStream_t>(stream),
+                    layer_first_pos);
 }
 
 int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,

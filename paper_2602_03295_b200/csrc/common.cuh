@@ -194,6 +194,8 @@ struct DecAttnArgs {
   float* partial;                            // [batch][n_q][splits][hd + 2] fp32 scratch
   bf16* out; int64_t ldo;
   int batch, n_q, n_kv, head_dim, kv_len, window;
+  int kv_first;                // first cache position the query may attend to (0: all; a layer whose
+                               // earlier rows were never generated)
   const int32_t* cu_seqlens;   // ragged: sequence b has cu[b+1] - cu[b] cache positions (kv_len = their maximum)
   const int32_t* pos_dev;      // run-time cache length - 1 (see RopeArgs::pos_dev)
   // optional [batch][n_kv] int32, all zero before the call and all zero again after it: with it the

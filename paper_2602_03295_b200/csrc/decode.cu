@@ -222,6 +222,7 @@ struct DecAttnDev {
   float* partial;                          // [B][n_q][splits][hd + 2]
   bf16* out; int64_t ldo;                  // [B][n_q*hd]
   int n_q, n_kv, kv_len, window, splits;
+  int kv_first;                            // positions before this one are never attended to
   float scale_log2;
   const int32_t* cu;                       // ragged: sequence b has cu[b+1] - cu[b] cache positions
   const int32_t* pos_dev;                  // run-time cache length - 1
@@ -328,7 +329,7 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   const int G = p.n_q / p.n_kv;   // <= DEC_MAXG
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kv_len = p.pos_dev ? *p.pos_dev + 1 : (p.cu ? p.cu[b + 1] - p.cu[b] : p.kv_len);
-  const int lo = p.window > 0 ? max(0, kv_len - p.window) : 0;
+  const int lo = max(p.window > 0 ? max(0, kv_len - p.window) : 0, min(p.kv_first, kv_len - 1));
   const int span = kv_len - lo;
   const int chunk = (span + p.splits - 1) / p.splits;
   const int j0 = lo + split * chunk;
@@ -618,6 +619,7 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.block_table = a.block_table; p.max_pages_per_seq = a.max_pages_per_seq; p.page_size = a.page_size;
   p.partial = a.partial; p.out = a.out; p.ldo = a.ldo;
   p.n_q = a.n_q; p.n_kv = a.n_kv; p.kv_len = a.kv_len; p.window = a.window;
+  p.kv_first = a.kv_first < 0 ? 0 : a.kv_first;
   p.cu = a.cu_seqlens;
   p.pos_dev = a.pos_dev;
   p.counters = reinterpret_cast<unsigned int*>(a.counters);
@@ -700,6 +702,7 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.partial = scratch;
   p.out = static_cast<bf16*>(out); p.ldo = ldo;
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
+  p.kv_first = 0;
   p.cu = nullptr;
   p.pos_dev = nullptr;
   // with a counter per (sequence, kv head) the attention kernel merges its own splits

@@ -139,6 +139,46 @@ def test_explicit_skip_sets(variant, skip, B, N):
                 assert rel_err(cache2.gather(l)[0], cache.gather(l)[0]) <= 1e-2
 
 
+@pytest.mark.parametrize("variant", ["c1", "gemma", "hd128"])
+@pytest.mark.parametrize("skip,B,N", [({3, 4}, 2, 150), ({2, 4}, 1, 129), ({4}, 3, 1)])
+@pytest.mark.parametrize("boundary,indep_kv", [(False, True), (True, False), (False, False)])
+def test_component_ablations(variant, skip, B, N, boundary, indep_kv):
+    # Sec. 4.4.1: without boundary handling, without independent KV projections, and both; then two
+    # decode steps that keep the pruned layers' attention horizon
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS[variant]
+    w = ps.SynthWeights(cfg)
+    tokens = ps.uniform_tokens(23, B, N, cfg.vocab)
+    ref = po.pop_prefill(cfg, w, tokens, None, 0, skip=skip, boundary=boundary, indep_kv=indep_kv)
+    model = build(cfg)
+    T = 2
+    cache = KVCache(cfg, B, N + T, 16, fill=float("nan"))
+    logits, first = model.prefill_ablation(tokens.to(DEV), None, skip, cache, boundary=boundary, indep_kv=indep_kv)
+    assert model.last_status() == 0
+    assert (first or [0] * cfg.n_layers) == ref["first_pos"]
+
+    def check(refK, refV, ref_logits, n):
+        assert not torch.isnan(logits).any()
+        assert (logits.cpu().double() - ref_logits).abs().max().item() <= LOGIT_TOL
+        for l in range(cfg.n_layers):
+            k, v = cache.gather(l, n)
+            have = ~torch.isnan(refK[l][0, :, 0, 0])                      # positions this layer holds
+            assert torch.isnan(k.float()[:, ~have]).all() and torch.isnan(v.float()[:, ~have]).all()   # untouched
+            if have.any():
+                assert rel_err(k[:, have], refK[l][:, have]) <= KV_TOL, f"K layer {l + 1}"
+                assert rel_err(v[:, have], refV[l][:, have]) <= KV_TOL, f"V layer {l + 1}"
+    check(ref["K"], ref["V"], ref["logits"], N)
+    # decode steps over that cache, teacher-forced with fixed tokens
+    K, V = ref["K"], ref["V"]
+    fp = ref["first_pos"] if not indep_kv else None
+    for t in range(T):
+        tok = ps.uniform_tokens(90 + t, B, 1, cfg.vocab)[:, 0]
+        K, V, lg = po.decode_step(cfg, w, tok, K, V, first_pos=fp)
+        model.decode_step(tok.to(torch.int32).to(DEV), N + t, cache, logits, layer_first_pos=first)
+        assert model.last_status() == 0
+        check(K, V, lg, N + t + 1)
+
+
 @pytest.mark.parametrize("variant", list(TINY_VARIANTS))
 @pytest.mark.parametrize("lens,l_keep,page", [([1, 17, 130, 64], 2, 16), ([200], 1, 64), ([129, 1, 1, 300, 5], 3, 128)])
 def test_ragged_batch(variant, lens, l_keep, page):
