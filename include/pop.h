@@ -139,6 +139,18 @@ int pop_prefill_ragged(pop_model_t* m, const pop_input_t* tokens_or_embeds, cons
 int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      const uint8_t* skip, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
+/* pop_prefill evaluated chunk by chunk over the positions: chunk_len positions of every sequence
+ * at a time through the kept layers (Eq. 1-3, attending over the cache entries the earlier chunks
+ * stored) and the pruned layers' projections (Eq. 14-15), the boundary token (Sec. 3.3) with the
+ * last chunk. By causality this is the same function as pop_prefill; what changes is the
+ * workspace: pop_workspace_bytes(m, chunk_len, batch) suffices whatever seq_len is, so prompts far
+ * beyond what a one-shot workspace allows fit (seq_len <= 2^24). Inputs, outputs and errors as
+ * pop_prefill; chunk_len >= 1 (a multiple of 128 keeps the attention tiles full; larger than
+ * seq_len means one chunk). */
+int pop_prefill_chunked(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
+                        int32_t L_keep, int32_t chunk_len, pop_kv_cache_t* kv_cache_out, float* logits_out,
+                        void* stream);
+
 /* The two component ablations of the paper's Sec. 4.4.1 ("Effectiveness of Design Choices") on top
  * of pop_prefill_skip; flags is a combination of
  *   POP_NO_BOUNDARY  "w/o Boundary Handling": the last prompt token is processed by the pruned

@@ -67,6 +67,8 @@ SIGNATURES = {
                                      _P, _P]),
     "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
                                    _P]),
+    "pop_prefill_chunked": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, _I32, _I32, C.POINTER(pop_kv_cache_t),
+                                      _P, _P]),
     "pop_prefill_ablation": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, _I32,
                                        C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
@@ -444,6 +446,19 @@ class PopModel:
         code = self.lib.dll.pop_prefill_skip(self.handle, C.byref(inp), N, B, mask, C.byref(kc), logits.data_ptr(),
                                              _stream_ptr(stream))
         self.lib.check(code, "pop_prefill_skip")
+        return logits
+
+    def prefill_chunked(self, tokens, embeds, l_keep: int, chunk_len: int, cache: KVCache,
+                        logits: Optional[torch.Tensor] = None, stream=None):
+        """pop_prefill_chunked: pop_prefill in chunks of chunk_len positions (workspace for one chunk)."""
+        B, N = tokens.shape
+        self.ensure_workspace(min(chunk_len, N), B)
+        if logits is None:
+            logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        inp, kc = self._input(tokens, embeds), cache.struct()
+        code = self.lib.dll.pop_prefill_chunked(self.handle, C.byref(inp), N, B, l_keep, chunk_len, C.byref(kc),
+                                                logits.data_ptr(), _stream_ptr(stream))
+        self.lib.check(code, "pop_prefill_chunked")
         return logits
 
     def prefill_ablation(self, tokens, embeds, skip, cache: KVCache, boundary: bool = True, indep_kv: bool = True,

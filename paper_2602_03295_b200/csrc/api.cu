@@ -154,8 +154,10 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
 // one full decoder layer (paper Eq. 1-3) on all M = B*N rows of the residual stream
 // Ragged batches: `cu` (device prefix sums, B + 1 entries) and `rows` (total packed rows) replace the
 // uniform B x N layout; N is then the longest sequence.
+// Chunked prefill: the N rows of every sequence are its positions pos0 .. pos0 + N - 1 (the cache
+// already holds positions < pos0 of this layer; w.rope holds the rotary rows of these N positions).
 int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_kv_cache_t* kc, cudaStream_t s,
-               const int32_t* cu = nullptr, int rows = 0) {
+               const int32_t* cu = nullptr, int rows = 0, int pos0 = 0) {
   const pop_config_t& c = m->cfg;
   const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -168,8 +170,9 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   r.page_size = kc->page_size;
   r.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
-  r.table = w.rope; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
-  r.rows = M; r.rows_per_seq = N; r.rows_written = N; r.pos0 = 0; r.groups = 1; r.eps = c.rms_eps;
+  // the epilogue indexes the table by absolute position: hand it the address row 0 would have
+  r.table = w.rope - (int64_t)pos0 * (c.head_dim / 2); r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
+  r.rows = M; r.rows_per_seq = N; r.rows_written = N; r.pos0 = pos0; r.groups = 1; r.eps = c.rms_eps;
   r.cu_seqlens = cu; r.batch = B; r.skip_last = 0;
   GemmArgs g{};
   g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
@@ -180,7 +183,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   a.k_pool = (const bf16*)kc->k_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.v_pool = (const bf16*)kc->v_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.block_table = kc->block_table; a.out = w.ao; a.ldo = m->q_dim;
-  a.batch = B; a.seq_len = N; a.q_pos0 = 0; a.kv_len = N; a.cu_seqlens = cu; a.total_rows = cu ? M : 0;
+  a.batch = B; a.seq_len = N; a.q_pos0 = pos0; a.kv_len = pos0 + N; a.cu_seqlens = cu; a.total_rows = cu ? M : 0;
   a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim;
   a.page_size = kc->page_size; a.num_pages = kc->num_pages; a.max_pages_per_seq = kc->max_pages_per_seq;
   a.window = layer_window(c, l);
@@ -221,7 +224,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
 // Independent K/V projections of pruned layers l0..l0+n-1 (paper Eq. 14) from the state H held in
 // w.x, for positions 0..N-2 of every sequence; the state itself is left unchanged (Eq. 15).
 int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, const pop_kv_cache_t* kc,
-              cudaStream_t s, const int32_t* cu = nullptr, int rows = 0, bool write_last = false) {
+              cudaStream_t s, const int32_t* cu = nullptr, int rows = 0, bool write_last = false, int pos0 = 0) {
   const pop_config_t& c = m->cfg;
   const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
@@ -235,8 +238,8 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   r.q_gain = nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l0, m->lo.k_norm) : nullptr;
   r.gain_group_stride = (int64_t)(m->layer_stride / 4);
-  r.table = w.rope; r.n_q = 0; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
-  r.rows = M; r.rows_per_seq = N; r.rows_written = write_last ? N : N - 1; r.pos0 = 0; r.groups = n;
+  r.table = w.rope - (int64_t)pos0 * (c.head_dim / 2); r.n_q = 0; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
+  r.rows = M; r.rows_per_seq = N; r.rows_written = write_last ? N : N - 1; r.pos0 = pos0; r.groups = n;
   r.eps = c.rms_eps;
   r.cu_seqlens = cu; r.batch = B; r.skip_last = write_last ? 0 : 1;
   // ONE batched GEMM over the pruned layers (the layer is the batch dimension of both operands);
@@ -347,6 +350,60 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
   }
   // final norm (kept in fp32) and output head on the last prompt position
+  POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
+                         true, s));
+  GemvArgs v{};
+  v.x = w.hb32; v.ldx = d; v.x_f32 = true; v.w = (const bf16*)(m->arena + m->off_lm_head); v.ldw = d;
+  v.out = logits; v.ldo = c.vocab; v.B = B; v.N = c.vocab; v.K = d; v.mode = 0;
+  POP_TRY(launch_gemv(v, s));
+  m->last_launches = launch_count() - launches0;
+  return POP_OK;
+}
+
+// pop_prefill evaluated chunk by chunk over the positions (workspace for chunk_len rows per sequence
+// instead of N): by causality, positions p0 .. p0+n-1 of a kept layer need the layer's cache entries
+// of positions < p0 (already stored by the earlier chunks, Eq. 3) and nothing of later positions;
+// Eq. 14 is per position. The last chunk carries the boundary token exactly as pop_prefill does.
+int run_prefill_chunked(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, int C, pop_kv_cache_t* kc,
+                        float* logits, cudaStream_t s) {
+  if (!m || !in || !in->tokens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
+    return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (N < 1 || B < 1 || C < 1 || L_keep < 1 || L_keep > c.n_layers) return POP_E_INVALID;
+  if (C > N) C = N;
+  if ((int64_t)C * B > (int64_t)1 << 24 || N > (1 << 24)) return POP_E_INVALID;
+  if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(N, kc->page_size) > kc->max_pages_per_seq) return POP_E_NOSPACE;
+  if ((int64_t)ceil_div(N, kc->page_size) * B > kc->num_pages) return POP_E_NOSPACE;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, C, B);
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  if (cudaMemsetAsync(w.dec_ctr, 0, (size_t)B * m->cfg.n_kv_heads * 4, s) != cudaSuccess) return POP_E_CUDA;
+  const int64_t launches0 = launch_count();
+  const int d = c.d_model;
+  const bf16* table = (const bf16*)(m->arena + m->off_embed);
+  for (int p0 = 0; p0 < N; p0 += C) {
+    const int n = std::min(C, N - p0);
+    const bool last = p0 + n == N;
+    POP_TRY(launch_rope_table(w.rope, n, c.head_dim, c.rope_theta, s, p0));
+    for (int b = 0; b < B; ++b) {
+      const int64_t row0 = (int64_t)b * N + p0;
+      POP_TRY(launch_embed(in->tokens + row0, table, in->embeds ? (const bf16*)in->embeds + row0 * d : nullptr,
+                           w.x + (int64_t)b * n * d, n, d, c.vocab, s));
+    }
+    for (int l = 1; l <= L_keep; ++l) POP_TRY(full_layer(m, w, l, n, B, kc, s, nullptr, 0, p0));
+    if (L_keep < c.n_layers && (!last || n > 1)) {
+      // every position but the boundary token (the last row of the last chunk) gets its Eq. 14 entries
+      for (int l0 = L_keep + 1; l0 <= c.n_layers; l0 += kMaxPrunedChunk) {
+        const int np = std::min(kMaxPrunedChunk, c.n_layers - l0 + 1);
+        POP_TRY(pruned_kv(m, w, l0, np, n, B, kc, s, nullptr, 0, !last, p0));
+      }
+    }
+    if (last) {
+      POP_TRY(launch_gather_rows(w.x, w.xb, B, d, n, n - 1, s));
+      for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, p0, s));
+    }
+  }
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};
@@ -720,6 +777,12 @@ int pop_prefill_skip(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
   return run_prefill_skip(m, in, seq_len, batch, skip, 0, kv_cache_out, logits_out,
                           static_cast<cudaStream_t>(stream));
+}
+
+int pop_prefill_chunked(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, int32_t L_keep,
+                        int32_t chunk_len, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream) {
+  return run_prefill_chunked(m, in, seq_len, batch, L_keep, chunk_len, kv_cache_out, logits_out,
+                             static_cast<cudaStream_t>(stream));
 }
 
 int pop_prefill_ablation(pop_model_t* m, const pop_input_t* in, int32_t seq_len, int32_t batch, const uint8_t* skip,

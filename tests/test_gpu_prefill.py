@@ -115,6 +115,47 @@ def test_embedding_rows_as_input():
     check_against(ref, logits, cache, cfg)
 
 
+@pytest.mark.parametrize("variant", list(TINY_VARIANTS))
+@pytest.mark.parametrize("B,N,chunk,l_keep", [(2, 300, 128, 2), (1, 257, 100, 3), (3, 130, 400, 1), (2, 70, 37, 4),
+                                             (1, 129, 128, 2)])
+def test_chunked_prefill(variant, B, N, chunk, l_keep):
+    # the same function as pop_prefill, evaluated chunk_len positions at a time with a workspace for one
+    # chunk: ragged last chunk, a last chunk of one row (the boundary token alone), one chunk for all
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS[variant]
+    l_keep = min(l_keep, cfg.n_layers)
+    tokens = ps.uniform_tokens(31, B, N, cfg.vocab)
+    ref = po.pop_prefill(cfg, ps.SynthWeights(cfg), tokens, None, l_keep)
+    model = build(cfg)
+    cache = KVCache(cfg, B, N, 16, fill=float("nan"))
+    logits = model.prefill_chunked(tokens.to(DEV), None, l_keep, chunk, cache)
+    assert model.last_status() == 0
+    check_against(ref, logits, cache, cfg)
+    # and it agrees with the one-shot call to kernel rounding
+    cache1 = KVCache(cfg, B, N, 16, fill=float("nan"))
+    logits1 = model.prefill(tokens.to(DEV), None, l_keep, cache1)
+    assert (logits1 - logits).abs().max().item() <= 1e-2
+    for l in range(cfg.n_layers):
+        assert rel_err(cache1.gather(l)[0], cache.gather(l)[0]) <= 1e-2
+
+
+def test_chunked_prefill_with_embedding_rows_and_a_small_workspace():
+    from paper_2602_03295_b200.binding import KVCache
+    cfg = TINY_VARIANTS["qknorm"]
+    wl = ps.Workload("t", cfg, 2, 200, 2, n_visual=150)
+    tokens, embeds = ps.make_prompt(wl, 21)
+    ref = po.pop_prefill(cfg, ps.SynthWeights(cfg), tokens, embeds, wl.l_keep)
+    model = build(cfg)
+    cache = KVCache(cfg, 2, 200, 32, fill=float("nan"))
+    logits = model.prefill_chunked(tokens.to(DEV), embeds.to(DEV), wl.l_keep, 64, cache)
+    assert model.last_status() == 0
+    check_against(ref, logits, cache, cfg)
+    # the workspace really is the chunk's: far smaller than the one-shot call would need
+    need_chunk = model.lib.dll.pop_workspace_bytes(model.handle, 64, 2)
+    need_full = model.lib.dll.pop_workspace_bytes(model.handle, 200, 2)
+    assert model.ws.numel() <= need_chunk + 1024 < need_full
+
+
 @pytest.mark.parametrize("variant,skip", [("c1", {1}), ("qknorm", {2, 4}), ("gemma", {1, 3, 5}), ("hd128", {3, 4}),
                                           ("hd256", set()), ("gemma", {1, 2, 3, 4, 5})])
 @pytest.mark.parametrize("B,N", [(1, 1), (2, 70)])
