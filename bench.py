@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="config-5 sweep on the workload's model shape: prompt length x batch x L_keep/L, one "
                          "JSON line per point (POP vs full-depth prefill, tokens/s, TTFT, path TFLOP/s)")
+    ap.add_argument("--chunked", action="store_true",
+                    help="long prompts through pop_prefill_chunked (one JSON line per point) instead of the default run")
     ap.add_argument("--kernel", default="", choices=[""] + KERNELS,
                     help="time ONE kernel of the path alone, at the workload's per-layer shape, through its "
                          "kernel-level C-ABI entry point (a small case for profiling)")
@@ -660,10 +662,56 @@ def run_sweep(a, wl0):
             del cache, tokens, logits
 
 
+def run_chunked(a, wl0):
+    """Long prompts on the workload's model, batch 1, L_keep = 3L/4: the one-shot call where its
+    workspace is reasonable, and pop_prefill_chunked at several chunk lengths up to 131072 positions.
+    Weights stream on every call and every chunk (far larger than L2)."""
+    from oracle import pop_oracle as po   # FLOP model only
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = wl0.model
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+    peaks = load_peaks()
+    lk = cfg.n_layers * 3 // 4
+    for n, chunk in ((32768, 0), (32768, 16384), (32768, 8192), (32768, 2048), (131072, 8192)):
+        tokens = ps.uniform_tokens(ps.DEFAULT_SEED + 1, 1, n, cfg.vocab).to(dev)
+        cache = KVCache(cfg, 1, n, a.page_size, device=dev)
+        logits = torch.empty(1, cfg.vocab, dtype=torch.float32, device=dev)
+        model.ws = None                                   # size the workspace for this point alone
+
+        def step():
+            if chunk:
+                model.prefill_chunked(tokens, None, lk, chunk, cache, logits)
+            else:
+                model.prefill(tokens, None, lk, cache, logits)
+        for _ in range(3 if n <= 32768 else 1):
+            step()
+        torch.cuda.synchronize()
+        steps = a.steps if n <= 32768 else max(1, min(a.steps, 2))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        assert model.last_status() == 0
+        flops = po.prefill_flops(cfg, 1, n, lk)
+        print(json.dumps({"chunked": wl0.key, "seq_len": n, "chunk_len": chunk or None, "l_keep": lk, "ttft_ms": ms,
+                          "tokens_per_s": n / (ms * 1e-3), "path_tflops": flops / (ms * 1e-3) / 1e12,
+                          "frac_of_measured_burst_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                          "workspace_mb": model.ws.numel() / 2 ** 20,
+                          "kv_cache_mb": 2 * cache.k.numel() * 2 / 2 ** 20, "steps": steps}), flush=True)
+        del cache, tokens, logits
+
+
 def main():
     a = parse_args()
     wl = resolve_workload(a)
-    if a.sweep:
+    if a.chunked:
+        run_chunked(a, wl)
+    elif a.sweep:
         run_sweep(a, wl)
     elif a.kernel:
         run_kernel(a, wl)
