@@ -60,6 +60,49 @@ def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
     return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
 
 
+# ---------------------------------------------------------------------------------------
+# FP8 operands (stage-aware quantisation is the paper's stated future direction, Sec. 6; the paper
+# fixes no format: this is the OCP E4M3 format with one scale per activation row and one per weight
+# matrix, the reading stated in the design notes)
+# ---------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_round(x: torch.Tensor) -> torch.Tensor:
+    """Nearest value of the OCP FP8 E4M3 format (1 sign, 4 exponent bits with bias 7, 3 mantissa
+    bits; no infinities; largest finite value 448; subnormals are multiples of 2^-9), ties to the
+    even mantissa, magnitudes above 448 saturate. Returned in float64."""
+    x = x.double()
+    a = x.abs().clamp(max=E4M3_MAX)
+    _, ex = torch.frexp(a)                       # a = m * 2^ex, m in [0.5, 1)
+    e = (ex - 1).clamp(min=-6)                   # exponent of the binade; subnormals share the lowest
+    quantum = torch.pow(torch.tensor(2.0, dtype=torch.float64), (e - 3).double())
+    q = torch.round(a / quantum) * quantum       # torch.round: halves to even
+    return torch.where(a == 0, torch.zeros_like(a), q) * torch.sign(x)
+
+
+def quant_rows_e4m3(h: torch.Tensor):
+    """One scale per row: codes e4m3(h * (448 / amax_row)) and the scale amax_row / 448 that maps
+    them back (a row of zeros gets scale 1). The decision is taken in fp32 as the kernel takes it.
+    h: [T, d] -> (codes [T, d] float64 holding E4M3 values, scale [T, 1] float64)."""
+    h32 = h.to(torch.float32)
+    amax = h32.abs().amax(dim=-1, keepdim=True)
+    safe = torch.where(amax > 0, amax, torch.ones_like(amax))
+    inv = torch.tensor(E4M3_MAX, dtype=torch.float32) / safe
+    scale = torch.where(amax > 0, amax / torch.tensor(E4M3_MAX, dtype=torch.float32), torch.ones_like(amax))
+    return e4m3_round(h32 * inv), scale.double()
+
+
+def quant_tensors_e4m3(ws):
+    """One scale for a group of weight matrices that the kernel stores as one fused matrix:
+    codes e4m3(w * (448 / amax)) for every matrix and the common scale amax / 448."""
+    amax = max(float(w.to(torch.float32).abs().max()) for w in ws)
+    amax32 = torch.tensor(amax if amax > 0 else E4M3_MAX, dtype=torch.float32)
+    inv = torch.tensor(E4M3_MAX, dtype=torch.float32) / amax32
+    scale = float(amax32 / torch.tensor(E4M3_MAX, dtype=torch.float32))
+    return [e4m3_round(w.to(torch.float32) * inv) for w in ws], scale
+
+
 def rmsnorm(x: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
     """LN(.) of Eq. 2 for the RMSNorm models evaluated in Sec. 4: x * g / sqrt(mean(x^2) + eps)."""
     ms = x.pow(2).mean(dim=-1, keepdim=True)

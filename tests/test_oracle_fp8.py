@@ -1,0 +1,62 @@
+"""Pins of the oracle's FP8 (E4M3) rounding and scaling: against the format's definition enumerated
+value by value, against torch's own float8_e4m3fn cast (a library routine the oracle does not call),
+and closed forms."""
+import itertools
+
+import torch
+
+from oracle import pop_oracle as po
+
+
+def _all_e4m3_values():
+    # every finite non-negative value from the format's definition: exponent field E (0..15), mantissa M (0..7);
+    # E = 0: M/8 * 2^-6; else (1 + M/8) * 2^(E-7); the pattern E = 15, M = 7 is NaN
+    vals = []
+    for E, M in itertools.product(range(16), range(8)):
+        if E == 15 and M == 7:
+            continue
+        vals.append(M / 8 * 2.0 ** -6 if E == 0 else (1 + M / 8) * 2.0 ** (E - 7))
+    return sorted(vals)
+
+
+def test_representable_values_are_fixed_points_and_the_largest_is_448():
+    v = torch.tensor(_all_e4m3_values(), dtype=torch.float64)
+    assert v.max().item() == 448.0 and v[1].item() == 2.0 ** -9 and len(v) == 127
+    assert torch.equal(po.e4m3_round(v), v)
+    assert torch.equal(po.e4m3_round(-v), -v)
+
+
+def test_rounding_goes_to_the_nearest_value_ties_to_even():
+    v = _all_e4m3_values()
+    for lo, hi in zip(v[:-1], v[1:]):
+        mid = (lo + hi) / 2
+        x = torch.tensor([lo + 0.49 * (hi - lo), lo + 0.51 * (hi - lo), mid], dtype=torch.float64)
+        r = po.e4m3_round(x)
+        assert r[0].item() == lo and r[1].item() == hi
+        # the tie goes to the value whose mantissa is even: consecutive values alternate parity
+        even = lo if v.index(lo) % 2 == 0 else hi
+        assert r[2].item() == even, (lo, hi)
+    assert po.e4m3_round(torch.tensor([1e9, -1e9, 460.0, 0.0, 2.0 ** -11])).tolist() == [448.0, -448.0, 448.0, 0.0, 0.0]
+
+
+def test_agrees_with_the_library_cast():
+    g = torch.Generator().manual_seed(3)
+    x = torch.cat([torch.randn(20000, generator=g) * s for s in (1e-3, 0.05, 1.0, 30.0, 200.0)])
+    x = x.clamp(-448, 448)                                    # the library cast does not saturate
+    lib = x.to(torch.float8_e4m3fn).to(torch.float64)
+    assert torch.equal(po.e4m3_round(x), lib)
+
+
+def test_row_and_tensor_scales():
+    g = torch.Generator().manual_seed(4)
+    h = torch.randn(5, 64, generator=g) * torch.tensor([[1e-3], [1.0], [50.0], [0.0], [7.0]])
+    q, s = po.quant_rows_e4m3(h)
+    assert s[3].item() == 1.0 and (q[3] == 0).all()
+    for r in (0, 1, 2, 4):
+        assert q[r].abs().max().item() == 448.0               # the row's largest magnitude maps to the format's
+        # dequantised values are within half a quantum (2^-4 relative for normal numbers) of the input
+        assert ((q[r] * s[r] - h[r].double()).abs() <= h[r].abs().double() * 2.0 ** -4 + s[r] * 2.0 ** -10).all()
+    ws = [torch.randn(8, 16, generator=g) * 0.02, torch.randn(4, 16, generator=g) * 0.05]
+    qs, sc = po.quant_tensors_e4m3(ws)
+    assert max(float(t.abs().max()) for t in qs) == 448.0
+    assert abs(sc - max(float(w.abs().max()) for w in ws) / 448.0) < 1e-9
