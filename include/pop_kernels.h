@@ -68,6 +68,25 @@ int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* 
                     int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t page_size, int32_t num_pages,
                     int32_t max_pages_per_seq, int32_t window, void* stream);
 
+/* FP8 operands for the projections of paper Eq. 1-2. The paper fixes no number format and names
+ * stage-aware quantisation as a direction (Sec. 6); this is the OCP E4M3 format (1-4-3 bits, bias 7,
+ * largest value 448, no infinities), round to nearest even, saturating, with one scale per
+ * activation row and one per weight matrix: value = code * scale.
+ *
+ * pop_k_rmsnorm_e4m3: y = LN(x[r]) as pop_k_rmsnorm computes it in fp32; out[r][:] = e4m3(y * 448 /
+ *   max|y|) as bytes (row stride ldo bytes, a multiple of 16), scale[r] = max|y| / 448 (1 for a zero row).
+ * pop_k_quantize_e4m3: the same for a whole bf16 array of n elements (n a multiple of 8) with one
+ *   scale: out[i] = e4m3(w[i] * 448 / max|w|), *scale = max|w| / 448. scratch4: 4 device bytes.
+ * pop_k_gemm_e4m3: D[m][n] = a_scale[m] * *b_scale * sum_k A[m][k] * B[n][k] on the codes (fp32
+ *   accumulation on the tensor cores, kind f8f6f4), then epilogue 0, 1 or 3 of pop_k_gemm. lda,
+ *   ldb, K count codes and are multiples of 16; pointers 16-byte aligned; a_scale, b_scale device fp32. */
+int pop_k_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, void* out, int64_t ldo, float* scale,
+                       int32_t rows, int32_t d, float eps, void* stream);
+int pop_k_quantize_e4m3(const void* w, int64_t n, void* out, float* scale, void* scratch4, void* stream);
+int pop_k_gemm_e4m3(const void* A, int64_t lda, const float* a_scale, const void* B, int64_t ldb,
+                    const float* b_scale, void* out, int64_t ldo, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                    int32_t act, int32_t n_valid, void* stream);
+
 /* RMSNorm, the LN of paper Eq. 2 / Eq. 14: out[g][r][:] = x[r][:] * rsqrt(mean(x[r]^2)+eps) * gain[g][:].
  * x fp32 [rows][ldx]; gain fp32, group g at gain + g*gain_stride; out bf16 (out_f32 = 0) or fp32,
  * group stride out_gs elements. */

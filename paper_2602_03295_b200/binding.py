@@ -80,6 +80,9 @@ SIGNATURES = {
     "pop_strerror": (C.c_char_p, [C.c_int]),
     "pop_k_gemm": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _I32, _I32, _I32,
                              _I32, _P]),
+    "pop_k_gemm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
+    "pop_k_rmsnorm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _I32, _I32, _F, _P]),
+    "pop_k_quantize_e4m3": (C.c_int, [_P, _I64, _P, _P, _P, _P]),
     "pop_k_gemm_norm": (C.c_int, [_P, _I64, _P, _I64, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P, _I64, _P, _P, _I32,
                                   _P, _I32, _I32, _I32, _F, _P]),
     "pop_k_gemm_qkv_rope": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _P, _I64, _P, _P, _I64, _I32,
@@ -171,6 +174,37 @@ class PopLibrary:
         self.check(code, "pop_k_gemm")
         return out
 
+
+    def rmsnorm_e4m3(self, x, gain, eps, stream=None):
+        """pop_k_rmsnorm_e4m3: returns (codes uint8 [rows, d], scale fp32 [rows])."""
+        rows, d = x.shape
+        out = torch.empty(rows, d, dtype=torch.uint8, device=x.device)
+        scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+        code = self.dll.pop_k_rmsnorm_e4m3(x.data_ptr(), x.stride(0), gain.data_ptr(), out.data_ptr(), out.stride(0),
+                                           scale.data_ptr(), rows, d, eps, _stream_ptr(stream))
+        self.check(code, "pop_k_rmsnorm_e4m3")
+        return out, scale
+
+    def quantize_e4m3(self, w, stream=None):
+        """pop_k_quantize_e4m3 of a contiguous bf16 tensor: returns (codes uint8 of w's shape, scale fp32 [1])."""
+        assert w.is_contiguous() and w.dtype == torch.bfloat16
+        out = torch.empty(w.shape, dtype=torch.uint8, device=w.device)
+        scale = torch.empty(1, dtype=torch.float32, device=w.device)
+        scratch = torch.empty(1, dtype=torch.int32, device=w.device)
+        code = self.dll.pop_k_quantize_e4m3(w.data_ptr(), w.numel(), out.data_ptr(), scale.data_ptr(),
+                                            scratch.data_ptr(), _stream_ptr(stream))
+        self.check(code, "pop_k_quantize_e4m3")
+        return out, scale
+
+    def gemm_e4m3(self, A, a_scale, B, b_scale, out, epilogue=1, act=0, n_valid=0, stream=None):
+        """pop_k_gemm_e4m3: A [M,K], B [N,K] uint8 codes; a_scale fp32 [M]; b_scale fp32 [1]."""
+        M, K = A.shape
+        N = B.shape[0]
+        code = self.dll.pop_k_gemm_e4m3(A.data_ptr(), A.stride(0), a_scale.data_ptr(), B.data_ptr(), B.stride(0),
+                                        b_scale.data_ptr(), out.data_ptr(), out.stride(0), M, N, K, epilogue, act,
+                                        n_valid, _stream_ptr(stream))
+        self.check(code, "pop_k_gemm_e4m3")
+        return out
 
     def gemm_norm(self, A, B, out, epilogue, act=0, n_valid=0, hn_out=None, gain_next=None, ss_out=None,
                   ss_in=None, norm_d=0, norm_eps=0.0, stream=None):

@@ -18,6 +18,31 @@ int pop_k_gemm(const void* A, int64_t lda, int64_t a_bs, const void* B, int64_t 
   return launch_gemm(a, static_cast<cudaStream_t>(stream));
 }
 
+int pop_k_gemm_e4m3(const void* A, int64_t lda, const float* a_scale, const void* B, int64_t ldb,
+                    const float* b_scale, void* out, int64_t ldo, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                    int32_t act, int32_t n_valid, void* stream) {
+  GemmArgs a{};
+  a.A = static_cast<const bf16*>(A); a.lda = lda;
+  a.B = static_cast<const bf16*>(B); a.ldb = ldb;
+  a.out = out; a.ldo = ldo;
+  a.M = M; a.N = N; a.K = K; a.batch = 1;
+  a.epilogue = epilogue; a.act = act; a.n_valid = n_valid;
+  a.fp8 = true; a.a_scale = a_scale; a.b_scale = b_scale;
+  if (epilogue != EPI_STORE_BF16 && epilogue != EPI_STORE_F32 && epilogue != EPI_GATED_BF16) return POP_E_INVALID;
+  return launch_gemm(a, static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, void* out, int64_t ldo, float* scale,
+                       int32_t rows, int32_t d, float eps, void* stream) {
+  return launch_rmsnorm_e4m3(x, ldx, gain, static_cast<uint8_t*>(out), ldo, scale, rows, d, eps,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_quantize_e4m3(const void* w, int64_t n, void* out, float* scale, void* scratch4, void* stream) {
+  return launch_quantize_weights_e4m3(static_cast<const bf16*>(w), n, static_cast<uint8_t*>(out), scale,
+                                      static_cast<unsigned int*>(scratch4), static_cast<cudaStream_t>(stream));
+}
+
 int pop_k_gemm_norm(const void* A, int64_t lda, const void* B, int64_t ldb, void* out, int64_t ldo, int32_t M,
                     int32_t N, int32_t K, int32_t epilogue, int32_t act, int32_t n_valid, void* hn_out, int64_t ld_hn,
                     const float* gain_next, float* ss_out, int32_t ss_ld, const float* ss_in, int32_t ss_cnt,

@@ -72,6 +72,9 @@ int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_
                       uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1);
 // 3-D fp32 tensor [dim2][dim1][dim0], 128-byte swizzle, box = [1][box1][32] (32 floats = 128 bytes): the
 // GEMM's output tiles
+// 3-D byte tensor (FP8 operands), 128-byte swizzle, box = [1][box1][128]
+int make_tmap_u8_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                    uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box1);
 int make_tmap_f32_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
                      uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box1);
 // rank-`rank` (3..5) bf16 tensor, dims/strides/box given innermost first (strides in elements, for
@@ -112,6 +115,10 @@ struct GemmArgs {
   // rsqrt(sum_i ss_in[row * ss_in_ld + i] / norm_d + norm_eps) before its own epilogue.
   bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
   const float* ss_in; int ss_cnt; int ss_in_ld; int norm_d; float norm_eps;
+  // FP8 operands (batch == 1; store, gated and QKV epilogues): A and B point at E4M3 codes, lda / ldb /
+  // K count codes (multiples of 16), and the accumulator is scaled by a_scale[row] * *b_scale (device)
+  // before the epilogue proper
+  bool fp8; const float* a_scale; const float* b_scale;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t stream);
 
@@ -178,6 +185,14 @@ int launch_argmax(const float* logits, int64_t ld, int vocab, int batch, int32_t
 int launch_set_counters(int32_t* counters, int a, int b, cudaStream_t s);
 int launch_bump_counters(int32_t* counters, cudaStream_t s);
 int launch_gather_last_rows(const float* src, float* dst, int batch, int d, const int32_t* cu, cudaStream_t s);
+
+// ------------------------------------------------------------------------------------ FP8 operands
+// out[row][:] = e4m3(LN(x[row]) * 448 / amax_row), scale[row] = amax_row / 448 (LN = RMSNorm with `gain`)
+int launch_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, uint8_t* out, int64_t ldo, float* scale,
+                        int rows, int d, float eps, cudaStream_t s);
+// out[i] = e4m3(w[i] * 448 / amax), *scale = amax / 448 over the n elements; scratch: 4 bytes
+int launch_quantize_weights_e4m3(const bf16* w, int64_t n, uint8_t* out, float* scale, unsigned int* scratch,
+                                 cudaStream_t s);
 
 // ------------------------------------------------------------------------------------ boundary path
 struct GemvArgs {

@@ -60,6 +60,7 @@ struct GemmDev {
   int act, n_valid;
   bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
   const float* ss_in; int ss_cnt; int ss_in_ld; float inv_d; float eps_in;
+  const float* a_scale; const float* b_scale;      // FP8 operands: accumulator scale a_scale[row] * *b_scale
 };
 
 __device__ __forceinline__ void tile_coords(const GemmDev& p, int t, int& g, int& m, int& n) {
@@ -209,7 +210,9 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
   }
 }
 
-template <int EPI, int HD>
+// FP8: the operands are E4M3 codes, a k-block of 128 bytes holds 128 of them (64 bf16 otherwise) and
+// one MMA instruction covers 32 (16): the smem tiles, descriptors and their 32-byte steps are the same.
+template <int EPI, int HD, bool FP8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmO, const GemmDev p,
@@ -219,7 +222,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
-  const int k_blocks = (p.K + BK - 1) / BK;
+  constexpr int BKE = FP8 ? 2 * BK : BK;          // operand elements per k-block
+  const int k_blocks = (p.K + BKE - 1) / BKE;
 
   if (status_raised(status, &s.raised)) return;
   if (threadIdx.x == 0) {
@@ -260,8 +264,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           mbar_expect_tx(&s.full[stage], A_BYTES + B_BYTES);
-          tma_load_3d(s.a[stage], &tmA, &s.full[stage], kb * BK, m * BM, g);
-          tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BK, n * BN, g);
+          tma_load_3d(s.a[stage], &tmA, &s.full[stage], kb * BKE, m * BM, g);
+          tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BKE, n * BN, g);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1;
@@ -274,7 +278,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // The whole warp walks this role with identical values; one elected lane issues.
     {
       const uint32_t leader = elect_one();
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, 0, 0);
+      constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(BM, BN) : umma_idesc_bf16(BM, BN, 0, 0);
       const uint64_t a_desc0 = umma_smem_desc(smem_u32(s.a[0]), 16, 1024);
       const uint64_t b_desc0 = umma_smem_desc(smem_u32(s.b[0]), 16, 1024);
       int stage = 0;
@@ -301,9 +305,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint64_t ad0 = a_desc0 + uint64_t(stage * (A_BYTES >> 4));
           const uint64_t bd0 = b_desc0 + uint64_t(stage * (B_BYTES >> 4));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            umma_bf16_ss_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
-                           (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < BK / 16; ++k) {
+            if constexpr (FP8)
+              umma_e4m3_ss_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
+                             (kb | k) != 0 ? 1u : 0u);
+            else
+              umma_bf16_ss_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
+                             (kb | k) != 0 ? 1u : 0u);
+          }
           umma_commit_w(leader, &s.empty[stage]);
           if (++stage == STAGES) {
             stage = 0;
@@ -345,6 +354,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int i = 0; i < p.ss_cnt; ++i) sum += p.ss_in[(int64_t)row * p.ss_in_ld + i];
         rs = rsqrtf(sum * p.inv_d + p.eps_in);
       }
+      if (FP8 && row_ok) rs = p.a_scale[row] * *p.b_scale;     // codes -> values: row scale x matrix scale
       if (EPI == EPI_QKV_ROPE) {
         qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok, rs);
       } else if (EPI == EPI_GATED_BF16) {
@@ -483,20 +493,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
-template <int EPI, int HD = 0>
+template <int EPI, int HD = 0, bool FP8 = false>
 int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p, int grid,
                cudaStream_t stream) {
   const size_t smem = sizeof(GemmSmem) + 1024;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(gemm_kernel<EPI, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_kernel<EPI, HD, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
       return POP_E_CUDA;
     configured = true;
   }
   int* status = status_word();
   if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
-  gemm_kernel<EPI, HD><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
+  gemm_kernel<EPI, HD, FP8><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }
@@ -524,12 +535,23 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     if (a.N % 4 || a.ldo % 4) return POP_E_INVALID;
   }
   CUtensorMap ta, tb;
-  int rc = make_tmap_bf16_3d(&ta, a.A, a.K, a.M, a.batch, a.lda, a.a_batch_stride ? a.a_batch_stride : a.lda * a.M,
-                             BK, BM);
-  if (rc) return rc;
-  rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
-                         BN);
-  if (rc) return rc;
+  int rc;
+  if (a.fp8) {
+    if (a.batch != 1 || !a.a_scale || !a.b_scale || a.K % 16 || a.lda % 16 || a.ldb % 16 || a.hn_out || a.ss_in ||
+        a.epilogue == EPI_ADD_F32)
+      return POP_E_INVALID;
+    rc = make_tmap_u8_3d(&ta, a.A, a.K, a.M, 1, a.lda, (uint64_t)a.lda * a.M, BM);
+    if (rc) return rc;
+    rc = make_tmap_u8_3d(&tb, a.B, a.K, a.N, 1, a.ldb, (uint64_t)a.ldb * a.N, BN);
+    if (rc) return rc;
+  } else {
+    rc = make_tmap_bf16_3d(&ta, a.A, a.K, a.M, a.batch, a.lda, a.a_batch_stride ? a.a_batch_stride : a.lda * a.M,
+                           BK, BM);
+    if (rc) return rc;
+    rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
+                           BN);
+    if (rc) return rc;
+  }
   if (a.hn_out != nullptr) {
     if (a.epilogue != EPI_ADD_F32 || a.batch != 1 || !a.gain_next || !a.ss_out || a.ld_hn % 4 ||
         a.ss_ld < ceil_div(a.N, BN))
@@ -548,6 +570,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   p.ss_in = a.ss_in; p.ss_cnt = a.ss_cnt; p.ss_in_ld = a.ss_in_ld;
   p.inv_d = a.norm_d > 0 ? 1.0f / (float)a.norm_d : 0.f;
   p.eps_in = a.norm_eps;
+  p.a_scale = a.a_scale; p.b_scale = a.b_scale;
   if (a.epilogue == EPI_QKV_ROPE) {
     const RopeArgs& r = *a.rope;
     p.rope.q_out = r.q_out; p.rope.ldq = r.ldq;
@@ -576,6 +599,21 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     return POP_E_CUDA;
   const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
   const int grid = (int)(total < sms ? total : sms);
+  if (a.fp8) {
+    switch (a.epilogue) {
+      case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, stream);
+      case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, stream);
+      case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, stream);
+      case EPI_QKV_ROPE:
+        switch (a.rope->hd) {
+          case 64: return launch_epi<EPI_QKV_ROPE, 64, true>(ta, tb, to, p, grid, stream);
+          case 128: return launch_epi<EPI_QKV_ROPE, 128, true>(ta, tb, to, p, grid, stream);
+          case 256: return launch_epi<EPI_QKV_ROPE, 256, true>(ta, tb, to, p, grid, stream);
+        }
+        return POP_E_INVALID;
+    }
+    return POP_E_INVALID;
+  }
   switch (a.epilogue) {
     case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, stream);
     case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, stream);

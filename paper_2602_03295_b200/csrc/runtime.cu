@@ -125,6 +125,20 @@ int make_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_
   return r == CUDA_SUCCESS ? POP_OK : POP_E_CUDA;
 }
 
+int make_tmap_u8_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                    uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return POP_E_CUDA;
+  cuuint64_t dims[3] = {dim0, dim1, dim2};
+  cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+  cuuint32_t box[3] = {128, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? POP_OK : POP_E_CUDA;
+}
+
 int make_tmap_f32_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
                      uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box1) {
   EncodeTiledFn fn = encode_fn();
