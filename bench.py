@@ -34,7 +34,8 @@ import pop_synth as ps  # noqa: E402
 METRIC = "pop_prefill_tokens_per_s"
 UNIT = "tokens/s"
 KERNELS = ["gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down", "kvproj", "attention", "attention_local", "gemv_head",
-           "decode_attention", "decode_step", "rmsnorm", "rope_cache"]
+           "decode_attention", "decode_step", "rmsnorm", "rope_cache", "gemm_gateup_fp8", "gemm_qkvshape_fp8",
+           "rmsnorm_fp8"]
 
 
 def parse_args():
@@ -428,7 +429,7 @@ def run_kernel(a, wl):
     peaks = load_peaks()
     k = a.kernel
     bound, work, sets = "tensor", 0.0, 1
-    if k.startswith("gemm_") or k == "kvproj":
+    if (k.startswith("gemm_") and not k.endswith("_fp8")) or k == "kvproj":
         f_pad = (F + 127) // 128 * 128
         shapes = {"gemm_qkv": (1, qd + 2 * kvd, d, 1), "gemm_o": (1, d, qd, 2), "gemm_gateup": (1, 2 * f_pad, d, 3),
                   "gemm_down": (1, d, F, 2), "kvproj": (P, 2 * kvd, d, 1)}
@@ -460,6 +461,28 @@ def run_kernel(a, wl):
             def launch(i):
                 lib.gemm(A if G > 1 else A[0], B if G > 1 else B[0], out if G > 1 else out[0], epilogue=epi,
                          act=cfg.act, n_valid=F if epi == 3 else 0)
+    elif k in ("gemm_gateup_fp8", "gemm_qkvshape_fp8"):
+        # the E4M3 GEMM at the gate/up shape (gated epilogue) and at the QKV shape (plain fp32 store)
+        f_pad = (F + 127) // 128 * 128
+        N, epi = (2 * f_pad, 3) if k == "gemm_gateup_fp8" else (qd + 2 * kvd, 1)
+        K = d
+        A8, sa = lib.rmsnorm_e4m3(rnd(M, K, dtype=torch.float32), torch.ones(K, dtype=torch.float32, device=dev),
+                                  cfg.rms_eps)
+        B8, sb = lib.quantize_e4m3(rnd(N, K, std=0.02))
+        out = torch.zeros(M, F if epi == 3 else N, dtype=torch.bfloat16 if epi == 3 else torch.float32, device=dev)
+        work = 2.0 * M * N * K
+        peaks = dict(peaks, bf16_tflops=2.0 * peaks["bf16_tflops"], source=peaks["source"] + " bf16 x 2 (nominal fp8 : bf16 ratio)")
+
+        def launch(i):
+            lib.gemm_e4m3(A8, sa, B8, sb, out, epilogue=epi, act=cfg.act, n_valid=F if epi == 3 else 0)
+    elif k == "rmsnorm_fp8":
+        bound = "hbm"
+        x = rnd(M, d, dtype=torch.float32)
+        gain = torch.ones(d, dtype=torch.float32, device=dev)
+        work = 5.0 * M * d
+
+        def launch(i):
+            lib.rmsnorm_e4m3(x, gain, cfg.rms_eps)
     elif k in ("attention", "attention_local"):
         from paper_2602_03295_b200.binding import KVCache
         window = cfg.window if k == "attention_local" else 0

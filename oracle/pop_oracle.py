@@ -54,7 +54,8 @@ import torch
 # ---------------------------------------------------------------------------------------
 
 def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
-    """Round to bf16 and back in "bf16ops" mode; identity in "exact" mode."""
+    """Identity in "exact" mode; otherwise ("kernel": bf16 operands; "fp8": E4M3 operands for the QKV and
+    gate/up projections, bf16 for the rest) round to bf16 and back."""
     if precision == "exact":
         return x
     return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
@@ -180,13 +181,27 @@ def embed(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], dt
     return x
 
 
+def _qkv_fp8(cfg, weights, layer: int, x: torch.Tensor, dtype):
+    """q, k, v projections of LN(x) with E4M3 operands: one scale per row of LN(x), one for the fused
+    [W^Q; W^K; W^V] matrix; the products are exact, the scales multiply the sum."""
+    hq, sa = quant_rows_e4m3(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps))
+    (wq, wk, wv), sw = quant_tensors_e4m3([weights.get(n, layer) for n in ("wq", "wk", "wv")])
+    hq = hq.to(dtype)
+    return tuple((hq @ w.to(dtype).T) * sa.to(dtype) * sw for w in (wq, wk, wv))
+
+
 def kv_generation(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Tensor,
                   dtype, precision: str):
     """Eq. 2 (and, applied to a pruned layer's input, Eq. 14): the layer's own input norm,
     K/V projections, optional per-head K norm, RoPE on k. x: [T, d] -> k, v [T, n_kv, hd]."""
-    h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
-    k = (h @ _w(weights, "wk", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
-    v = (h @ _w(weights, "wv", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+    if precision == "fp8":
+        _, k, v = _qkv_fp8(cfg, weights, layer, x, dtype)
+        k = k.reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+        v = v.reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+    else:
+        h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
+        k = (h @ _w(weights, "wk", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+        v = (h @ _w(weights, "wv", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
     if cfg.qk_norm:
         k = rmsnorm(k, _w(weights, "k_norm", layer, dtype), cfg.rms_eps)
     k = rope(k, positions, cfg.rope_theta)
@@ -206,8 +221,11 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
     else:
         k_cur, v_cur = k_new, v_new
         k_pos0 = int(positions[0])
-    h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
-    q = (h @ _w(weights, "wq", layer, dtype).T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
+    if precision == "fp8":
+        q = _qkv_fp8(cfg, weights, layer, x, dtype)[0].reshape(-1, cfg.n_q_heads, cfg.head_dim)
+    else:
+        h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
+        q = (h @ _w(weights, "wq", layer, dtype).T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
     if cfg.qk_norm:
         q = rmsnorm(q, _w(weights, "q_norm", layer, dtype), cfg.rms_eps)
     q = _rnd(rope(q, positions, cfg.rope_theta), precision)
@@ -217,9 +235,15 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
     if cfg.post_norms:
         o = rmsnorm(o, _w(weights, "post_attn_norm", layer, dtype), cfg.rms_eps)
     y = x + o                                                           # Eq. 1, first line
-    h2 = _rnd(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps), precision)
-    gate = h2 @ _w(weights, "w_gate", layer, dtype).T
-    up = h2 @ _w(weights, "w_up", layer, dtype).T
+    if precision == "fp8":
+        h2q, sa = quant_rows_e4m3(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps))
+        (wg, wu), sw = quant_tensors_e4m3([weights.get(n, layer) for n in ("w_gate", "w_up")])
+        gate = (h2q.to(dtype) @ wg.to(dtype).T) * sa.to(dtype) * sw
+        up = (h2q.to(dtype) @ wu.to(dtype).T) * sa.to(dtype) * sw
+    else:
+        h2 = _rnd(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps), precision)
+        gate = h2 @ _w(weights, "w_gate", layer, dtype).T
+        up = h2 @ _w(weights, "w_up", layer, dtype).T
     f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w(weights, "w_down", layer, dtype).T
     if cfg.post_norms:
         f = rmsnorm(f, _w(weights, "post_ffn_norm", layer, dtype), cfg.rms_eps)
@@ -272,7 +296,7 @@ def full_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tens
 
 def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor], l_keep: int,
                 dtype=torch.float64, precision: str = "exact", skip=None, boundary: bool = True,
-                indep_kv: bool = True):
+                indep_kv: bool = True, fp8_kept: bool = False):
     """POP inference up to the first generated token, in the paper's two phases (Sec. 3.3).
 
     Phase 1, pruned prefill on x_{1:N-1}: layers 1..L_keep run in full; each layer
@@ -294,6 +318,10 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
       indep_kv=False ("w/o Indep. KV Proj."): pruned layers generate no cache entries in phase 1;
         in phase 2 (and in later decode steps) such a layer can only attend to positions >= N.
         Their K, V rows of positions 1..N-1 are returned as NaN ("absent").
+
+    fp8_kept (deep-suffix set only): every position, x_N included, passes the kept layers with
+    E4M3 operands in the QKV and gate/up projections (precision "fp8"); the pruned layers'
+    projections and x_N's pass through the deep layers use `precision`.
 
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
     H [B, N-1, d] (the state leaving the last layer of phase 1 at positions 1..N-1; for the
@@ -323,7 +351,7 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
             for l in range(1, L + 1):
                 if l not in skip:
                     x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, pos, None, None,
-                                                            dtype, precision)
+                                                            dtype, "fp8" if fp8_kept else precision)
                 elif indep_kv:
                     kc[l - 1], vc[l - 1] = kv_generation(cfg, weights, l, x, pos, dtype, precision)
                     # Eq. 15: x is handed to layer l+1 unchanged
@@ -333,8 +361,8 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
             posN = torch.tensor([N - 1])
             x = x_all[N - 1: N]
             for l in range(1, L + 1):
-                x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1],
-                                                        dtype, precision)
+                x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1], dtype,
+                                                        "fp8" if (fp8_kept and l not in skip) else precision)
             x_last = x[0]
         else:
             x_last = x[N - 1]

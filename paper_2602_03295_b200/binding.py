@@ -67,6 +67,8 @@ SIGNATURES = {
                                      _P, _P]),
     "pop_prefill_skip": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, C.POINTER(pop_kv_cache_t), _P,
                                    _P]),
+    "pop_fp8_arena_bytes": (C.c_size_t, [_P]),
+    "pop_enable_fp8": (C.c_int, [_P, _P, C.c_size_t, _P]),
     "pop_prefill_chunked": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, _I32, _I32, C.POINTER(pop_kv_cache_t),
                                       _P, _P]),
     "pop_prefill_ablation": (C.c_int, [_P, C.POINTER(pop_input_t), _I32, _I32, C.c_char_p, _I32,
@@ -481,6 +483,18 @@ class PopModel:
                                              _stream_ptr(stream))
         self.lib.check(code, "pop_prefill_skip")
         return logits
+
+    def enable_fp8(self, on: bool = True, stream=None):
+        """pop_enable_fp8: E4M3 copies of the kept layers' QKV and gate/up weights (the arena is a torch
+        tensor this object keeps); on=False goes back to bf16 operands."""
+        if not on:
+            self.lib.check(self.lib.dll.pop_enable_fp8(self.handle, None, 0, _stream_ptr(stream)), "pop_enable_fp8")
+            self.fp8_arena = None
+            return
+        need = self.lib.dll.pop_fp8_arena_bytes(self.handle)
+        self.fp8_arena = torch.empty(need + 1024, dtype=torch.uint8, device=self.device)
+        base = (self.fp8_arena.data_ptr() + 1023) // 1024 * 1024
+        self.lib.check(self.lib.dll.pop_enable_fp8(self.handle, base, need, _stream_ptr(stream)), "pop_enable_fp8")
 
     def prefill_chunked(self, tokens, embeds, l_keep: int, chunk_len: int, cache: KVCache,
                         logits: Optional[torch.Tensor] = None, stream=None):

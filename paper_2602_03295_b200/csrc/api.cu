@@ -43,6 +43,7 @@ struct Workspace {
   int32_t* ctr;      // [2] device counters of the greedy loop: position, step
   int32_t* tok;      // [B] current token of every sequence in the greedy loop
   int32_t* dec_ctr;  // [B][n_kv] arrival counters of the decode attention's split merge (zero between launches)
+  float* a_scale;    // [M] row scales of FP8 activations
   size_t total;
 };
 
@@ -60,6 +61,12 @@ struct pop_model {
   void* ws;
   size_t ws_bytes;
   int64_t last_launches;
+  // FP8 copies of the kept layers' widest matrices (caller's memory, filled by pop_enable_fp8):
+  // per layer E4M3 codes of wqkv [qkv_dim][d] and of the fused gate/up matrix [2 f_pad][d], then
+  // per layer two fp32 scales
+  uint8_t* fp8;            // null = bf16 operands everywhere
+  size_t fp8_layer_bytes;  // codes of one layer
+  float* fp8_scales;       // [n_layers][2]
 };
 
 namespace {
@@ -141,6 +148,7 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.ctr = (int32_t*)take(2 * 4);
   w.tok = (int32_t*)take((size_t)B * 4);
   w.dec_ctr = (int32_t*)take((size_t)B * c.n_kv_heads * 4);
+  w.a_scale = (float*)take(M * 4);
   w.total = o;
   return w;
 }
@@ -161,7 +169,12 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   const pop_config_t& c = m->cfg;
   const int M = cu ? rows : B * N, d = c.d_model;
   const int64_t pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
-  POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_in), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
+  const bool fp8 = m->fp8 != nullptr;
+  const uint8_t* w8 = fp8 ? m->fp8 + (size_t)(l - 1) * m->fp8_layer_bytes : nullptr;
+  if (fp8)
+    POP_TRY(launch_rmsnorm_e4m3(w.x, d, lp<float>(m, l, m->lo.ln_in), (uint8_t*)w.hn, d, w.a_scale, M, d, c.rms_eps, s));
+  else
+    POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_in), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
   // QKV projection with per-head norm, RoPE and the cache append (Eq. 2-3) in the GEMM's epilogue
   RopeArgs r{};
   r.q_out = w.q; r.ldq = m->q_dim;
@@ -177,6 +190,9 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   GemmArgs g{};
   g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
   g.M = M; g.N = m->qkv_dim; g.K = d; g.batch = 1; g.epilogue = EPI_QKV_ROPE; g.rope = &r;
+  if (fp8) {
+    g.fp8 = true; g.B = (const bf16*)w8; g.a_scale = w.a_scale; g.b_scale = m->fp8_scales + 2 * (l - 1);
+  }
   POP_TRY(launch_gemm(g, s));
   AttnArgs a{};
   a.q = w.q; a.ldq = m->q_dim;
@@ -201,11 +217,18 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
     POP_TRY(launch_gemm(g, s));
   }
   // gated FFN + residual
-  POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_ffn), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
+  if (fp8)
+    POP_TRY(launch_rmsnorm_e4m3(w.x, d, lp<float>(m, l, m->lo.ln_ffn), (uint8_t*)w.hn, d, w.a_scale, M, d, c.rms_eps, s));
+  else
+    POP_TRY(launch_rmsnorm(w.x, d, lp<float>(m, l, m->lo.ln_ffn), 0, w.hn, d, 0, M, d, 1, c.rms_eps, false, s));
   g = GemmArgs{};
   g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wgu); g.ldb = d;
   g.out = w.act; g.ldo = c.d_ffn; g.M = M; g.N = 2 * m->f_pad; g.K = d; g.batch = 1;
   g.epilogue = EPI_GATED_BF16; g.act = c.act; g.n_valid = c.d_ffn;
+  if (fp8) {
+    g.fp8 = true; g.B = (const bf16*)(w8 + (size_t)m->qkv_dim * d); g.a_scale = w.a_scale;
+    g.b_scale = m->fp8_scales + 2 * (l - 1) + 1;
+  }
   POP_TRY(launch_gemm(g, s));
   g = GemmArgs{};
   g.A = w.act; g.lda = c.d_ffn; g.B = lp<bf16>(m, l, m->lo.wd); g.ldb = c.d_ffn;
@@ -419,6 +442,7 @@ int run_prefill_ragged(pop_model* m, const pop_input_t* in, const int32_t* seq_l
                        pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
   if (!m || !in || !in->tokens || !seq_lens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
     return POP_E_INVALID;
+  if (m->fp8) return POP_E_INVALID;   // FP8 operands: pop_prefill, pop_full_prefill and pop_prefill_chunked only
   const pop_config_t& c = m->cfg;
   if (B < 1 || B > 4096 || L_keep < 1 || L_keep > c.n_layers) return POP_E_INVALID;
   std::vector<int32_t> cu(B + 1, 0);
@@ -479,6 +503,7 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
   const bool boundary = !(flags & POP_NO_BOUNDARY), indep_kv = !(flags & POP_NO_INDEP_KV);
   if (!m || !in || !in->tokens || !skip || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
     return POP_E_INVALID;
+  if (m->fp8) return POP_E_INVALID;   // FP8 operands: pop_prefill, pop_full_prefill and pop_prefill_chunked only
   const pop_config_t& c = m->cfg;
   if (N < 1 || B < 1 || (int64_t)N * B > (int64_t)1 << 24) return POP_E_INVALID;
   if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;
@@ -752,6 +777,40 @@ int pop_set_workspace(pop_model_t* m, void* dev_ws, size_t bytes) {
   if (!m || !dev_ws || reinterpret_cast<uintptr_t>(dev_ws) % kAlign) return POP_E_INVALID;
   m->ws = dev_ws;
   m->ws_bytes = bytes;
+  return POP_OK;
+}
+
+size_t pop_fp8_arena_bytes(const pop_model_t* m) {
+  if (!m) return 0;
+  const size_t layer = align_up(((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * m->cfg.d_model, kAlign);
+  return layer * m->cfg.n_layers + align_up((size_t)m->cfg.n_layers * 2 * 4 + 4, kAlign);
+}
+
+int pop_enable_fp8(pop_model_t* m, void* dev_arena, size_t bytes, void* stream) {
+  if (!m) return POP_E_INVALID;
+  if (!dev_arena) {
+    m->fp8 = nullptr;
+    return POP_OK;
+  }
+  if (reinterpret_cast<uintptr_t>(dev_arena) % kAlign || m->cfg.d_model % 16) return POP_E_INVALID;
+  if (bytes < pop_fp8_arena_bytes(m)) return POP_E_NOSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const pop_config_t& c = m->cfg;
+  const size_t d = c.d_model;
+  const size_t layer = align_up(((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * d, kAlign);
+  uint8_t* base = static_cast<uint8_t*>(dev_arena);
+  float* scales = reinterpret_cast<float*>(base + layer * c.n_layers);
+  unsigned int* scratch = reinterpret_cast<unsigned int*>(scales + 2 * c.n_layers);
+  for (int l = 1; l <= c.n_layers; ++l) {
+    uint8_t* dst = base + layer * (l - 1);
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wqkv), (int64_t)m->qkv_dim * d, dst,
+                                         scales + 2 * (l - 1), scratch, s));
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wgu), (int64_t)2 * m->f_pad * d,
+                                         dst + (size_t)m->qkv_dim * d, scales + 2 * (l - 1) + 1, scratch, s));
+  }
+  m->fp8 = base;
+  m->fp8_layer_bytes = layer;
+  m->fp8_scales = scales;
   return POP_OK;
 }
 

@@ -60,3 +60,48 @@ def test_row_and_tensor_scales():
     qs, sc = po.quant_tensors_e4m3(ws)
     assert max(float(t.abs().max()) for t in qs) == 448.0
     assert abs(sc - max(float(w.abs().max()) for w in ws) / 448.0) < 1e-9
+
+
+def test_fp8_projections_restated_with_the_library_cast():
+    # the QKV and gate/up products of a layer in "fp8" precision, restated with torch's float8 cast:
+    # codes of LN(x) per row and of the fused weight matrices per matrix, exact products, scales last
+    import pop_synth as ps
+    cfg = ps.ModelConfig("pin8", 2, 32, 4, 2, 8, 48, 50, 1e-5, 100.0, distinct_gains=True, weight_std=0.3)
+    w = ps.SynthWeights(cfg)
+    x = torch.randn(6, cfg.d_model, generator=torch.Generator().manual_seed(8), dtype=torch.float64) * 3
+    f8 = torch.float8_e4m3fn
+
+    def rows(h):
+        h32 = h.float()
+        amax = h32.abs().amax(-1, keepdim=True)
+        return (h32 * (448.0 / amax)).to(f8).double(), (amax / 448.0).double()
+
+    def mats(names, layer):
+        ws = [w.get(n, layer).float() for n in names]
+        amax = torch.stack([t.abs().max() for t in ws]).max()
+        return [(t * (448.0 / amax)).to(f8).double() for t in ws], float(amax / 448.0)
+
+    pos = torch.arange(6)
+    k, v = po.kv_generation(cfg, w, 1, x, pos, torch.float64, "fp8")
+    hq, sa = rows(po.rmsnorm(x, w.get("ln_in", 1).double(), cfg.rms_eps))
+    (wq, wk, wv), sw = mats(("wq", "wk", "wv"), 1)
+    v_ref = ((hq @ wv.T) * sa * sw).reshape(6, cfg.n_kv_heads, cfg.head_dim)
+    v_ref = v_ref.float().to(torch.bfloat16).double()                      # cache entries are bf16
+    assert (v - v_ref).abs().max().item() < 1e-12
+    k_ref = po.rope(((hq @ wk.T) * sa * sw).reshape(6, cfg.n_kv_heads, cfg.head_dim), pos, cfg.rope_theta)
+    assert (k - k_ref.float().to(torch.bfloat16).double()).abs().max().item() < 1e-12
+    # the quantised model stays near the unquantised one, and is not it
+    tokens = ps.uniform_tokens(3, 1, 12, cfg.vocab)
+    a = po.full_prefill(cfg, w, tokens, precision="fp8")
+    b = po.full_prefill(cfg, w, tokens, precision="kernel")
+    for l in range(cfg.n_layers):
+        err = (a["V"][l] - b["V"][l]).abs().max() / b["V"][l].abs().max()
+        assert 0 < err.item() < 0.25          # 3 mantissa bits, rows of 32 terms
+    # kept layers only: with every layer pruned but the first, the deep layers' entries of positions < N-1
+    # are bf16 projections of an fp8-computed state
+    r = po.pop_prefill(cfg, w, tokens, None, 1, precision="kernel", fp8_kept=True)
+    r0 = po.pop_prefill(cfg, w, tokens, None, 1, precision="kernel")
+    assert (r["K"][0] - a["K"][0]).abs().max().item() == 0                 # layer 1 is the fp8 layer of the full run
+    assert (r["K"][1] - r0["K"][1]).abs().max().item() > 0                 # H differs
+    kk, vv = po.kv_generation(cfg, w, 2, r["H"][0], torch.arange(11), torch.float64, "kernel")
+    assert (r["K"][1][0, :11] - kk).abs().max().item() == 0
