@@ -69,3 +69,61 @@ def test_gemm_on_codes(L, M, N, K):
     outb = torch.zeros(M, N, dtype=torch.bfloat16, device=DEV)
     L.gemm_e4m3(A8, sa, B8, sb, outb, epilogue=0)
     assert rel_err(outb, ref) < 1e-2
+
+
+TINY8 = {
+    "c1": ps.C1_TINY,
+    "qknorm": ps.C1_TINY.replace(qk_norm=1, distinct_gains=True),
+    "gemma": ps.C1_TINY.replace(act=1, post_norms=1, window=32, global_every=2, distinct_gains=True, n_layers=5),
+    "hd128": ps.C1_TINY.replace(head_dim=128, n_q_heads=2, n_kv_heads=2, distinct_gains=True),
+}
+
+
+@pytest.mark.parametrize("variant", list(TINY8))
+@pytest.mark.parametrize("B,N,l_keep,chunk", [(2, 150, 3, 0), (1, 129, 2, 0), (2, 200, 4, 64), (1, 1, 2, 0)])
+def test_kept_layers_on_fp8_operands(variant, B, N, l_keep, chunk):
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    from paper_2602_03295_b200 import PopError, POP_E_INVALID
+    cfg = TINY8[variant]
+    l_keep = min(l_keep, cfg.n_layers)
+    w = ps.SynthWeights(cfg)
+    tokens = ps.uniform_tokens(41, B, N, cfg.vocab)
+    ref = po.pop_prefill(cfg, w, tokens, None, l_keep, precision="kernel", fp8_kept=True)
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
+    model.enable_fp8()
+    cache = KVCache(cfg, B, N, 16, fill=float("nan"))
+    if chunk:
+        logits = model.prefill_chunked(tokens.to(DEV), None, l_keep, chunk, cache)
+    else:
+        logits = model.prefill(tokens.to(DEV), None, l_keep, cache)
+    assert model.last_status() == 0
+    assert not torch.isnan(logits).any()
+    # Tolerances. Layer 1 sees identical inputs on both sides, so its codes agree (up to the rare boundary
+    # case the kernel test bounds) and the bf16 tolerance holds. From layer 2 on the two sides' inputs
+    # differ the way the bf16 path's do (accumulation order, bf16 roundings of intermediate operands that
+    # fall on the other side: ~3e-3 relative RMS), and E4M3 rounding is a step function with steps of
+    # 6-12 %: a fraction ~ 3e-3 / 0.09 of the values lands on the neighbouring code, and a projection
+    # then differs by sqrt(that fraction) * 0.09 ~ 1.5-2 % RMS per quantised operand whatever d is,
+    # growing with depth, with a tail of several times that over thousands of outputs. Hence for
+    # layers >= 2: RMS <= 5e-2 and max <= 2e-1 relative (measured: RMS 2-3 %).
+    def rms_rel(a, b):
+        a, b = a.detach().cpu().double(), b.double()
+        return ((a - b).pow(2).mean().sqrt() / b.pow(2).mean().sqrt()).item()
+    assert (logits.cpu().double() - ref["logits"]).abs().max().item() <= 1e-1
+    for l in range(cfg.n_layers):
+        k, v = cache.gather(l)
+        tol, rtol = (2e-2, 1e-2) if l == 0 else (2e-1, 5e-2)
+        assert rel_err(k, ref["K"][l]) <= tol and rel_err(v, ref["V"][l]) <= tol, f"layer {l + 1}"
+        assert rms_rel(k, ref["K"][l]) <= rtol and rms_rel(v, ref["V"][l]) <= rtol, f"layer {l + 1} (rms)"
+    # it is a different function from the bf16 path (the quantisation is really there) ...
+    cache16 = KVCache(cfg, B, N, 16, fill=float("nan"))
+    model.enable_fp8(False)
+    logits16 = model.prefill(tokens.to(DEV), None, l_keep, cache16)
+    if N > 1:
+        assert rel_err(cache.gather(0)[1], cache16.gather(0)[1]) > 1e-3
+    assert (logits16 - logits).abs().max().item() < 1.0
+    # ... and the entry points it does not cover say so
+    model.enable_fp8()
+    with pytest.raises(PopError) as e:
+        model.prefill_skip(tokens.to(DEV), None, {cfg.n_layers}, cache16)
+    assert e.value.code == POP_E_INVALID
