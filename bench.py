@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="config-5 sweep on the workload's model shape: prompt length x batch x L_keep/L, one "
                          "JSON line per point (POP vs full-depth prefill, tokens/s, TTFT, path TFLOP/s)")
+    ap.add_argument("--precision", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: E4M3 operands in the kept layers' QKV and gate/up GEMMs (a second workload; "
+                         "the default line is bf16 throughout)")
     ap.add_argument("--chunked", action="store_true",
                     help="long prompts through pop_prefill_chunked (one JSON line per point) instead of the default run")
     ap.add_argument("--kernel", default="", choices=[""] + KERNELS,
@@ -71,7 +74,7 @@ def resolve_workload(a) -> ps.Workload:
 # DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
 # summarised in profiles/gemm_kernel_residual_proj_c2.md; valid only for the kernel source it was taken on.
 GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
-                "gemm_cu_sha256": "569bc6fe80dddbecdbc1b12b0b3fb7a58d2b68bd9e3695c2668d2888855c019e"}
+                "gemm_cu_sha256": "9ec5b3097774497e2b2a7e3e9c662cb27cb4deecbead86a57f5fa8083106824a"}
 
 
 def gemm_traffic():
@@ -269,6 +272,9 @@ def run_ours(a, wl):
     cfg = wl.model
     lib = pk.lib()
     model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+    fp8 = a.precision == "fp8"
+    if fp8:
+        model.enable_fp8()
     tokens_h, embeds_h = ps.make_prompt(wl, replica_seed(rank))
     tokens_h = tokens_h.pin_memory()
     embeds_h = None if embeds_h is None else embeds_h.pin_memory()
@@ -371,9 +377,18 @@ def run_ours(a, wl):
     breakdown = {k: {"ms": round(v[0], 3), "launches": v[2]} for k, v in prof.items()}
     breakdown["attention"]["tflops"] = round(att_flops / (att_ms * 1e-3) / 1e12, 1) if att_ms > 0 else None
 
+    if fp8:
+        # the GEMM class mixes dtypes: its peak is total flop / (fp8 flop / (2 x bf16 peak) + bf16 flop / bf16 peak),
+        # 2 being the nominal fp8 : bf16 ratio
+        f_pad = (cfg.d_ffn + 127) // 128 * 128
+        rows = wl.batch * wl.seq_len
+        f8 = 2.0 * rows * cfg.d_model * ((cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim + 2 * f_pad) * wl.l_keep
+        tot = achieved_tf * 1e12 * gemm_ms * 1e-3
+        peak_tf = tot / (f8 / (2 * peak_tf) + (tot - f8) / peak_tf) if peak_tf else peak_tf
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(a.warmup, 3),
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-           "dtype": "bf16", "data": "synthetic", "config": workload_config(wl, a),
+           "dtype": "e4m3 (QKV, gate/up of kept layers) + bf16" if fp8 else "bf16", "data": "synthetic",
+           "config": workload_config(wl, a),
            "ttft_ms": ms_step, "full_prefill_ms": full_ms, "speedup_vs_full_prefill": full_ms / ms_step,
            "speedup_ceiling_flop_ratio": po.prefill_flops(cfg, wl.batch, wl.seq_len, None) / flops,
            "algorithmic_tflop": flops / 1e12,
@@ -394,7 +409,8 @@ def run_ours(a, wl):
            "roofline": {"kernel": "gemm_kernel (tcgen05 projection GEMM, all epilogues)", "bound": "tensor",
                         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                         "frac": achieved_tf / peak_tf if peak_tf else None,
-                        "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})",
+                        "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})"
+                                       + (", fp8 launches at 2 x that (nominal ratio), flop-weighted" if fp8 else ""),
                         "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": gemm_traffic(),
                         "traffic_launch": GEMM_TRAFFIC["launch"]},
            "kernel_breakdown": breakdown}

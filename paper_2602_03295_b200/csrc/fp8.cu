@@ -18,23 +18,6 @@ __device__ __forceinline__ float warp_sum_f(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
-// block-wide reductions, result broadcast to every thread; `red` holds >= 32 floats
-__device__ __forceinline__ float block_reduce(float v, float* red, bool is_max) {
-  v = is_max ? warp_max(v) : warp_sum_f(v);
-  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
-  __syncthreads();
-  if (l == 0) red[w] = v;
-  __syncthreads();
-  const int nw = (blockDim.x + 31) >> 5;
-  float t = (threadIdx.x < nw) ? red[threadIdx.x] : (is_max ? 0.f : 0.f);
-  if (w == 0) {
-    t = is_max ? warp_max(t) : warp_sum_f(t);
-    if (l == 0) red[0] = t;
-  }
-  __syncthreads();
-  return red[0];
-}
-
 // two fp32 values -> two E4M3 codes (round to nearest even, saturating), `lo` in the low byte
 __device__ __forceinline__ uint16_t cvt_e4m3x2(float lo, float hi) {
   uint16_t r;
@@ -46,62 +29,65 @@ __device__ __forceinline__ uint32_t cvt_e4m3x4(float a, float b, float c, float 
 }
 
 // RMSNorm with an E4M3 result: y = x * rsqrt(mean(x^2) + eps) * gain in fp32, amax = max |y| over the row,
-// codes e4m3(y * (448 / amax)), scale[row] = amax / 448 (1 for a row of zeros). The row stays in
-// registers (rows up to 16 floats per thread; longer rows re-read their remainder).
+// codes e4m3(y * (448 / amax)), scale[row] = amax / 448 (1 for a row of zeros). The row and the gain stay
+// in registers (rows up to 16 floats per thread; longer rows re-read their remainder). Since the row
+// scale rstd is positive, max |y| = rstd * max |x * gain|: the sum of squares and that maximum are
+// reduced over the block in one pass.
 constexpr int QN_CACHE = 4;
 __global__ void rmsnorm_e4m3_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ gain,
                                     uint8_t* __restrict__ out, int64_t ldo, float* __restrict__ scale, int d,
                                     float eps) {
-  __shared__ float red[32];
+  __shared__ float red_s[32], red_m[32];
   const int row = blockIdx.x;
   const float* xr = x + (int64_t)row * ldx;
   const int step = blockDim.x * 4;
-  float4 yv[QN_CACHE];
-  float ss = 0.f;
-#pragma unroll
-  for (int i = 0; i < QN_CACHE; ++i) {
-    const int c = threadIdx.x * 4 + i * step;
-    yv[i] = c < d ? *reinterpret_cast<const float4*>(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-    if (c < d) ss += yv[i].x * yv[i].x + yv[i].y * yv[i].y + yv[i].z * yv[i].z + yv[i].w * yv[i].w;
-  }
-  for (int c = threadIdx.x * 4 + QN_CACHE * step; c < d; c += step) {
-    const float4 v = *reinterpret_cast<const float4*>(xr + c);
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-  }
-  ss = block_reduce(ss, red, false);
-  const float rstd = rsqrtf(ss / (float)d + eps);
-  float amax = 0.f;
+  float4 yv[QN_CACHE];                      // x * gain
+  float ss = 0.f, am = 0.f;
 #pragma unroll
   for (int i = 0; i < QN_CACHE; ++i) {
     const int c = threadIdx.x * 4 + i * step;
     if (c < d) {
+      const float4 v = *reinterpret_cast<const float4*>(xr + c);
       const float4 g = *reinterpret_cast<const float4*>(gain + c);
-      yv[i].x = yv[i].x * rstd * g.x; yv[i].y = yv[i].y * rstd * g.y;
-      yv[i].z = yv[i].z * rstd * g.z; yv[i].w = yv[i].w * rstd * g.w;
-      amax = fmaxf(amax, fmaxf(fmaxf(fabsf(yv[i].x), fabsf(yv[i].y)), fmaxf(fabsf(yv[i].z), fabsf(yv[i].w))));
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      yv[i] = make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w);
+      am = fmaxf(am, fmaxf(fmaxf(fabsf(yv[i].x), fabsf(yv[i].y)), fmaxf(fabsf(yv[i].z), fabsf(yv[i].w))));
+    } else {
+      yv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
   for (int c = threadIdx.x * 4 + QN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(xr + c);
     const float4 g = *reinterpret_cast<const float4*>(gain + c);
-    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x * rstd * g.x), fabsf(v.y * rstd * g.y)),
-                             fmaxf(fabsf(v.z * rstd * g.z), fabsf(v.w * rstd * g.w))));
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    am = fmaxf(am, fmaxf(fmaxf(fabsf(v.x * g.x), fabsf(v.y * g.y)), fmaxf(fabsf(v.z * g.z), fabsf(v.w * g.w))));
   }
-  amax = block_reduce(amax, red, true);
-  const float inv = amax > 0.f ? E4M3_MAX / amax : 1.0f;
+  // one block-wide pass for both values
+  ss = warp_sum_f(ss);
+  am = warp_max(am);
+  const int wp = threadIdx.x >> 5, ln = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  if (ln == 0) {
+    red_s[wp] = ss;
+    red_m[wp] = am;
+  }
+  __syncthreads();
+  ss = warp_sum_f(ln < nw ? red_s[ln] : 0.f);
+  am = warp_max(ln < nw ? red_m[ln] : 0.f);
+  const float rstd = rsqrtf(ss / (float)d + eps);
+  const float amax = am * rstd;             // max |y|
+  // y * (448 / amax) = (x * gain) * (rstd * 448 / amax)
+  const float k = amax > 0.f ? rstd * (E4M3_MAX / amax) : 0.f;
   if (threadIdx.x == 0) scale[row] = amax > 0.f ? amax / E4M3_MAX : 1.0f;
   uint8_t* orow = out + (int64_t)row * ldo;
 #pragma unroll
   for (int i = 0; i < QN_CACHE; ++i) {
     const int c = threadIdx.x * 4 + i * step;
-    if (c < d)
-      *reinterpret_cast<uint32_t*>(orow + c) = cvt_e4m3x4(yv[i].x * inv, yv[i].y * inv, yv[i].z * inv, yv[i].w * inv);
+    if (c < d) *reinterpret_cast<uint32_t*>(orow + c) = cvt_e4m3x4(yv[i].x * k, yv[i].y * k, yv[i].z * k, yv[i].w * k);
   }
   for (int c = threadIdx.x * 4 + QN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(xr + c);
     const float4 g = *reinterpret_cast<const float4*>(gain + c);
-    *reinterpret_cast<uint32_t*>(orow + c) =
-        cvt_e4m3x4(v.x * rstd * g.x * inv, v.y * rstd * g.y * inv, v.z * rstd * g.z * inv, v.w * rstd * g.w * inv);
+    *reinterpret_cast<uint32_t*>(orow + c) = cvt_e4m3x4(v.x * g.x * k, v.y * g.y * k, v.z * g.z * k, v.w * g.w * k);
   }
 }
 
