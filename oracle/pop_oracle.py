@@ -54,8 +54,8 @@ import torch
 # ---------------------------------------------------------------------------------------
 
 def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
-    """Identity in "exact" mode; otherwise ("kernel": bf16 operands; "fp8": E4M3 operands for the QKV and
-    gate/up projections, bf16 for the rest) round to bf16 and back."""
+    """Identity in "exact" mode; otherwise ("kernel": bf16 operands; "fp8": E4M3 operands for the four
+    projections of a layer, bf16 for attention and everything stored) round to bf16 and back."""
     if precision == "exact":
         return x
     return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
@@ -190,6 +190,14 @@ def _qkv_fp8(cfg, weights, layer: int, x: torch.Tensor, dtype):
     return tuple((hq @ w.to(dtype).T) * sa.to(dtype) * sw for w in (wq, wk, wv))
 
 
+def _proj_fp8(a: torch.Tensor, w: torch.Tensor, dtype) -> torch.Tensor:
+    """a @ w^T with E4M3 operands: one scale per row of a (already rounded to bf16, as it is stored),
+    one for the matrix."""
+    aq, sa = quant_rows_e4m3(a)
+    (wq,), sw = quant_tensors_e4m3([w])
+    return (aq.to(dtype) @ wq.to(dtype).T) * sa.to(dtype) * sw
+
+
 def kv_generation(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Tensor,
                   dtype, precision: str):
     """Eq. 2 (and, applied to a pruned layer's input, Eq. 14): the layer's own input norm,
@@ -231,7 +239,10 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
     q = _rnd(rope(q, positions, cfg.rope_theta), precision)
     a = attention(q, k_cur, v_cur, positions, cfg.layer_window(layer), precision, k_pos0)
     a = _rnd(a.reshape(-1, cfg.q_dim), precision)
-    o = a @ _w(weights, "wo", layer, dtype).T
+    if precision == "fp8":
+        o = _proj_fp8(a, weights.get("wo", layer), dtype)
+    else:
+        o = a @ _w(weights, "wo", layer, dtype).T
     if cfg.post_norms:
         o = rmsnorm(o, _w(weights, "post_attn_norm", layer, dtype), cfg.rms_eps)
     y = x + o                                                           # Eq. 1, first line
@@ -244,7 +255,10 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
         h2 = _rnd(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps), precision)
         gate = h2 @ _w(weights, "w_gate", layer, dtype).T
         up = h2 @ _w(weights, "w_up", layer, dtype).T
-    f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w(weights, "w_down", layer, dtype).T
+    if precision == "fp8":
+        f = _proj_fp8(_rnd(gated_act(gate, up, cfg.act), precision), weights.get("w_down", layer), dtype)
+    else:
+        f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w(weights, "w_down", layer, dtype).T
     if cfg.post_norms:
         f = rmsnorm(f, _w(weights, "post_ffn_norm", layer, dtype), cfg.rms_eps)
     return y + f, k_cur, v_cur                                          # Eq. 1, second line
@@ -320,7 +334,7 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
         Their K, V rows of positions 1..N-1 are returned as NaN ("absent").
 
     fp8_kept (deep-suffix set only): every position, x_N included, passes the kept layers with
-    E4M3 operands in the QKV and gate/up projections (precision "fp8"); the pruned layers'
+    E4M3 operands in their four projections (precision "fp8"); the pruned layers'
     projections and x_N's pass through the deep layers use `precision`.
 
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
