@@ -139,17 +139,18 @@ int pop_prefill_ragged(pop_model_t* m, const pop_input_t* tokens_or_embeds, cons
 int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      const uint8_t* skip, pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
-/* FP8 operands for the two widest projections of every kept layer (QKV and gate/up: 65 % of a layer's
- * GEMM work). The paper runs unquantised models and names stage-aware quantisation as a direction
- * (Sec. 6); this is that second precision, off by default. pop_enable_fp8 writes E4M3 copies of those
- * weight matrices (one scale per matrix) into dev_arena (caller's device memory, 1024-byte aligned,
- * at least pop_fp8_arena_bytes(m); it must stay valid while enabled; d_model a multiple of 16).
- * While enabled, pop_prefill, pop_full_prefill and pop_prefill_chunked normalise the rows entering
- * those projections straight to E4M3 codes with one scale per row and run the two GEMMs on the
- * codes (fp32 accumulation; scales applied to the accumulator before the usual epilogue); the
- * output projection, the down projection, the pruned layers' Eq. 14 projections and the boundary
- * token's deep layers keep bf16 operands. pop_prefill_ragged, pop_prefill_skip and
- * pop_prefill_ablation return POP_E_INVALID while it is enabled. dev_arena = NULL disables it. */
+/* FP8 operands for the four projections of every kept layer (QKV, output, gate/up, down). The paper
+ * runs unquantised models and names stage-aware quantisation as a direction (Sec. 6); this is that
+ * second precision, off by default. pop_enable_fp8 writes E4M3 copies of those weight matrices (one
+ * scale per matrix) into dev_arena (caller's device memory, 1024-byte aligned, at least
+ * pop_fp8_arena_bytes(m); it must stay valid while enabled; d_model, q_dim, d_ffn multiples of 16 and
+ * q_dim, d_ffn <= 16384, POP_E_INVALID otherwise). While enabled, pop_prefill, pop_full_prefill and
+ * pop_prefill_chunked turn the rows entering those projections into E4M3 codes with one scale per
+ * row (the normalised rows straight from the norm, the stored bf16 attention output and gated
+ * activation in place) and run the four GEMMs on the codes (fp32 accumulation; scales applied to
+ * the accumulator before the usual epilogue); attention, the pruned layers' Eq. 14 projections
+ * and the boundary token's deep layers keep bf16 operands. pop_prefill_ragged, pop_prefill_skip
+ * and pop_prefill_ablation return POP_E_INVALID while it is enabled. dev_arena = NULL disables it. */
 size_t pop_fp8_arena_bytes(const pop_model_t* m);
 int pop_enable_fp8(pop_model_t* m, void* dev_arena, size_t bytes, void* stream);
 

@@ -75,13 +75,18 @@ int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* 
  *
  * pop_k_rmsnorm_e4m3: y = LN(x[r]) as pop_k_rmsnorm computes it in fp32; out[r][:] = e4m3(y * 448 /
  *   max|y|) as bytes (row stride ldo bytes, a multiple of 16), scale[r] = max|y| / 448 (1 for a zero row).
+ * pop_k_quant_rows_e4m3: rows of stored bf16 values (row stride ld_in elements, d <= 16384 a multiple of 8):
+ *   out[r][:] = e4m3(in[r][:] * 448 / max|in[r]|) (row stride ld_out bytes, a multiple of 16), scale[r] as
+ *   above. out may be in itself (each row's codes then fill the first d bytes of the row).
  * pop_k_quantize_e4m3: the same for a whole bf16 array of n elements (n a multiple of 8) with one
  *   scale: out[i] = e4m3(w[i] * 448 / max|w|), *scale = max|w| / 448. scratch4: 4 device bytes.
  * pop_k_gemm_e4m3: D[m][n] = a_scale[m] * *b_scale * sum_k A[m][k] * B[n][k] on the codes (fp32
- *   accumulation on the tensor cores, kind f8f6f4), then epilogue 0, 1 or 3 of pop_k_gemm. lda,
+ *   accumulation on the tensor cores, kind f8f6f4), then epilogue 0, 1, 2 or 3 of pop_k_gemm. lda,
  *   ldb, K count codes and are multiples of 16; pointers 16-byte aligned; a_scale, b_scale device fp32. */
 int pop_k_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, void* out, int64_t ldo, float* scale,
                        int32_t rows, int32_t d, float eps, void* stream);
+int pop_k_quant_rows_e4m3(const void* in, int64_t ld_in, void* out, int64_t ld_out, float* scale, int32_t rows,
+                          int32_t d, void* stream);
 int pop_k_quantize_e4m3(const void* w, int64_t n, void* out, float* scale, void* scratch4, void* stream);
 int pop_k_gemm_e4m3(const void* A, int64_t lda, const float* a_scale, const void* B, int64_t ldb,
                     const float* b_scale, void* out, int64_t ldo, int32_t M, int32_t N, int32_t K, int32_t epilogue,

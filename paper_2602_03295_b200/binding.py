@@ -85,6 +85,7 @@ SIGNATURES = {
     "pop_k_gemm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
     "pop_k_rmsnorm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _I32, _I32, _F, _P]),
     "pop_k_quantize_e4m3": (C.c_int, [_P, _I64, _P, _P, _P, _P]),
+    "pop_k_quant_rows_e4m3": (C.c_int, [_P, _I64, _P, _I64, _P, _I32, _I32, _P]),
     "pop_k_gemm_norm": (C.c_int, [_P, _I64, _P, _I64, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P, _I64, _P, _P, _I32,
                                   _P, _I32, _I32, _I32, _F, _P]),
     "pop_k_gemm_qkv_rope": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _P, _I64, _P, _P, _I64, _I32,
@@ -185,6 +186,17 @@ class PopLibrary:
         code = self.dll.pop_k_rmsnorm_e4m3(x.data_ptr(), x.stride(0), gain.data_ptr(), out.data_ptr(), out.stride(0),
                                            scale.data_ptr(), rows, d, eps, _stream_ptr(stream))
         self.check(code, "pop_k_rmsnorm_e4m3")
+        return out, scale
+
+    def quant_rows_e4m3(self, x, in_place=False, stream=None):
+        """pop_k_quant_rows_e4m3 of bf16 rows [rows, d]: returns (codes uint8 [rows, d], scale fp32 [rows]);
+        in_place writes each row's codes over the start of the row (the view returned has row stride 2 d)."""
+        rows, d = x.shape
+        scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+        out = x.view(torch.uint8)[:, :d] if in_place else torch.empty(rows, d, dtype=torch.uint8, device=x.device)
+        code = self.dll.pop_k_quant_rows_e4m3(x.data_ptr(), x.stride(0), out.data_ptr(), out.stride(0),
+                                              scale.data_ptr(), rows, d, _stream_ptr(stream))
+        self.check(code, "pop_k_quant_rows_e4m3")
         return out, scale
 
     def quantize_e4m3(self, w, stream=None):

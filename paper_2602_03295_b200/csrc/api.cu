@@ -62,11 +62,11 @@ struct pop_model {
   size_t ws_bytes;
   int64_t last_launches;
   // FP8 copies of the kept layers' widest matrices (caller's memory, filled by pop_enable_fp8):
-  // per layer E4M3 codes of wqkv [qkv_dim][d] and of the fused gate/up matrix [2 f_pad][d], then
-  // per layer two fp32 scales
+  // per layer E4M3 codes of wqkv [qkv_dim][d], the fused gate/up matrix [2 f_pad][d], wo [d][q_dim]
+  // and w_down [d][d_ffn], then per layer four fp32 scales (same order)
   uint8_t* fp8;            // null = bf16 operands everywhere
   size_t fp8_layer_bytes;  // codes of one layer
-  float* fp8_scales;       // [n_layers][2]
+  float* fp8_scales;       // [n_layers][4]
 };
 
 namespace {
@@ -191,7 +191,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   g.A = w.hn; g.lda = d; g.B = lp<bf16>(m, l, m->lo.wqkv); g.ldb = d;
   g.M = M; g.N = m->qkv_dim; g.K = d; g.batch = 1; g.epilogue = EPI_QKV_ROPE; g.rope = &r;
   if (fp8) {
-    g.fp8 = true; g.B = (const bf16*)w8; g.a_scale = w.a_scale; g.b_scale = m->fp8_scales + 2 * (l - 1);
+    g.fp8 = true; g.B = (const bf16*)w8; g.a_scale = w.a_scale; g.b_scale = m->fp8_scales + 4 * (l - 1);
   }
   POP_TRY(launch_gemm(g, s));
   AttnArgs a{};
@@ -208,6 +208,13 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   g = GemmArgs{};
   g.A = w.ao; g.lda = m->q_dim; g.B = lp<bf16>(m, l, m->lo.wo); g.ldb = m->q_dim;
   g.M = M; g.N = d; g.K = m->q_dim; g.batch = 1;
+  if (fp8) {
+    // the stored bf16 rows become codes in place (a row's codes fill the first half of its bytes)
+    POP_TRY(launch_quant_rows_e4m3(w.ao, m->q_dim, (uint8_t*)w.ao, 2 * (int64_t)m->q_dim, w.a_scale, M, m->q_dim, s));
+    g.fp8 = true; g.lda = 2 * (int64_t)m->q_dim; g.a_scale = w.a_scale;
+    g.B = (const bf16*)(w8 + ((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * d);
+    g.b_scale = m->fp8_scales + 4 * (l - 1) + 2;
+  }
   if (c.post_norms) {
     g.out = w.t; g.ldo = d; g.epilogue = EPI_STORE_F32;
     POP_TRY(launch_gemm(g, s));
@@ -227,12 +234,18 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   g.epilogue = EPI_GATED_BF16; g.act = c.act; g.n_valid = c.d_ffn;
   if (fp8) {
     g.fp8 = true; g.B = (const bf16*)(w8 + (size_t)m->qkv_dim * d); g.a_scale = w.a_scale;
-    g.b_scale = m->fp8_scales + 2 * (l - 1) + 1;
+    g.b_scale = m->fp8_scales + 4 * (l - 1) + 1;
   }
   POP_TRY(launch_gemm(g, s));
   g = GemmArgs{};
   g.A = w.act; g.lda = c.d_ffn; g.B = lp<bf16>(m, l, m->lo.wd); g.ldb = c.d_ffn;
   g.M = M; g.N = d; g.K = c.d_ffn; g.batch = 1;
+  if (fp8) {
+    POP_TRY(launch_quant_rows_e4m3(w.act, c.d_ffn, (uint8_t*)w.act, 2 * (int64_t)c.d_ffn, w.a_scale, M, c.d_ffn, s));
+    g.fp8 = true; g.lda = 2 * (int64_t)c.d_ffn; g.a_scale = w.a_scale;
+    g.B = (const bf16*)(w8 + ((size_t)m->qkv_dim + 2 * (size_t)m->f_pad + (size_t)m->q_dim) * d);
+    g.b_scale = m->fp8_scales + 4 * (l - 1) + 3;
+  }
   if (c.post_norms) {
     g.out = w.t; g.ldo = d; g.epilogue = EPI_STORE_F32;
     POP_TRY(launch_gemm(g, s));
@@ -780,10 +793,14 @@ int pop_set_workspace(pop_model_t* m, void* dev_ws, size_t bytes) {
   return POP_OK;
 }
 
+static size_t fp8_layer_codes(const pop_model* m) {
+  const size_t d = m->cfg.d_model;
+  return ((size_t)m->qkv_dim + 2 * (size_t)m->f_pad + (size_t)m->q_dim + (size_t)m->cfg.d_ffn) * d;
+}
+
 size_t pop_fp8_arena_bytes(const pop_model_t* m) {
   if (!m) return 0;
-  const size_t layer = align_up(((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * m->cfg.d_model, kAlign);
-  return layer * m->cfg.n_layers + align_up((size_t)m->cfg.n_layers * 2 * 4 + 4, kAlign);
+  return align_up(fp8_layer_codes(m), kAlign) * m->cfg.n_layers + align_up((size_t)m->cfg.n_layers * 4 * 4 + 4, kAlign);
 }
 
 int pop_enable_fp8(pop_model_t* m, void* dev_arena, size_t bytes, void* stream) {
@@ -792,21 +809,27 @@ int pop_enable_fp8(pop_model_t* m, void* dev_arena, size_t bytes, void* stream) 
     m->fp8 = nullptr;
     return POP_OK;
   }
-  if (reinterpret_cast<uintptr_t>(dev_arena) % kAlign || m->cfg.d_model % 16) return POP_E_INVALID;
+  const pop_config_t& c = m->cfg;
+  if (reinterpret_cast<uintptr_t>(dev_arena) % kAlign) return POP_E_INVALID;
+  // code rows are GEMM operands (16-byte granules), activation rows are quantised by one CTA each
+  if (c.d_model % 16 || m->q_dim % 16 || c.d_ffn % 16 || c.d_ffn > 16384 || m->q_dim > 16384) return POP_E_INVALID;
   if (bytes < pop_fp8_arena_bytes(m)) return POP_E_NOSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const pop_config_t& c = m->cfg;
   const size_t d = c.d_model;
-  const size_t layer = align_up(((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * d, kAlign);
+  const size_t layer = align_up(fp8_layer_codes(m), kAlign);
   uint8_t* base = static_cast<uint8_t*>(dev_arena);
   float* scales = reinterpret_cast<float*>(base + layer * c.n_layers);
-  unsigned int* scratch = reinterpret_cast<unsigned int*>(scales + 2 * c.n_layers);
+  unsigned int* scratch = reinterpret_cast<unsigned int*>(scales + 4 * c.n_layers);
   for (int l = 1; l <= c.n_layers; ++l) {
     uint8_t* dst = base + layer * (l - 1);
-    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wqkv), (int64_t)m->qkv_dim * d, dst,
-                                         scales + 2 * (l - 1), scratch, s));
-    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wgu), (int64_t)2 * m->f_pad * d,
-                                         dst + (size_t)m->qkv_dim * d, scales + 2 * (l - 1) + 1, scratch, s));
+    float* sc = scales + 4 * (l - 1);
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wqkv), (int64_t)m->qkv_dim * d, dst, sc, scratch, s));
+    dst += (size_t)m->qkv_dim * d;
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wgu), (int64_t)2 * m->f_pad * d, dst, sc + 1, scratch, s));
+    dst += (size_t)2 * m->f_pad * d;
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wo), (int64_t)m->q_dim * d, dst, sc + 2, scratch, s));
+    dst += (size_t)m->q_dim * d;
+    POP_TRY(launch_quantize_weights_e4m3(lp<bf16>(m, l, m->lo.wd), (int64_t)c.d_ffn * d, dst, sc + 3, scratch, s));
   }
   m->fp8 = base;
   m->fp8_layer_bytes = layer;

@@ -28,7 +28,9 @@ int pop_k_gemm_e4m3(const void* A, int64_t lda, const float* a_scale, const void
   a.M = M; a.N = N; a.K = K; a.batch = 1;
   a.epilogue = epilogue; a.act = act; a.n_valid = n_valid;
   a.fp8 = true; a.a_scale = a_scale; a.b_scale = b_scale;
-  if (epilogue != EPI_STORE_BF16 && epilogue != EPI_STORE_F32 && epilogue != EPI_GATED_BF16) return POP_E_INVALID;
+  if (epilogue != EPI_STORE_BF16 && epilogue != EPI_STORE_F32 && epilogue != EPI_ADD_F32 &&
+      epilogue != EPI_GATED_BF16)
+    return POP_E_INVALID;
   return launch_gemm(a, static_cast<cudaStream_t>(stream));
 }
 
@@ -36,6 +38,12 @@ int pop_k_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, void* out
                        int32_t rows, int32_t d, float eps, void* stream) {
   return launch_rmsnorm_e4m3(x, ldx, gain, static_cast<uint8_t*>(out), ldo, scale, rows, d, eps,
                              static_cast<cudaStream_t>(stream));
+}
+
+int pop_k_quant_rows_e4m3(const void* in, int64_t ld_in, void* out, int64_t ld_out, float* scale, int32_t rows,
+                          int32_t d, void* stream) {
+  return launch_quant_rows_e4m3(static_cast<const bf16*>(in), ld_in, static_cast<uint8_t*>(out), ld_out, scale, rows, d,
+                                static_cast<cudaStream_t>(stream));
 }
 
 int pop_k_quantize_e4m3(const void* w, int64_t n, void* out, float* scale, void* scratch4, void* stream) {

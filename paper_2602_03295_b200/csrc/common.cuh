@@ -115,7 +115,7 @@ struct GemmArgs {
   // rsqrt(sum_i ss_in[row * ss_in_ld + i] / norm_d + norm_eps) before its own epilogue.
   bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
   const float* ss_in; int ss_cnt; int ss_in_ld; int norm_d; float norm_eps;
-  // FP8 operands (batch == 1; store, gated and QKV epilogues): A and B point at E4M3 codes, lda / ldb /
+  // FP8 operands (batch == 1, no folded norm): A and B point at E4M3 codes, lda / ldb /
   // K count codes (multiples of 16), and the accumulator is scaled by a_scale[row] * *b_scale (device)
   // before the epilogue proper
   bool fp8; const float* a_scale; const float* b_scale;
@@ -190,6 +190,9 @@ int launch_gather_last_rows(const float* src, float* dst, int batch, int d, cons
 // out[row][:] = e4m3(LN(x[row]) * 448 / amax_row), scale[row] = amax_row / 448 (LN = RMSNorm with `gain`)
 int launch_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, uint8_t* out, int64_t ldo, float* scale,
                         int rows, int d, float eps, cudaStream_t s);
+// rows of bf16 values -> codes and one scale per row (d <= 16384); out may alias in (row by row in place)
+int launch_quant_rows_e4m3(const bf16* in, int64_t ld_in, uint8_t* out, int64_t ld_out, float* scale, int rows, int d,
+                           cudaStream_t s);
 // out[i] = e4m3(w[i] * 448 / amax), *scale = amax / 448 over the n elements; scratch: 4 bytes
 int launch_quantize_weights_e4m3(const bf16* w, int64_t n, uint8_t* out, float* scale, unsigned int* scratch,
                                  cudaStream_t s);

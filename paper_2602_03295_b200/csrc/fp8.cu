@@ -91,6 +91,55 @@ __global__ void rmsnorm_e4m3_kernel(const float* __restrict__ x, int64_t ldx, co
   }
 }
 
+// Rows of stored bf16 activations (attention output, gated FFN activation) -> E4M3 codes with one scale per
+// row: amax = max |row|, codes e4m3(v * (448 / amax)), scale = amax / 448. The whole row sits in registers
+// (up to 8 x 8 values per thread) before the first code is written, so `out` may be the row's own memory.
+constexpr int QR_CACHE = 8;
+__global__ void __launch_bounds__(256) quant_rows_bf16_e4m3_kernel(const bf16* in, int64_t ld_in, uint8_t* out,
+                                                                   int64_t ld_out, float* __restrict__ scale, int d) {
+  __shared__ float red_m[8];
+  const int row = blockIdx.x;
+  const bf16* ir = in + (int64_t)row * ld_in;
+  uint4 raw[QR_CACHE];
+  float am = 0.f;
+#pragma unroll
+  for (int i = 0; i < QR_CACHE; ++i) {
+    const int c = (i * 256 + threadIdx.x) * 8;
+    raw[i] = c < d ? *reinterpret_cast<const uint4*>(ir + c) : make_uint4(0, 0, 0, 0);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[i]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h[j]);
+      am = fmaxf(am, fmaxf(fabsf(f.x), fabsf(f.y)));
+    }
+  }
+  am = warp_max(am);
+  if ((threadIdx.x & 31) == 0) red_m[threadIdx.x >> 5] = am;
+  __syncthreads();                           // also: every thread holds its part of the row by now
+  am = warp_max((threadIdx.x & 31) < 8 ? red_m[threadIdx.x & 31] : 0.f);
+  const float inv = am > 0.f ? E4M3_MAX / am : 1.0f;
+  if (threadIdx.x == 0) scale[row] = am > 0.f ? am / E4M3_MAX : 1.0f;
+  uint8_t* orow = out + (int64_t)row * ld_out;
+#pragma unroll
+  for (int i = 0; i < QR_CACHE; ++i) {
+    const int c = (i * 256 + threadIdx.x) * 8;
+    if (c < d) {
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[i]);
+      float f[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 t = __bfloat1622float2(h[j]);
+        f[2 * j] = t.x * inv;
+        f[2 * j + 1] = t.y * inv;
+      }
+      uint2 o;
+      o.x = cvt_e4m3x4(f[0], f[1], f[2], f[3]);
+      o.y = cvt_e4m3x4(f[4], f[5], f[6], f[7]);
+      *reinterpret_cast<uint2*>(orow + c) = o;
+    }
+  }
+}
+
 // weight matrices, once per model: amax over the matrix (non-negative floats order like their bit patterns),
 // then codes e4m3(w * (448 / amax)) and scale = amax / 448
 __global__ void amax_bf16_kernel(const bf16* __restrict__ w, int64_t n, unsigned int* __restrict__ amax_bits) {
@@ -136,6 +185,16 @@ int launch_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, uint8_t*
   if (!x || !gain || !out || !scale || d % 4 || ldx % 4 || ldo % 16 || rows < 1) return POP_E_INVALID;
   ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 5.0, s);
   rmsnorm_e4m3_kernel<<<rows, d >= 2048 ? 256 : 128, 0, s>>>(x, ldx, gain, out, ldo, scale, d, eps);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+int launch_quant_rows_e4m3(const bf16* in, int64_t ld_in, uint8_t* out, int64_t ld_out, float* scale, int rows, int d,
+                           cudaStream_t s) {
+  if (!in || !out || !scale || rows < 1 || d < 8 || d % 8 || ld_in % 8 || ld_out % 16) return POP_E_INVALID;
+  if (d > QR_CACHE * 256 * 8) return POP_E_INVALID;     // the row must fit the registers of one CTA
+  ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 3.0, s);
+  quant_rows_bf16_e4m3_kernel<<<rows, 256, 0, s>>>(in, ld_in, out, ld_out, scale, d);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

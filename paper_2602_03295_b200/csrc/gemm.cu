@@ -407,7 +407,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int v = 0; v < 8; ++v) {
             float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
                                    __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-            if (EPI == EPI_STORE_F32) { x.x *= rs; x.y *= rs; x.z *= rs; x.w *= rs; }
+            if (EPI == EPI_STORE_F32 || FP8) { x.x *= rs; x.y *= rs; x.z *= rs; x.w *= rs; }
             *reinterpret_cast<float4*>(mine + ((v ^ (lane & 7)) << 4)) = x;
           }
           fence_proxy_async_smem();
@@ -537,8 +537,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   CUtensorMap ta, tb;
   int rc;
   if (a.fp8) {
-    if (a.batch != 1 || !a.a_scale || !a.b_scale || a.K % 16 || a.lda % 16 || a.ldb % 16 || a.hn_out || a.ss_in ||
-        a.epilogue == EPI_ADD_F32)
+    if (a.batch != 1 || !a.a_scale || !a.b_scale || a.K % 16 || a.lda % 16 || a.ldb % 16 || a.hn_out || a.ss_in)
       return POP_E_INVALID;
     rc = make_tmap_u8_3d(&ta, a.A, a.K, a.M, 1, a.lda, (uint64_t)a.lda * a.M, BM);
     if (rc) return rc;
@@ -603,6 +602,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     switch (a.epilogue) {
       case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, stream);
       case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, stream);
+      case EPI_ADD_F32: return launch_epi<EPI_ADD_F32, 0, true>(ta, tb, to, p, grid, stream);
       case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, stream);
       case EPI_QKV_ROPE:
         switch (a.rope->hd) {
