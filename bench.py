@@ -54,7 +54,7 @@ def parse_args():
                     help="config-5 sweep on the workload's model shape: prompt length x batch x L_keep/L, one "
                          "JSON line per point (POP vs full-depth prefill, tokens/s, TTFT, path TFLOP/s)")
     ap.add_argument("--precision", default="bf16", choices=["bf16", "fp8"],
-                    help="fp8: E4M3 operands in the kept layers' QKV and gate/up GEMMs (a second workload; "
+                    help="fp8: E4M3 operands in the kept layers' four projection GEMMs (a second workload; "
                          "the default line is bf16 throughout)")
     ap.add_argument("--chunked", action="store_true",
                     help="long prompts through pop_prefill_chunked (one JSON line per point) instead of the default run")
@@ -74,7 +74,7 @@ def resolve_workload(a) -> ps.Workload:
 # DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
 # summarised in profiles/gemm_kernel_residual_proj_c2.md; valid only for the kernel source it was taken on.
 GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
-                "gemm_cu_sha256": "9ec5b3097774497e2b2a7e3e9c662cb27cb4deecbead86a57f5fa8083106824a"}
+                "gemm_cu_sha256": "b020e6f3dc461ff535a8595aa3cb4c3e2e020095c472c6b99ae5e15467c0139e"}
 
 
 def gemm_traffic():
@@ -382,12 +382,13 @@ def run_ours(a, wl):
         # 2 being the nominal fp8 : bf16 ratio
         f_pad = (cfg.d_ffn + 127) // 128 * 128
         rows = wl.batch * wl.seq_len
-        f8 = 2.0 * rows * cfg.d_model * ((cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim + 2 * f_pad) * wl.l_keep
+        qd_ = cfg.n_q_heads * cfg.head_dim
+        f8 = 2.0 * rows * cfg.d_model * (qd_ + 2 * cfg.n_kv_heads * cfg.head_dim + 2 * f_pad + qd_ + cfg.d_ffn) * wl.l_keep
         tot = achieved_tf * 1e12 * gemm_ms * 1e-3
         peak_tf = tot / (f8 / (2 * peak_tf) + (tot - f8) / peak_tf) if peak_tf else peak_tf
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(a.warmup, 3),
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-           "dtype": "e4m3 (QKV, gate/up of kept layers) + bf16" if fp8 else "bf16", "data": "synthetic",
+           "dtype": "e4m3 (the four projections of kept layers) + bf16" if fp8 else "bf16", "data": "synthetic",
            "config": workload_config(wl, a),
            "ttft_ms": ms_step, "full_prefill_ms": full_ms, "speedup_vs_full_prefill": full_ms / ms_step,
            "speedup_ceiling_flop_ratio": po.prefill_flops(cfg, wl.batch, wl.seq_len, None) / flops,
