@@ -55,7 +55,8 @@ import torch
 
 def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
     """Identity in "exact" mode; otherwise ("kernel": bf16 operands; "fp8": E4M3 operands for the four
-    projections of a layer, bf16 for attention and everything stored) round to bf16 and back."""
+    projections of a layer; "fp8w": E4M3 weights of those projections, bf16 activations; bf16 for
+    attention and everything stored in all three) round to bf16 and back."""
     if precision == "exact":
         return x
     return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
@@ -190,6 +191,14 @@ def _qkv_fp8(cfg, weights, layer: int, x: torch.Tensor, dtype):
     return tuple((hq @ w.to(dtype).T) * sa.to(dtype) * sw for w in (wq, wk, wv))
 
 
+def _w_deq(weights, names, layer: int, dtype):
+    """The matrices `names` of a layer as the E4M3 kernels see them when only the weights are
+    quantised (precision "fp8w": single-position passes stream codes and keep bf16 activations):
+    code * scale, one scale for the group (it is stored as one fused matrix)."""
+    qs, sw = quant_tensors_e4m3([weights.get(n, layer) for n in names])
+    return [(q * sw).to(dtype) for q in qs]
+
+
 def _proj_fp8(a: torch.Tensor, w: torch.Tensor, dtype) -> torch.Tensor:
     """a @ w^T with E4M3 operands: one scale per row of a (already rounded to bf16, as it is stored),
     one for the matrix."""
@@ -208,8 +217,12 @@ def kv_generation(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
         v = v.reshape(-1, cfg.n_kv_heads, cfg.head_dim)
     else:
         h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
-        k = (h @ _w(weights, "wk", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
-        v = (h @ _w(weights, "wv", layer, dtype).T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+        if precision == "fp8w":
+            _, wk, wv = _w_deq(weights, ("wq", "wk", "wv"), layer, dtype)
+        else:
+            wk, wv = _w(weights, "wk", layer, dtype), _w(weights, "wv", layer, dtype)
+        k = (h @ wk.T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+        v = (h @ wv.T).reshape(-1, cfg.n_kv_heads, cfg.head_dim)
     if cfg.qk_norm:
         k = rmsnorm(k, _w(weights, "k_norm", layer, dtype), cfg.rms_eps)
     k = rope(k, positions, cfg.rope_theta)
@@ -233,7 +246,8 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
         q = _qkv_fp8(cfg, weights, layer, x, dtype)[0].reshape(-1, cfg.n_q_heads, cfg.head_dim)
     else:
         h = _rnd(rmsnorm(x, _w(weights, "ln_in", layer, dtype), cfg.rms_eps), precision)
-        q = (h @ _w(weights, "wq", layer, dtype).T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
+        wq_ = _w_deq(weights, ("wq", "wk", "wv"), layer, dtype)[0] if precision == "fp8w" else _w(weights, "wq", layer, dtype)
+        q = (h @ wq_.T).reshape(-1, cfg.n_q_heads, cfg.head_dim)
     if cfg.qk_norm:
         q = rmsnorm(q, _w(weights, "q_norm", layer, dtype), cfg.rms_eps)
     q = _rnd(rope(q, positions, cfg.rope_theta), precision)
@@ -241,6 +255,8 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
     a = _rnd(a.reshape(-1, cfg.q_dim), precision)
     if precision == "fp8":
         o = _proj_fp8(a, weights.get("wo", layer), dtype)
+    elif precision == "fp8w":
+        o = a @ _w_deq(weights, ("wo",), layer, dtype)[0].T
     else:
         o = a @ _w(weights, "wo", layer, dtype).T
     if cfg.post_norms:
@@ -253,10 +269,16 @@ def layer_forward(cfg, weights, layer: int, x: torch.Tensor, positions: torch.Te
         up = (h2q.to(dtype) @ wu.to(dtype).T) * sa.to(dtype) * sw
     else:
         h2 = _rnd(rmsnorm(y, _w(weights, "ln_ffn", layer, dtype), cfg.rms_eps), precision)
-        gate = h2 @ _w(weights, "w_gate", layer, dtype).T
-        up = h2 @ _w(weights, "w_up", layer, dtype).T
+        if precision == "fp8w":
+            wg_, wu_ = _w_deq(weights, ("w_gate", "w_up"), layer, dtype)
+        else:
+            wg_, wu_ = _w(weights, "w_gate", layer, dtype), _w(weights, "w_up", layer, dtype)
+        gate = h2 @ wg_.T
+        up = h2 @ wu_.T
     if precision == "fp8":
         f = _proj_fp8(_rnd(gated_act(gate, up, cfg.act), precision), weights.get("w_down", layer), dtype)
+    elif precision == "fp8w":
+        f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w_deq(weights, ("w_down",), layer, dtype)[0].T
     else:
         f = _rnd(gated_act(gate, up, cfg.act), precision) @ _w(weights, "w_down", layer, dtype).T
     if cfg.post_norms:
@@ -334,8 +356,9 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
         Their K, V rows of positions 1..N-1 are returned as NaN ("absent").
 
     fp8_kept (deep-suffix set only): every position, x_N included, passes the kept layers with
-    E4M3 operands in their four projections (precision "fp8"); the pruned layers'
-    projections and x_N's pass through the deep layers use `precision`.
+    E4M3 operands in their four projections (precision "fp8"); x_N's pass through the deep layers
+    streams E4M3 weights with bf16 activations ("fp8w"); the pruned layers' Eq. 14 projections use
+    `precision`.
 
     Returns dict: K, V (N entries for every layer), logits [B, vocab],
     H [B, N-1, d] (the state leaving the last layer of phase 1 at positions 1..N-1; for the
@@ -376,7 +399,7 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
             x = x_all[N - 1: N]
             for l in range(1, L + 1):
                 x, kc[l - 1], vc[l - 1] = layer_forward(cfg, weights, l, x, posN, kc[l - 1], vc[l - 1], dtype,
-                                                        "fp8" if (fp8_kept and l not in skip) else precision)
+                                                        ("fp8" if l not in skip else "fp8w") if fp8_kept else precision)
             x_last = x[0]
         else:
             x_last = x[N - 1]

@@ -200,9 +200,11 @@ int launch_quantize_weights_e4m3(const bf16* w, int64_t n, uint8_t* out, float* 
 // ------------------------------------------------------------------------------------ boundary path
 struct GemvArgs {
   const void* x; int64_t ldx; bool x_f32;    // [B][K] bf16 or fp32
-  const bf16* w; int64_t ldw;                // [N][K]
+  const void* w; int64_t ldw;                // [N][K] bf16; or E4M3 codes (w_fp8, bf16 x only, K and ldw
+                                             // multiples of 16) with the matrix's scale at *w_scale (device)
   void* out; int64_t ldo;                    // mode 0: fp32 store; 2: fp32 +=; 3: gated -> bf16 [B][n_valid]
   int B, N, K, mode, act, n_valid;
+  bool w_fp8; const float* w_scale;
 };
 int launch_gemv(const GemvArgs& a, cudaStream_t s);
 struct DecAttnArgs {

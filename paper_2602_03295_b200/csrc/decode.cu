@@ -28,6 +28,19 @@ __device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
   }
 }
 
+// 16 E4M3 codes -> fp32 (exact: every E4M3 value is an fp16 value)
+__device__ __forceinline__ void unpack16_e4m3(const uint4& raw, float (&f)[16]) {
+  const uint16_t* h = reinterpret_cast<const uint16_t*>(&raw);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(h[j]));
+    const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    f[2 * j] = t.x;
+    f[2 * j + 1] = t.y;
+  }
+}
+
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -44,7 +57,8 @@ __device__ __forceinline__ float act_fn(float g, int act) {
 
 struct GemvDev {
   const void* x; int64_t ldx;      // [B][K] bf16 or fp32
-  const bf16* w; int64_t ldw;      // [N][K]
+  const void* w; int64_t ldw;      // [N][K] bf16, or E4M3 codes (W8 kernels) whose common scale is *w_scale
+  const float* w_scale;
   void* out; int64_t ldo;
   int B, N, K;
   int mode;                        // 0 store fp32, 2 fp32 +=, 3 gated -> bf16
@@ -72,8 +86,12 @@ __device__ __forceinline__ void load_x8(const void* x, int64_t off, float (&xf)[
 // KS = warps of a CTA that share the same rows and split K between them (KS consecutive warps act
 // as one group of 32 KS lanes); their partial sums meet in shared memory in a fixed order. Few
 // output rows with KS = 1 would leave most of the SMs' load slots empty.
-template <bool X_F32, int NB, bool GATED, int KS>
+// W8: the weights are E4M3 codes (16 per 16-byte load instead of 8 bf16), the activations stay as they
+// are; the sums are scaled by the matrix's scale at the end.
+template <bool X_F32, int NB, bool GATED, int KS, bool W8 = false>
 __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
+  constexpr int EL = W8 ? 16 : 8;                 // weight elements per 16-byte load
+  constexpr int WBYTES = W8 ? 1 : 2;
   const int lane = threadIdx.x & 31;
   const int wic = threadIdx.x >> 5;                         // warp in CTA
   const int slice = wic % KS;
@@ -85,13 +103,13 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   chain_trigger();
   if (KS == 1 && o0 >= n_out) return;
   // weight rows for output o: plain -> o; gated -> gate row (o/128)*256 + o%128, up row +128
-  const bf16* wr[RW];
+  const char* wr[RW];                             // byte addresses of the rows
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const int o = min(o0 + r, n_out - 1);
     const int64_t row = GATED ? (int64_t)(o >> 7) * 256 + (o & 127) : o;
-    wr[r] = p.w + row * p.ldw;
-    if (GATED) wr[R + r] = p.w + (row + 128) * p.ldw;
+    wr[r] = static_cast<const char*>(p.w) + row * p.ldw * WBYTES;
+    if (GATED) wr[R + r] = static_cast<const char*>(p.w) + (row + 128) * p.ldw * WBYTES;
   }
   float acc[RW][NB];
 #pragma unroll
@@ -104,38 +122,44 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   auto load_batch = [&](uint4 (&wraw)[GEMV_U][RW], int k0) {
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
-      const int k = k0 + u * 256 * KS;
+      const int k = k0 + u * 32 * EL * KS;
 #pragma unroll
       for (int r = 0; r < RW; ++r)
-        wraw[u][r] = (k < p.K) ? ld_stream(wr[r] + k) : make_uint4(0, 0, 0, 0);
+        wraw[u][r] = (k < p.K) ? ld_stream(wr[r] + (int64_t)k * WBYTES) : make_uint4(0, 0, 0, 0);
     }
   };
-  int k0 = (slice * 32 + lane) * 8;
+  int k0 = (slice * 32 + lane) * EL;
   uint4 wraw[GEMV_U][RW];
   if (k0 < p.K) load_batch(wraw, k0);
   chain_wait();
   while (k0 < p.K) {
 #pragma unroll
     for (int u = 0; u < GEMV_U; ++u) {
-      const int k = k0 + u * 256 * KS;
+      const int k = k0 + u * 32 * EL * KS;
       if (k < p.K) {
-        float wf[RW][8];
+        float wf[RW][EL];
 #pragma unroll
-        for (int r = 0; r < RW; ++r) unpack8(wraw[u][r], wf[r]);
+        for (int r = 0; r < RW; ++r) {
+          if constexpr (W8) unpack16_e4m3(wraw[u][r], wf[r]);
+          else unpack8(wraw[u][r], wf[r]);
+        }
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
           if (b < p.B) {
-            float xf[8];
-            load_x8<X_F32>(p.x, (int64_t)b * p.ldx + k, xf);
 #pragma unroll
-            for (int r = 0; r < RW; ++r)
+            for (int hh = 0; hh < EL / 8; ++hh) {
+              float xf[8];
+              load_x8<X_F32>(p.x, (int64_t)b * p.ldx + k + hh * 8, xf);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) acc[r][b] = fmaf(wf[r][e], xf[e], acc[r][b]);
+              for (int r = 0; r < RW; ++r)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[r][b] = fmaf(wf[r][hh * 8 + e], xf[e], acc[r][b]);
+            }
           }
         }
       }
     }
-    k0 += 256 * KS * GEMV_U;
+    k0 += 32 * EL * KS * GEMV_U;
     if (k0 < p.K) load_batch(wraw, k0);
   }
   if (KS > 1) {
@@ -167,6 +191,11 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
       if (b < p.B) {
         float v = KS > 1 ? acc[r][b] : warp_sum(acc[r][b]);
         float u = GATED ? (KS > 1 ? acc[GATED ? R + r : r][b] : warp_sum(acc[GATED ? R + r : r][b])) : 0.f;
+        if (W8) {
+          const float ws = *p.w_scale;
+          v *= ws;
+          u *= ws;
+        }
         const int o = o0 + r;
         if (lane == 0 && o < n_out) {
           if (p.mode == 0) {
@@ -182,25 +211,25 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   }
 }
 
-template <bool X_F32, bool GATED, int KS>
+template <bool X_F32, bool GATED, int KS, bool W8>
 void launch_gemv_nb(const GemvDev& p, int blocks, int threads, cudaStream_t s) {
-  if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
-  else if (p.B <= 2) launch_chained(gemv_kernel<X_F32, 2, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
-  else if (p.B <= 4) launch_chained(gemv_kernel<X_F32, 4, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
-  else launch_chained(gemv_kernel<X_F32, 8, GATED, KS>, dim3(blocks), dim3(threads), 0, s, p);
+  if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS, W8>, dim3(blocks), dim3(threads), 0, s, p);
+  else if (p.B <= 2) launch_chained(gemv_kernel<X_F32, 2, GATED, KS, W8>, dim3(blocks), dim3(threads), 0, s, p);
+  else if (p.B <= 4) launch_chained(gemv_kernel<X_F32, 4, GATED, KS, W8>, dim3(blocks), dim3(threads), 0, s, p);
+  else launch_chained(gemv_kernel<X_F32, 8, GATED, KS, W8>, dim3(blocks), dim3(threads), 0, s, p);
 }
 
-template <bool X_F32, bool GATED>
+template <bool X_F32, bool GATED, bool W8 = false>
 void launch_gemv_ks(const GemvDev& p, int row_warps, int ks, cudaStream_t s) {
   // the slices of a row group sit in one CTA of 8 warps; without a K split the warps are
   // independent and CTAs of 4 warps spread more evenly over the SMs (fewer, shorter stragglers)
   const int wpc = ks == 1 ? 4 : 8;
   const int blocks = ceil_div(row_warps * ks, wpc);
   switch (ks) {
-    case 8: launch_gemv_nb<X_F32, GATED, 8>(p, blocks, 256, s); break;
-    case 4: launch_gemv_nb<X_F32, GATED, 4>(p, blocks, 256, s); break;
-    case 2: launch_gemv_nb<X_F32, GATED, 2>(p, blocks, 256, s); break;
-    default: launch_gemv_nb<X_F32, GATED, 1>(p, blocks, wpc * 32, s); break;
+    case 8: launch_gemv_nb<X_F32, GATED, 8, W8>(p, blocks, 256, s); break;
+    case 4: launch_gemv_nb<X_F32, GATED, 4, W8>(p, blocks, 256, s); break;
+    case 2: launch_gemv_nb<X_F32, GATED, 2, W8>(p, blocks, 256, s); break;
+    default: launch_gemv_nb<X_F32, GATED, 1, W8>(p, blocks, wpc * 32, s); break;
   }
 }
 
@@ -534,28 +563,32 @@ __global__ void dec_combine_kernel(const DecAttnDev p) {
 int launch_gemv(const GemvArgs& a, cudaStream_t s) {
   if (!a.x || !a.w || !a.out || a.B < 1 || a.N < 1 || a.K < 1) return POP_E_INVALID;
   if (a.K % 8 || a.ldw % 8 || a.ldx % 8) return POP_E_INVALID;
+  if (a.w_fp8 && (a.x_f32 || !a.w_scale || a.K % 16 || a.ldw % 16)) return POP_E_INVALID;
+  const int el = a.w_fp8 ? 16 : 8;
   if (a.mode == 3 && (a.N % 256 || a.n_valid > a.N / 2)) return POP_E_INVALID;
   const int n_out = a.mode == 3 ? a.N / 2 : a.N;
   const int warps = ceil_div(n_out, GEMV_R);
   // split K between the warps of a CTA while all warps still fit on the GPU at once (148 SMs x 64)
   int ks = 1;
-  while (ks < 8 && warps * ks * 2 <= 148 * 64 && a.K >= 256 * ks * 2) ks *= 2;
+  while (ks < 8 && warps * ks * 2 <= 148 * 64 && a.K >= 32 * el * ks * 2) ks *= 2;
   const int elt = a.x_f32 ? 4 : 2;
   for (int b0 = 0; b0 < a.B; b0 += GEMV_MAXB) {
     GemvDev p;
     p.x = static_cast<const char*>(a.x) + (int64_t)b0 * a.ldx * elt;
     p.ldx = a.ldx;
-    p.w = a.w; p.ldw = a.ldw;
+    p.w = a.w; p.ldw = a.ldw; p.w_scale = a.w_scale;
     p.out = static_cast<char*>(a.out) + (int64_t)b0 * a.ldo * (a.mode == 3 ? 2 : 4);
     p.ldo = a.ldo;
     p.B = a.B - b0 < GEMV_MAXB ? a.B - b0 : GEMV_MAXB;
     p.N = a.N; p.K = a.K; p.mode = a.mode; p.act = a.act; p.n_valid = a.n_valid;
-    ProfScope prof(PROF_GEMV, (double)a.N * a.K * 2, s);
+    ProfScope prof(PROF_GEMV, (double)a.N * a.K * (a.w_fp8 ? 1 : 2), s);
     if (a.mode == 3) {
-      if (a.x_f32) launch_gemv_ks<true, true>(p, warps, ks, s);
+      if (a.w_fp8) launch_gemv_ks<false, true, true>(p, warps, ks, s);
+      else if (a.x_f32) launch_gemv_ks<true, true>(p, warps, ks, s);
       else launch_gemv_ks<false, true>(p, warps, ks, s);
     } else {
-      if (a.x_f32) launch_gemv_ks<true, false>(p, warps, ks, s);
+      if (a.w_fp8) launch_gemv_ks<false, false, true>(p, warps, ks, s);
+      else if (a.x_f32) launch_gemv_ks<true, false>(p, warps, ks, s);
       else launch_gemv_ks<false, false>(p, warps, ks, s);
     }
     count_launch();

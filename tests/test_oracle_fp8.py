@@ -110,3 +110,30 @@ def test_fp8_projections_restated_with_the_library_cast():
     assert (r["K"][1] - r0["K"][1]).abs().max().item() > 0                 # H differs
     kk, vv = po.kv_generation(cfg, w, 2, r["H"][0], torch.arange(11), torch.float64, "kernel")
     assert (r["K"][1][0, :11] - kk).abs().max().item() == 0
+
+
+def test_weight_only_precision_is_the_kernel_precision_on_dequantised_weights():
+    # "fp8w": a layer in kernel (bf16) precision whose four projection matrices are replaced by
+    # code * scale -- restated by running kernel precision on a weight set patched that way
+    import pop_synth as ps
+    cfg = ps.ModelConfig("pin8w", 2, 32, 4, 2, 8, 48, 50, 1e-5, 100.0, distinct_gains=True, weight_std=0.3)
+    w = ps.SynthWeights(cfg)
+    f8 = torch.float8_e4m3fn
+
+    class Patched:
+        def get(self, name, layer):
+            groups = [("wq", "wk", "wv"), ("w_gate", "w_up"), ("wo",), ("w_down",)]
+            for g in groups:
+                if name in g:
+                    amax = max(float(w.get(n, layer).float().abs().max()) for n in g)
+                    t = w.get(name, layer).float()
+                    return (t * (448.0 / amax)).to(f8).double() * (amax / 448.0)
+            return w.get(name, layer)
+    x = torch.randn(5, cfg.d_model, generator=torch.Generator().manual_seed(12), dtype=torch.float64)
+    pos = torch.arange(5)
+    a = po.layer_forward(cfg, w, 2, x, pos, None, None, torch.float64, "fp8w")
+    b = po.layer_forward(cfg, Patched(), 2, x, pos, None, None, torch.float64, "kernel")
+    for u, v in zip(a, b):
+        assert (u - v).abs().max().item() < 1e-5          # the scale is an fp32 number in the oracle
+    c = po.layer_forward(cfg, w, 2, x, pos, None, None, torch.float64, "kernel")
+    assert (a[0] - c[0]).abs().max().item() > 1e-4
