@@ -83,6 +83,12 @@ int pop_k_attention(const void* q, int64_t ldq, const void* k_pool, const void* 
  * pop_k_gemm_e4m3: D[m][n] = a_scale[m] * *b_scale * sum_k A[m][k] * B[n][k] on the codes (fp32
  *   accumulation on the tensor cores, kind f8f6f4), then epilogue 0, 1, 2 or 3 of pop_k_gemm. lda,
  *   ldb, K count codes and are multiples of 16; pointers 16-byte aligned; a_scale, b_scale device fp32. */
+/* pop_k_gemv with E4M3 weights (the single-position passes of Sec. 3.3 / the decode stage stream half the
+ * bytes): out[b][n] = *w_scale * sum_k x[b][k] * W[n][k], x bf16 [B][ldx] unquantised, W codes [N][ldw]
+ * (K and ldw multiples of 16), w_scale device fp32. Modes as pop_k_gemv. */
+int pop_k_gemv_e4m3(const void* x, int64_t ldx, const void* w, int64_t ldw, const float* w_scale, void* out,
+                    int64_t ldo, int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid,
+                    void* stream);
 int pop_k_rmsnorm_e4m3(const float* x, int64_t ldx, const float* gain, void* out, int64_t ldo, float* scale,
                        int32_t rows, int32_t d, float eps, void* stream);
 int pop_k_quant_rows_e4m3(const void* in, int64_t ld_in, void* out, int64_t ld_out, float* scale, int32_t rows,

@@ -82,6 +82,7 @@ SIGNATURES = {
     "pop_strerror": (C.c_char_p, [C.c_int]),
     "pop_k_gemm": (C.c_int, [_P, _I64, _I64, _P, _I64, _I64, _P, _I64, _I64, _I32, _I32, _I32, _I32, _I32, _I32,
                              _I32, _P]),
+    "pop_k_gemv_e4m3": (C.c_int, [_P, _I64, _P, _I64, _P, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_gemm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _P, _I64, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
     "pop_k_rmsnorm_e4m3": (C.c_int, [_P, _I64, _P, _P, _I64, _P, _I32, _I32, _F, _P]),
     "pop_k_quantize_e4m3": (C.c_int, [_P, _I64, _P, _P, _P, _P]),
@@ -177,6 +178,15 @@ class PopLibrary:
         self.check(code, "pop_k_gemm")
         return out
 
+
+    def gemv_e4m3(self, x, w8, w_scale, out, mode=0, act=0, n_valid=0, stream=None):
+        """pop_k_gemv_e4m3: x bf16 [B, K]; w8 uint8 codes [N, K]; w_scale fp32 [1]."""
+        B, K = x.shape
+        code = self.dll.pop_k_gemv_e4m3(x.data_ptr(), x.stride(0), w8.data_ptr(), w8.stride(0), w_scale.data_ptr(),
+                                        out.data_ptr(), out.stride(0), B, w8.shape[0], K, mode, act, n_valid,
+                                        _stream_ptr(stream))
+        self.check(code, "pop_k_gemv_e4m3")
+        return out
 
     def rmsnorm_e4m3(self, x, gain, eps, stream=None):
         """pop_k_rmsnorm_e4m3: returns (codes uint8 [rows, d], scale fp32 [rows])."""

@@ -300,6 +300,11 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   GemvArgs v{};
   v.x = w.hb; v.ldx = d; v.x_f32 = false; v.w = lp<bf16>(m, l, m->lo.wqkv); v.ldw = d;
   v.out = w.qkvb; v.ldo = m->qkv_dim; v.B = B; v.N = m->qkv_dim; v.K = d; v.mode = 0;
+  // with FP8 enabled the single-position passes stream the E4M3 copies of the four matrices (half the
+  // bytes) and keep their bf16 activations
+  const uint8_t* w8 = m->fp8 ? m->fp8 + (size_t)(l - 1) * m->fp8_layer_bytes : nullptr;
+  const float* sc8 = m->fp8 ? m->fp8_scales + 4 * (l - 1) : nullptr;
+  if (w8) { v.w = w8; v.w_fp8 = true; v.w_scale = sc8; }
   POP_TRY(launch_gemv(v, s));
   RopeArgs r{};
   r.in = w.qkvb; r.ld_in = m->qkv_dim; r.q_out = w.qb; r.ldq = m->q_dim;
@@ -325,6 +330,9 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};
   v.x = w.ob; v.ldx = m->q_dim; v.w = lp<bf16>(m, l, m->lo.wo); v.ldw = m->q_dim; v.B = B; v.N = d; v.K = m->q_dim;
+  if (w8) {
+    v.w = w8 + ((size_t)m->qkv_dim + 2 * (size_t)m->f_pad) * d; v.w_fp8 = true; v.w_scale = sc8 + 2;
+  }
   if (c.post_norms) {
     v.out = w.tb; v.ldo = d; v.mode = 0;
     POP_TRY(launch_gemv(v, s));
@@ -337,9 +345,13 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   v = GemvArgs{};
   v.x = w.hb; v.ldx = d; v.w = lp<bf16>(m, l, m->lo.wgu); v.ldw = d; v.out = w.ab; v.ldo = c.d_ffn;
   v.B = B; v.N = 2 * m->f_pad; v.K = d; v.mode = 3; v.act = c.act; v.n_valid = c.d_ffn;
+  if (w8) { v.w = w8 + (size_t)m->qkv_dim * d; v.w_fp8 = true; v.w_scale = sc8 + 1; }
   POP_TRY(launch_gemv(v, s));
   v = GemvArgs{};
   v.x = w.ab; v.ldx = c.d_ffn; v.w = lp<bf16>(m, l, m->lo.wd); v.ldw = c.d_ffn; v.B = B; v.N = d; v.K = c.d_ffn;
+  if (w8) {
+    v.w = w8 + ((size_t)m->qkv_dim + 2 * (size_t)m->f_pad + (size_t)m->q_dim) * d; v.w_fp8 = true; v.w_scale = sc8 + 3;
+  }
   if (c.post_norms) {
     v.out = w.tb; v.ldo = d; v.mode = 0;
     POP_TRY(launch_gemv(v, s));

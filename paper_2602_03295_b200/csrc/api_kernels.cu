@@ -146,6 +146,15 @@ int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t
   return launch_gemv(v, static_cast<cudaStream_t>(stream));
 }
 
+int pop_k_gemv_e4m3(const void* x, int64_t ldx, const void* w, int64_t ldw, const float* w_scale, void* out,
+                    int64_t ldo, int32_t B, int32_t N, int32_t K, int32_t mode, int32_t act, int32_t n_valid,
+                    void* stream) {
+  GemvArgs v{};
+  v.x = x; v.ldx = ldx; v.x_f32 = false; v.w = w; v.ldw = ldw; v.w_fp8 = true; v.w_scale = w_scale;
+  v.out = out; v.ldo = ldo; v.B = B; v.N = N; v.K = K; v.mode = mode; v.act = act; v.n_valid = n_valid;
+  return launch_gemv(v, static_cast<cudaStream_t>(stream));
+}
+
 int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
                            const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
                            int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,

@@ -87,6 +87,23 @@ def test_gemm_on_codes(L, M, N, K):
         assert rel_err(out, 2 * ref) < 1e-5
 
 
+@pytest.mark.parametrize("B,N,K", [(1, 4096, 4096), (3, 520, 688 + 16), (8, 64, 256), (2, 1000, 14336)])
+def test_gemv_on_e4m3_weights(L, B, N, K):
+    g = torch.Generator().manual_seed(13)
+    x = torch.randn(B, K, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * 0.02).to(torch.bfloat16)
+    (wq,), w_s = po.quant_tensors_e4m3([w])
+    ref = (x.double() @ wq.T) * w_s
+    W8 = wq.to(torch.float32).to(torch.float8_e4m3fn).view(torch.uint8).to(DEV)
+    sb = torch.tensor([w_s], dtype=torch.float32, device=DEV)
+    out = torch.zeros(B, N, dtype=torch.float32, device=DEV)
+    L.gemv_e4m3(x.to(DEV), W8, sb, out, mode=0)
+    assert L.status() == 0
+    assert rel_err(out, ref) < 1e-4
+    L.gemv_e4m3(x.to(DEV), W8, sb, out, mode=2)
+    assert rel_err(out, 2 * ref) < 1e-4
+
+
 TINY8 = {
     "c1": ps.C1_TINY,
     "qknorm": ps.C1_TINY.replace(qk_norm=1, distinct_gains=True),
@@ -135,6 +152,28 @@ def test_kept_layers_on_fp8_operands(variant, B, N, l_keep, chunk):
         tol = 2e-2 if l == 0 else 4 * rtol
         assert rel_err(k, ref["K"][l]) <= tol and rel_err(v, ref["V"][l]) <= tol, f"layer {l + 1}"
         assert rms_rel(k, ref["K"][l]) <= rtol and rms_rel(v, ref["V"][l]) <= rtol, f"layer {l + 1} (rms)"
+    # decode steps stream the E4M3 weights with bf16 activations: from the oracle's own state (its cache
+    # written into a second paged cache) they are deterministic functions of identical inputs, so the
+    # bf16 tolerances hold again
+    if N > 1 and not chunk:
+        T = 2
+        cd = KVCache(cfg, B, N + T, 16, fill=float("nan"))
+        pos = torch.arange(N)
+        for l in range(cfg.n_layers):
+            pages = cd.block_table[:, pos // 16].long()
+            cd.k[l][pages, (pos % 16)[None, :].expand_as(pages).to(DEV)] = ref["K"][l].to(torch.bfloat16).to(DEV)
+            cd.v[l][pages, (pos % 16)[None, :].expand_as(pages).to(DEV)] = ref["V"][l].to(torch.bfloat16).to(DEV)
+        K_, V_ = [k.to(torch.bfloat16).double() for k in ref["K"]], [v.to(torch.bfloat16).double() for v in ref["V"]]
+        for t in range(T):
+            tok = ps.uniform_tokens(70 + t, B, 1, cfg.vocab)[:, 0]
+            K_, V_, lg = po.decode_step(cfg, w, tok, K_, V_, precision="fp8w")
+            lg_gpu = model.decode_step(tok.to(torch.int32).to(DEV), N + t, cd)
+            assert model.last_status() == 0
+            assert (lg_gpu.cpu().double() - lg).abs().max().item() <= 5e-2
+            for l in range(cfg.n_layers):
+                k, v = cd.gather(l, N + t + 1)
+                assert rel_err(k[:, N + t:], K_[l][:, N + t:]) <= 2e-2 and rel_err(v[:, N + t:], V_[l][:, N + t:]) <= 2e-2
+            K_, V_ = [k.to(torch.bfloat16).double() for k in K_], [v.to(torch.bfloat16).double() for v in V_]
     # it is a different function from the bf16 path (the quantisation is really there) ...
     cache16 = KVCache(cfg, B, N, 16, fill=float("nan"))
     model.enable_fp8(False)
