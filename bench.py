@@ -356,7 +356,8 @@ def run_ours(a, wl):
     barrier()
     gen_ms = max_over_ranks(d0.elapsed_time(d1), dev) / DECODE_STEPS
     dec_status = dec_status or model.last_status()
-    weight_bytes = 2.0 * (cfg.n_layers * po.layer_params(cfg) + cfg.vocab * cfg.d_model)
+    # bytes a decode step streams: bf16 weights, or E4M3 layer matrices (1 byte) and the bf16 output head
+    weight_bytes = (1.0 if fp8 else 2.0) * cfg.n_layers * po.layer_params(cfg) + 2.0 * cfg.vocab * cfg.d_model
 
     # per-kernel-class durations of one more step, CUDA events on the launching stream
     # (as many steps as the timed region, back to back, so that clocks sit where they sat there)
@@ -412,7 +413,7 @@ def run_ours(a, wl):
                         "frac": achieved_tf / peak_tf if peak_tf else None,
                         "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})"
                                        + (", fp8 launches at 2 x that (nominal ratio), flop-weighted" if fp8 else ""),
-                        "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": gemm_traffic(),
+                        "launches_per_step": gemm_n, "ms_per_step": gemm_ms, "traffic": None if fp8 else gemm_traffic(),
                         "traffic_launch": GEMM_TRAFFIC["launch"]},
            "kernel_breakdown": breakdown}
     if rank == 0 and world == 1 and not a.no_cpu_baseline:
@@ -550,13 +551,16 @@ def run_kernel(a, wl):
         bound = "hbm"
         N = wl.seq_len
         model = PopModel(cfg, ps.SynthWeights(cfg, device=dev), device=dev)
+        if a.precision == "fp8":
+            model.enable_fp8()
         cache = KVCache(cfg, wl.batch, N + 64, a.page_size, device=dev)
         tokens, embeds = ps.make_prompt(wl)
         model.prefill(tokens.to(dev), None if embeds is None else embeds.to(dev), cfg.n_layers, cache)
         tok = torch.zeros(wl.batch, dtype=torch.int32, device=dev)
         logits = torch.zeros(wl.batch, cfg.vocab, dtype=torch.float32, device=dev)
         per_layer = d * (qd + 2 * kvd) + qd * d + 3 * d * F
-        work = 2.0 * (cfg.n_layers * per_layer + cfg.vocab * d) + 4.0 * wl.batch * N * kvd * cfg.n_layers
+        wbytes = 1.0 if a.precision == "fp8" else 2.0
+        work = wbytes * cfg.n_layers * per_layer + 2.0 * cfg.vocab * d + 4.0 * wl.batch * N * kvd * cfg.n_layers
 
         def launch(i):
             model.decode_step(tok, N + i % 64, cache, logits)
