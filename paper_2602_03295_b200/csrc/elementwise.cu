@@ -118,20 +118,51 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, int64_t ldx, const f
 // x[row][:] += rmsnorm(t[row][:]) * gain      (post-norm models: norm of the sublayer output)
 __global__ void postnorm_add_kernel(float* __restrict__ x, int64_t ldx, const float* __restrict__ t, int64_t ldt,
                                     const float* __restrict__ gain, int d, float eps) {
+  // the sublayer output row stays in registers (rows up to 16 floats per thread are read once)
+  constexpr int PN_CACHE = 4;
   __shared__ float red[32];
   chain_trigger();
-  chain_wait();
   const int row = blockIdx.x;
   const float* tr = t + (int64_t)row * ldt;
   float* xr = x + (int64_t)row * ldx;
+  const int step = blockDim.x * 4;
+  float4 gv[PN_CACHE];                      // weights: loaded before the wait on the producer of t
+#pragma unroll
+  for (int i = 0; i < PN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    gv[i] = c < d ? *reinterpret_cast<const float4*>(gain + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  chain_wait();
+  float4 tv[PN_CACHE], xv[PN_CACHE];
+#pragma unroll
+  for (int i = 0; i < PN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    tv[i] = c < d ? *reinterpret_cast<const float4*>(tr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    xv[i] = c < d ? *reinterpret_cast<const float4*>(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+#pragma unroll
+  for (int i = 0; i < PN_CACHE; ++i) {
+    const float4 v = tv[i];
+    if (threadIdx.x * 4 + i * step < d) ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  for (int c = threadIdx.x * 4 + PN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(tr + c);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, red);
   const float rstd = rsqrtf(ss / (float)d + eps);
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+#pragma unroll
+  for (int i = 0; i < PN_CACHE; ++i) {
+    const int c = threadIdx.x * 4 + i * step;
+    if (c < d) {
+      const float4 v = tv[i], w = gv[i];
+      float4 o = xv[i];
+      o.x += v.x * rstd * w.x; o.y += v.y * rstd * w.y; o.z += v.z * rstd * w.z; o.w += v.w * rstd * w.w;
+      *reinterpret_cast<float4*>(xr + c) = o;
+    }
+  }
+  for (int c = threadIdx.x * 4 + PN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(tr + c);
     const float4 w = *reinterpret_cast<const float4*>(gain + c);
     float4 o = *reinterpret_cast<float4*>(xr + c);

@@ -41,20 +41,23 @@ __global__ void rmsnorm_e4m3_kernel(const float* __restrict__ x, int64_t ldx, co
   const int row = blockIdx.x;
   const float* xr = x + (int64_t)row * ldx;
   const int step = blockDim.x * 4;
-  float4 yv[QN_CACHE];                      // x * gain
+  float4 yv[QN_CACHE];                      // x, then x * gain
+  float4 gv[QN_CACHE];
   float ss = 0.f, am = 0.f;
+  // all loads first (a zero row element contributes nothing to either reduction), the arithmetic after:
+  // the eight loads of a thread are in flight together
 #pragma unroll
   for (int i = 0; i < QN_CACHE; ++i) {
     const int c = threadIdx.x * 4 + i * step;
-    if (c < d) {
-      const float4 v = *reinterpret_cast<const float4*>(xr + c);
-      const float4 g = *reinterpret_cast<const float4*>(gain + c);
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-      yv[i] = make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w);
-      am = fmaxf(am, fmaxf(fmaxf(fabsf(yv[i].x), fabsf(yv[i].y)), fmaxf(fabsf(yv[i].z), fabsf(yv[i].w))));
-    } else {
-      yv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    gv[i] = c < d ? *reinterpret_cast<const float4*>(gain + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    yv[i] = c < d ? *reinterpret_cast<const float4*>(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int i = 0; i < QN_CACHE; ++i) {
+    const float4 v = yv[i], g = gv[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    yv[i] = make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w);
+    am = fmaxf(am, fmaxf(fmaxf(fabsf(yv[i].x), fabsf(yv[i].y)), fmaxf(fabsf(yv[i].z), fabsf(yv[i].w))));
   }
   for (int c = threadIdx.x * 4 + QN_CACHE * step; c < d; c += step) {
     const float4 v = *reinterpret_cast<const float4*>(xr + c);
@@ -103,9 +106,12 @@ __global__ void __launch_bounds__(256) quant_rows_bf16_e4m3_kernel(const bf16* i
   uint4 raw[QR_CACHE];
   float am = 0.f;
 #pragma unroll
-  for (int i = 0; i < QR_CACHE; ++i) {
+  for (int i = 0; i < QR_CACHE; ++i) {           // all loads of the row first
     const int c = (i * 256 + threadIdx.x) * 8;
     raw[i] = c < d ? *reinterpret_cast<const uint4*>(ir + c) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int i = 0; i < QR_CACHE; ++i) {
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[i]);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
