@@ -453,6 +453,13 @@ def layer_params(cfg) -> int:
     return cfg.d_model * (cfg.q_dim + 2 * cfg.kv_dim) + cfg.q_dim * cfg.d_model + 3 * cfg.d_model * cfg.d_ffn
 
 
+def deep_third(n_layers: int):
+    """The pruned set the paper uses throughout (Sec. 3.3: "the last 1/3 of the layers"): the last
+    floor(L / 3) layers, as 1-based layer numbers."""
+    p = n_layers // 3
+    return set(range(n_layers - p + 1, n_layers + 1))
+
+
 def kv_param_share(cfg) -> float:
     """Share of a layer's matrix parameters held by W^K and W^V (compare Sec. 3.3's "<5%")."""
     return 2 * cfg.kv_dim * cfg.d_model / layer_params(cfg)

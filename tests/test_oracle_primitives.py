@@ -153,3 +153,38 @@ def test_cost_model_matches_the_papers_claim_where_it_holds():
     pop = po.prefill_flops(ps.C2_LLAMA8B, 1, 8192, 24)
     assert abs(full / 1e12 - 131.94) < 0.05 and abs(pop / 1e12 - 100.06) < 0.05
     assert po.attention_pairs(5, 0) == 15 and po.attention_pairs(5, 2) == 3 + 3 * 2
+
+
+def _golden():
+    import os
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "paper_values.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split("=")
+                vals[k.strip()] = float(v)
+    return vals
+
+
+def test_values_the_paper_prints():
+    import pop_synth as ps
+    g = _golden()
+    # the pruned set "last 1/3 of the layers" gives the fractions the results table prints, and the layer
+    # range the appendix names for the 36-layer model
+    for L in (32, 36, 48):
+        frac = 100.0 * len(po.deep_third(L)) / L
+        assert abs(frac - g[f"pruned_fraction_percent.{L}"]) < 0.05, L
+    s = po.deep_third(36)
+    assert min(s) == g["deep_third_first_layer.36"] and max(s) == g["deep_third_last_layer.36"]
+    assert s == set(range(25, 37))
+    # the K/V projections' share stays under the printed bound for the Llama-3 and Qwen-3 shapes
+    for cfg in (ps.C2_LLAMA8B, ps.WORKLOADS["c3"].model):
+        assert 100.0 * po.kv_param_share(cfg) < g["kv_share_upper_bound_percent"]
+    # no measured speedup can beat the ratio of algorithmic work at the same pruned set and length
+    for key, cfg in (("32", ps.C2_LLAMA8B), ("48", ps.WORKLOADS["c4"].model)):
+        L = cfg.n_layers
+        l_keep = L - len(po.deep_third(L))
+        ceiling = po.prefill_flops(cfg, 1, 2048, None) / po.prefill_flops(cfg, 1, 2048, l_keep)
+        assert ceiling > g[f"measured_speedup_2048.{key}"], (key, ceiling)
+        assert ceiling < L / l_keep + 1e-9          # and pruning p layers cannot save more than p layers' worth
