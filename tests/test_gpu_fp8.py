@@ -186,3 +186,44 @@ def test_kept_layers_on_fp8_operands(variant, B, N, l_keep, chunk):
     with pytest.raises(PopError) as e:
         model.prefill_skip(tokens.to(DEV), None, {cfg.n_layers}, cache16)
     assert e.value.code == POP_E_INVALID
+
+
+def test_argument_errors_of_the_newer_entry_points():
+    # refused before anything is enqueued: bad arena, short arena, chunk length 0, horizons beyond the position
+    import ctypes as C
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    from paper_2602_03295_b200 import PopError, POP_E_INVALID, POP_E_NOSPACE
+    cfg = ps.C1_TINY
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
+    dll = model.lib.dll
+    need = dll.pop_fp8_arena_bytes(model.handle)
+    assert need > 0
+    arena = torch.empty(need + 2048, dtype=torch.uint8, device=DEV)
+    base = (arena.data_ptr() + 1023) // 1024 * 1024
+    assert dll.pop_enable_fp8(model.handle, base + 8, need, None) == POP_E_INVALID      # misaligned
+    assert dll.pop_enable_fp8(model.handle, base, need - 1, None) == POP_E_NOSPACE
+    assert dll.pop_enable_fp8(None, base, need, None) == POP_E_INVALID
+    tokens = ps.uniform_tokens(5, 1, 40, cfg.vocab).to(DEV)
+    cache = KVCache(cfg, 1, 48, 16, fill=float("nan"))
+    with pytest.raises(PopError) as e:
+        model.prefill_chunked(tokens, None, 2, 0, cache)
+    assert e.value.code == POP_E_INVALID
+    with pytest.raises(PopError) as e:
+        model.prefill_chunked(tokens, None, cfg.n_layers + 1, 16, cache)
+    assert e.value.code == POP_E_INVALID
+    model.prefill(tokens, None, 2, cache)
+    tok = torch.zeros(1, dtype=torch.int32, device=DEV)
+    with pytest.raises(PopError) as e:
+        model.decode_step(tok, 40, cache, layer_first_pos=[0] * (cfg.n_layers - 1) + [41])
+    assert e.value.code == POP_E_INVALID
+    with pytest.raises(PopError) as e:
+        model.decode_step(tok, 40, cache, layer_first_pos=[-1] + [0] * (cfg.n_layers - 1))
+    assert e.value.code == POP_E_INVALID
+    assert model.last_status() == 0
+    inp = model._input(tokens, None)
+    kc = cache.struct()
+    logits = torch.zeros(1, cfg.vocab, dtype=torch.float32, device=DEV)
+    mask = bytes([0] * (cfg.n_layers - 1) + [1])
+    assert dll.pop_prefill_ablation(model.handle, C.byref(inp), 40, 1, mask, 4, C.byref(kc), logits.data_ptr(),
+                                    None) == POP_E_INVALID                                # unknown flag bit
+    assert (logits == 0).all()
