@@ -144,14 +144,15 @@ int pop_prefill_skip(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_
  * second precision, off by default. pop_enable_fp8 writes E4M3 copies of those weight matrices (one
  * scale per matrix) into dev_arena (caller's device memory, 1024-byte aligned, at least
  * pop_fp8_arena_bytes(m); it must stay valid while enabled; d_model, q_dim, d_ffn multiples of 16 and
- * q_dim, d_ffn <= 16384, POP_E_INVALID otherwise). While enabled, pop_prefill, pop_full_prefill and
- * pop_prefill_chunked turn the rows entering those projections into E4M3 codes with one scale per
- * row (the normalised rows straight from the norm, the stored bf16 attention output and gated
- * activation in place) and run the four GEMMs on the codes (fp32 accumulation; scales applied to
- * the accumulator before the usual epilogue). The single-position passes -- the boundary token's
- * deep layers, pop_decode_step, pop_generate_greedy -- stream the E4M3 weights (half the bytes) and
- * keep bf16 activations. Attention and the pruned layers' Eq. 14 projections keep bf16 operands. pop_prefill_ragged, pop_prefill_skip
- * and pop_prefill_ablation return POP_E_INVALID while it is enabled. dev_arena = NULL disables it. */
+ * q_dim, d_ffn <= 16384, POP_E_INVALID otherwise). While enabled, pop_prefill, pop_full_prefill,
+ * pop_prefill_chunked and pop_prefill_ragged turn the rows entering those projections into E4M3
+ * codes with one scale per row (the normalised rows straight from the norm, the stored bf16
+ * attention output and gated activation in place) and run the four GEMMs on the codes (fp32
+ * accumulation; scales applied to the accumulator before the usual epilogue). The single-position
+ * passes -- the boundary token's deep layers, pop_decode_step, pop_generate_greedy -- stream the
+ * E4M3 weights (half the bytes) and keep bf16 activations. Attention and the pruned layers' Eq. 14
+ * projections keep bf16 operands. pop_prefill_skip and pop_prefill_ablation (the literal two-phase
+ * evaluation) return POP_E_INVALID while it is enabled. dev_arena = NULL disables it. */
 size_t pop_fp8_arena_bytes(const pop_model_t* m);
 int pop_enable_fp8(pop_model_t* m, void* dev_arena, size_t bytes, void* stream);
 

@@ -467,7 +467,6 @@ int run_prefill_ragged(pop_model* m, const pop_input_t* in, const int32_t* seq_l
                        pop_kv_cache_t* kc, float* logits, cudaStream_t s) {
   if (!m || !in || !in->tokens || !seq_lens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
     return POP_E_INVALID;
-  if (m->fp8) return POP_E_INVALID;   // FP8 operands: pop_prefill, pop_full_prefill and pop_prefill_chunked only
   const pop_config_t& c = m->cfg;
   if (B < 1 || B > 4096 || L_keep < 1 || L_keep > c.n_layers) return POP_E_INVALID;
   std::vector<int32_t> cu(B + 1, 0);
@@ -528,7 +527,7 @@ int run_prefill_skip(pop_model* m, const pop_input_t* in, int N, int B, const ui
   const bool boundary = !(flags & POP_NO_BOUNDARY), indep_kv = !(flags & POP_NO_INDEP_KV);
   if (!m || !in || !in->tokens || !skip || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
     return POP_E_INVALID;
-  if (m->fp8) return POP_E_INVALID;   // FP8 operands: pop_prefill, pop_full_prefill and pop_prefill_chunked only
+  if (m->fp8) return POP_E_INVALID;   // FP8 operands: not in the literal two-phase evaluation
   const pop_config_t& c = m->cfg;
   if (N < 1 || B < 1 || (int64_t)N * B > (int64_t)1 << 24) return POP_E_INVALID;
   if (!page_size_ok(kc->page_size) || kc->num_pages < 1) return POP_E_INVALID;

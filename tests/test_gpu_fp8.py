@@ -188,6 +188,32 @@ def test_kept_layers_on_fp8_operands(variant, B, N, l_keep, chunk):
     assert e.value.code == POP_E_INVALID
 
 
+def test_ragged_batch_on_fp8_operands():
+    # row scales are per packed row, so packing changes nothing: every sequence equals the oracle's FP8
+    # run on that sequence alone (tolerances as in test_kept_layers_on_fp8_operands)
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    cfg = TINY8["qknorm"]
+    lens, l_keep = [1, 17, 130, 64], 2
+    w = ps.SynthWeights(cfg)
+    seqs = [ps.uniform_tokens(50 + i, 1, n, cfg.vocab) for i, n in enumerate(lens)]
+    packed = torch.cat([t[0] for t in seqs]).contiguous()
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
+    model.enable_fp8()
+    cache = KVCache(cfg, len(lens), max(lens), 16, fill=float("nan"))
+    logits = model.prefill_ragged(packed.to(DEV), None, lens, l_keep, cache)
+    assert model.last_status() == 0 and not torch.isnan(logits).any()
+    for b, (t, n) in enumerate(zip(seqs, lens)):
+        ref = po.pop_prefill(cfg, w, t, None, l_keep, precision="kernel", fp8_kept=True)
+        assert (logits[b].cpu().double() - ref["logits"][0]).abs().max().item() <= 3e-1, f"seq {b}"
+        for l in range(cfg.n_layers):
+            k, v = cache.gather(l, n)
+            tol = 2e-2 if l == 0 else 4 * min(3e-2 * (4 * l) ** 0.5, 1e-1)
+            assert rel_err(k[b], ref["K"][l][0]) <= tol and rel_err(v[b], ref["V"][l][0]) <= tol, (b, l)
+            if n < max(lens):
+                kk, _ = cache.gather(l, max(lens))
+                assert torch.isnan(kk[b, n:].float()).all()
+
+
 def test_argument_errors_of_the_newer_entry_points():
     # refused before anything is enqueued: bad arena, short arena, chunk length 0, horizons beyond the position
     import ctypes as C
