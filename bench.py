@@ -498,9 +498,11 @@ def run_kernel(a, wl):
         x = rnd(M, d, dtype=torch.float32)
         gain = torch.ones(d, dtype=torch.float32, device=dev)
         work = 5.0 * M * d
+        codes = torch.empty(M, d, dtype=torch.uint8, device=dev)
+        scales = torch.empty(M, dtype=torch.float32, device=dev)
 
         def launch(i):
-            lib.rmsnorm_e4m3(x, gain, cfg.rms_eps)
+            lib.rmsnorm_e4m3(x, gain, cfg.rms_eps, out=codes, scale=scales)
     elif k in ("attention", "attention_local"):
         from paper_2602_03295_b200.binding import KVCache
         window = cfg.window if k == "attention_local" else 0

@@ -188,11 +188,13 @@ class PopLibrary:
         self.check(code, "pop_k_gemv_e4m3")
         return out
 
-    def rmsnorm_e4m3(self, x, gain, eps, stream=None):
-        """pop_k_rmsnorm_e4m3: returns (codes uint8 [rows, d], scale fp32 [rows])."""
+    def rmsnorm_e4m3(self, x, gain, eps, stream=None, out=None, scale=None):
+        """pop_k_rmsnorm_e4m3: returns (codes uint8 [rows, d], scale fp32 [rows]); out / scale may be given."""
         rows, d = x.shape
-        out = torch.empty(rows, d, dtype=torch.uint8, device=x.device)
-        scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+        if out is None:
+            out = torch.empty(rows, d, dtype=torch.uint8, device=x.device)
+        if scale is None:
+            scale = torch.empty(rows, dtype=torch.float32, device=x.device)
         code = self.dll.pop_k_rmsnorm_e4m3(x.data_ptr(), x.stride(0), gain.data_ptr(), out.data_ptr(), out.stride(0),
                                            scale.data_ptr(), rows, d, eps, _stream_ptr(stream))
         self.check(code, "pop_k_rmsnorm_e4m3")
