@@ -11,6 +11,7 @@ namespace {
 
 constexpr int GEMV_MAXB = 8;     // rows (sequences) handled per pass
 constexpr int GEMV_R = 2;        // weight rows per warp
+constexpr int GEMV_RG = 1;       // gated form: gate rows per warp (each with its up row)
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -65,7 +66,7 @@ struct GemvDev {
   int act, n_valid;
 };
 
-// Each warp owns GEMV_R weight rows (mode 3: GEMV_R gate rows and their up rows) and streams them
+// Each warp owns GEMV_R weight rows (mode 3: GEMV_RG gate rows and their up rows) and streams them
 // once with 16-byte loads, GEMV_U k-steps (8 or 16 loads per lane) in flight at a time; the few
 // activation rows come through L1. NB = activation rows handled (1, 2, 4 or 8).
 constexpr int GEMV_U = 4;
@@ -96,7 +97,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   const int wic = threadIdx.x >> 5;                         // warp in CTA
   const int slice = wic % KS;
   const int warp = blockIdx.x * ((blockDim.x >> 5) / KS) + wic / KS;   // row group
-  constexpr int R = GEMV_R;
+  constexpr int R = GATED ? GEMV_RG : GEMV_R;
   constexpr int RW = GATED ? 2 * R : R;           // weight rows streamed per warp
   const int n_out = GATED ? p.N / 2 : p.N;        // logical output rows
   const int o0 = warp * R;
@@ -567,7 +568,7 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
   const int el = a.w_fp8 ? 16 : 8;
   if (a.mode == 3 && (a.N % 256 || a.n_valid > a.N / 2)) return POP_E_INVALID;
   const int n_out = a.mode == 3 ? a.N / 2 : a.N;
-  const int warps = ceil_div(n_out, GEMV_R);
+  const int warps = ceil_div(n_out, a.mode == 3 ? GEMV_RG : GEMV_R);
   // split K between the warps of a CTA while all warps still fit on the GPU at once (148 SMs x 64)
   int ks = 1;
   while (ks < 8 && warps * ks * 2 <= 148 * 64 && a.K >= 32 * el * ks * 2) ks *= 2;
