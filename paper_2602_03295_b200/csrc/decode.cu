@@ -569,9 +569,10 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
   if (a.mode == 3 && (a.N % 256 || a.n_valid > a.N / 2)) return POP_E_INVALID;
   const int n_out = a.mode == 3 ? a.N / 2 : a.N;
   const int warps = ceil_div(n_out, a.mode == 3 ? GEMV_RG : GEMV_R);
-  // split K between the warps of a CTA while all warps still fit on the GPU at once (148 SMs x 64)
+  // split K between the warps of a CTA while the warps of the doubled split still fit 1.5 times the
+  // GPU's resident warps (148 SMs x 64; 1 and 2 measured slower on the decode step)
   int ks = 1;
-  while (ks < 8 && warps * ks * 2 <= 148 * 64 && a.K >= 32 * el * ks * 2) ks *= 2;
+  while (ks < 8 && warps * ks * 4 <= 148 * 64 * 3 && a.K >= 32 * el * ks * 2) ks *= 2;
   const int elt = a.x_f32 ? 4 : 2;
   for (int b0 = 0; b0 < a.B; b0 += GEMV_MAXB) {
     GemvDev p;
