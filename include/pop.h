@@ -15,8 +15,13 @@
  *     The library borrows it; it allocates no device memory of its own and frees none.
  *   - `stream` is a cudaStream_t passed as void*. Calls enqueue work on it and return without
  *     synchronising (pop_last_status is the exception).
- *   - Return value: POP_OK (0) or a negative pop_status code. A call that returns an error has
- *     enqueued nothing and written nothing.
+ *   - Return value: POP_OK (0) or a negative pop_status code. Arguments are checked before the first
+ *     launch: POP_E_INVALID and POP_E_NOSPACE mean nothing was enqueued and nothing written. POP_E_CUDA
+ *     (a launch or runtime call failed part-way) may leave earlier kernels of the call queued; the
+ *     outputs are then undefined.
+ *   - One device per process: the library caches per-process launch attributes and the address of its
+ *     device status word for the device that is current at the first call. Replicas on several GPUs
+ *     run as one process per GPU.
  *   - Matrices are row-major bf16 [out_features, in_features] (y = x W^T). Norm gains are fp32.
  *   - Sequences of a batch have equal length; positions are 0-based.
  */
@@ -81,7 +86,10 @@ typedef struct {
 
 /* Prompt. tokens: device int32 [batch][seq_len]. embeds: device bf16 [batch][seq_len][d_model] or
  * NULL; when given, a position whose token id is negative takes its input row from embeds (visual
- * or other pre-computed embeddings) instead of the embedding table. */
+ * or other pre-computed embeddings) instead of the embedding table. Token ids live on the device, so
+ * the host cannot check them: an id >= vocab, or a negative id while embeds is NULL, makes that
+ * position's input a row of zeros, raises the device status word to POP_E_INVALID (the remaining
+ * kernels of the call return without computing) and is reported by pop_last_status. */
 typedef struct {
   const int32_t* tokens;
   const void* embeds;
@@ -119,8 +127,8 @@ int pop_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq
 int pop_full_prefill(pop_model_t* m, const pop_input_t* tokens_or_embeds, int32_t seq_len, int32_t batch,
                      pop_kv_cache_t* kv_cache_out, float* logits_out, void* stream);
 
-/* pop_prefill for a batch of sequences of DIFFERENT lengths (the paper batches real prompts, Sec. 4.1 /
- * App. C; padding is not part of the method, so none is used): the sequences are packed back to
+/* pop_prefill for a batch of sequences of DIFFERENT lengths (the paper batches real prompts, Sec. 4.3:
+ * batch 8; padding is not part of the method, so none is used): the sequences are packed back to
  * back, tokens_or_embeds->tokens is device int32 [sum of lengths] (embeds, if given, device bf16
  * [sum of lengths][d_model]), seq_lens is a HOST array of `batch` lengths (each >= 1). Sequence b
  * uses row b of the block table and gets seq_lens[b] cache entries in every layer; its boundary
@@ -168,13 +176,13 @@ int pop_prefill_chunked(pop_model_t* m, const pop_input_t* tokens_or_embeds, int
                         int32_t L_keep, int32_t chunk_len, pop_kv_cache_t* kv_cache_out, float* logits_out,
                         void* stream);
 
-/* The two component ablations of the paper's Sec. 4.4.1 ("Effectiveness of Design Choices") on top
+/* The two component ablations of the paper's Sec. 4.4.1 (the design-choice ablation table) on top
  * of pop_prefill_skip; flags is a combination of
- *   POP_NO_BOUNDARY  "w/o Boundary Handling": the last prompt token is processed by the pruned
+ *   POP_NO_BOUNDARY  no boundary handling: the last prompt token is processed by the pruned
  *                    prefill model like every other position (pruned layers store their Eq. 14
  *                    projections for all seq_len positions, there is no full-depth pass for the last
  *                    token) and logits_out comes from the state that leaves the pruned model there;
- *   POP_NO_INDEP_KV  "w/o Indep. KV Proj.": pruned layers generate no cache entries for the prompt
+ *   POP_NO_INDEP_KV  no independent KV projections: pruned layers generate no cache entries for the prompt
  *                    (their rows of positions 0..seq_len-2 are left untouched); in the last token's
  *                    full-depth pass such a layer attends to position seq_len-1 only. Later decode
  *                    steps must keep that horizon: use pop_decode_step_from.
@@ -189,14 +197,14 @@ int pop_prefill_ablation(pop_model_t* m, const pop_input_t* tokens_or_embeds, in
 /* pop_decode_step with an attention horizon per layer: layer_first_pos is a HOST array of n_layers
  * int32; layer l attends to cache positions layer_first_pos[l-1] .. pos only (and within its window,
  * if it has one). After pop_prefill_ablation(POP_NO_INDEP_KV) on seq_len = N tokens the pruned layers
- * take N-1 (N if POP_NO_BOUNDARY was set as well: they then hold nothing of the prompt), the others 0 (paper Sec. 4.4.1: the model "can only access the last input token and the
- * generated tokens" in those layers). NULL = pop_decode_step. POP_E_INVALID if an entry is negative
+ * take N-1 (N if POP_NO_BOUNDARY was set as well: they then hold nothing of the prompt), the others 0
+ * (paper Sec. 4.4.1: in those layers only the last prompt token and the generated tokens are visible). NULL = pop_decode_step. POP_E_INVALID if an entry is negative
  * or beyond pos. */
 int pop_decode_step_from(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch,
                          const int32_t* layer_first_pos, pop_kv_cache_t* kv_cache, float* logits_out, void* stream);
 
-/* One decode step of the FULL model over the cache a prefill left (paper Sec. 2.2, decode stage;
- * Sec. 3: "retaining the full model for decode"): tokens is device int32 [batch], the token of
+/* One decode step of the FULL model over the cache a prefill left (the decode stage D of paper
+ * Sec. 3.2, Eq. 11, which Sec. 3.3 keeps at full depth): tokens is device int32 [batch], the token of
  * each sequence at position `pos` = number of entries its cache already holds. Every layer
  * appends its k, v at `pos` (Eq. 2-3), attends over positions 0..pos (the window in local
  * layers), and logits_out (device fp32 [batch][vocab]) receives the next-token logits. After
@@ -206,7 +214,7 @@ int pop_decode_step_from(pop_model_t* m, const int32_t* tokens, int32_t pos, int
 int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t batch, pop_kv_cache_t* kv_cache,
                     float* logits_out, void* stream);
 
-/* Greedy generation on the device (the decode stage of paper Sec. 2.2 run as a loop): starting from
+/* Greedy generation on the device (the decode stage of paper Sec. 3.2, Eq. 11, run as a loop): starting from
  * first_tokens (device int32 [batch], the token of each sequence at position pos0 -- normally the
  * arg-max of the prefill's logits), n_steps times: one full-model decode step as pop_decode_step,
  * then the arg-max of its logits (lowest index among equal values) becomes the next token.
@@ -220,8 +228,23 @@ int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t 
 int pop_generate_greedy(pop_model_t* m, const int32_t* first_tokens, int32_t pos0, int32_t n_steps, int32_t batch,
                         pop_kv_cache_t* kv_cache, int32_t* tokens_out, float* logits_scratch, void* stream);
 
-/* Synchronise `stream`, then read and clear the device status word: POP_OK, or
- * POP_E_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or POP_E_CUDA. */
+/* The hidden states the last pop_prefill / pop_full_prefill call with the same (seq_len, batch) left in
+ * the workspace, copied out on `stream` (either pointer may be NULL, not both):
+ *   hidden_out  device fp32 [batch][seq_len][d_model]: the residual stream leaving the last layer that
+ *               ran over the whole prompt. After pop_prefill this is x_{L_keep+1}; its rows 0..seq_len-2
+ *               are the state H every pruned layer projects (paper Eq. 14) and hands on unchanged
+ *               (Eq. 15). After pop_full_prefill it is x_{L+1} of Eq. 1.
+ *   last_out    device fp32 [batch][d_model]: the last prompt position after ALL n_layers layers (the
+ *               boundary token's state, paper Sec. 3.3), i.e. the input of the final norm.
+ * Meaningful only until the next call that uses the workspace. Errors: POP_E_INVALID, POP_E_NOSPACE
+ * (no workspace, or one too small for these sizes), POP_E_CUDA. */
+int pop_read_hidden(pop_model_t* m, int32_t seq_len, int32_t batch, float* hidden_out, float* last_out,
+                    void* stream);
+
+/* Synchronise `stream`, then read and clear the device status word: POP_OK, POP_E_DEVICE_TIMEOUT if
+ * a kernel gave up on a bounded wait, POP_E_INVALID if a kernel met an unusable token id, or
+ * POP_E_CUDA. Once the word is raised the library's GEMM and attention kernels return at once, so
+ * the outputs of that call (and of calls queued behind it) are undefined until it is read. */
 int pop_last_status(pop_model_t* m, void* stream);
 
 /* Number of kernel launches the last prefill call on this model enqueued. */

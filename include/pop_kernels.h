@@ -168,6 +168,16 @@ int pop_k_decode_attention_static(const void* q, int64_t ldq, const void* k_pool
 /* Synchronise the stream, then read and clear the library's device status word. */
 int pop_k_status(void* stream);
 
+/* Self-test of the library's failure path (no counterpart in the paper). Every device-side wait of
+ * the GEMM and attention kernels (on an mbarrier that a TMA copy or a tensor-core commit completes)
+ * is bounded: when it runs out, the kernel raises the status word to POP_E_DEVICE_TIMEOUT, unwinds and
+ * returns, and kernels launched while the word is raised return at once. This call launches one small
+ * kernel that performs that very wait on a barrier nothing arrives at, for at most limit_cycles SM
+ * cycles (1 .. 1 000 000, i.e. well under a millisecond; POP_E_INVALID otherwise), so the path can be
+ * exercised without a fault, a trap or an endless loop: afterwards pop_k_status returns
+ * POP_E_DEVICE_TIMEOUT once and POP_OK from then on. */
+int pop_k_wait_selftest(int64_t limit_cycles, void* stream);
+
 /* Per-kernel timing for benchmarks. pop_k_profile(1) makes every launch of this library record a
  * CUDA-event pair on its stream; pop_k_profile_summary waits for the recorded events of one kind
  * (0 projection GEMM, 1 prefill attention, 2 elementwise, 3 GEMV, 4 decode attention), returns

@@ -54,11 +54,13 @@ import torch
 # ---------------------------------------------------------------------------------------
 
 def _rnd(x: torch.Tensor, precision: str) -> torch.Tensor:
-    """Identity in "exact" mode; otherwise ("kernel": bf16 operands; "fp8": E4M3 operands for the four
+    """Identity in "exact" mode; otherwise ("bf16ops": bf16 operands; "fp8": E4M3 operands for the four
     projections of a layer; "fp8w": E4M3 weights of those projections, bf16 activations; bf16 for
     attention and everything stored in all three) round to bf16 and back."""
     if precision == "exact":
         return x
+    if precision not in ("bf16ops", "fp8", "fp8w"):
+        raise ValueError(f"unknown precision {precision!r}")
     return x.to(torch.float32).to(torch.bfloat16).to(x.dtype)
 
 
@@ -308,8 +310,8 @@ def lm_logits(cfg, weights, x_last: torch.Tensor, dtype) -> torch.Tensor:
 
 def full_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tensor] = None,
                  dtype=torch.float64, precision: str = "exact", n_layers: Optional[int] = None):
-    """Standard prefill of the unpruned model over x_{1:N} (Sec. 3.3, "standard inference
-    pipeline"). tokens: int [B, N]; embeds: [B, N, d] or None.
+    """Standard prefill of the unpruned model over x_{1:N} (Sec. 3.3, the ordinary
+    pipeline POP is compared with). tokens: int [B, N]; embeds: [B, N, d] or None.
 
     Returns dict: K, V lists over layers of [B, N, n_kv, hd]; logits [B, vocab];
     hidden [B, N, d] = the state leaving the last evaluated layer."""
@@ -348,10 +350,10 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     layer-selection ablation of Sec. 4.4). A pruned layer projects whatever state reaches it.
 
     The two component ablations of Sec. 4.4.1 (Table "design choices"):
-      boundary=False ("w/o Boundary Handling"): x_N is processed by the pruned prefill model like
+      boundary=False (the row without boundary handling): x_N is processed by the pruned prefill model like
         every other position: phase 1 covers all N positions, there is no phase 2, and the logits
         come from the state that leaves phase 1 at position N.
-      indep_kv=False ("w/o Indep. KV Proj."): pruned layers generate no cache entries in phase 1;
+      indep_kv=False (the row without independent KV projections): pruned layers generate no cache entries in phase 1;
         in phase 2 (and in later decode steps) such a layer can only attend to positions >= N.
         Their K, V rows of positions 1..N-1 are returned as NaN ("absent").
 
@@ -364,7 +366,8 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     H [B, N-1, d] (the state leaving the last layer of phase 1 at positions 1..N-1; for the
     deep-suffix set this is the state leaving the kept stack), first_pos (per layer, 0-based: the
     first cache position later decode steps may attend to: 0, or for pruned layers when
-    indep_kv is off N-1, the entry phase 2 wrote -- N if there was no phase 2 either)."""
+    indep_kv is off N-1, the entry phase 2 wrote -- N if there was no phase 2 either),
+    x_last [B, d] (the state of x_N that enters the final norm)."""
     L = cfg.n_layers
     if skip is None:
         assert 1 <= l_keep <= L
@@ -376,6 +379,7 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
     V = [torch.empty(B, N, cfg.n_kv_heads, cfg.head_dim, dtype=dtype) for _ in range(L)]
     H = torch.empty(B, max(N - 1, 0), cfg.d_model, dtype=dtype)
     logits = torch.empty(B, cfg.vocab, dtype=dtype)
+    x_out = torch.empty(B, cfg.d_model, dtype=dtype)
     for b in range(B):
         x_all = embed(cfg, weights, tokens[b], None if embeds is None else embeds[b], dtype)
         kc = [None] * L
@@ -413,18 +417,19 @@ def pop_prefill(cfg, weights, tokens: torch.Tensor, embeds: Optional[torch.Tenso
                 V[l][b, :absent] = float("nan")
                 K[l][b, absent:], V[l][b, absent:] = kc[l], vc[l]
         logits[b] = lm_logits(cfg, weights, x_last, dtype)
+        x_out[b] = x_last
     horizon = N - 1 if boundary else N           # without phase 2 a pruned layer holds nothing at all
     first_pos = [horizon if (not indep_kv and (l + 1) in skip) else 0 for l in range(L)]
-    return {"K": K, "V": V, "logits": logits, "H": H, "first_pos": first_pos}
+    return {"K": K, "V": V, "logits": logits, "H": H, "first_pos": first_pos, "x_last": x_out}
 
 
 def decode_step(cfg, weights, tokens: torch.Tensor, K, V, dtype=torch.float64, precision: str = "exact",
                 first_pos=None):
-    """One decode step of the FULL model over an existing cache (Sec. 2.2, decode stage; Eq. 1-3):
-    POP prunes nothing here ("retaining the full model for decode"). tokens: int [B], the token at
+    """One decode step of the FULL model over an existing cache (the decode stage D of Sec. 3.2, Eq. 11, kept at full depth by Sec. 3.3; Eq. 1-3):
+    POP prunes nothing in this stage. tokens: int [B], the token at
     position n = current cache length; K, V: lists (one per layer) of [B, n, n_kv, hd].
     first_pos (per layer, 0-based) is the first cache position a layer may attend to: positions
-    before it hold nothing (the "w/o Indep. KV Proj." ablation of Sec. 4.4.1).
+    before it hold nothing (the ablation without independent KV projections, Sec. 4.4.1).
     Returns (K', V', logits): caches with n + 1 entries and the next-token logits [B, vocab]."""
     L = cfg.n_layers
     B = tokens.shape[0]
@@ -454,7 +459,7 @@ def layer_params(cfg) -> int:
 
 
 def deep_third(n_layers: int):
-    """The pruned set the paper uses throughout (Sec. 3.3: "the last 1/3 of the layers"): the last
+    """The pruned set the paper uses throughout (Sec. 3.3: the deepest third of the layers): the last
     floor(L / 3) layers, as 1-based layer numbers."""
     p = n_layers // 3
     return set(range(n_layers - p + 1, n_layers + 1))

@@ -76,6 +76,7 @@ SIGNATURES = {
     "pop_decode_step": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_decode_step_from": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_I32), C.POINTER(pop_kv_cache_t), _P, _P]),
     "pop_generate_greedy": (C.c_int, [_P, _P, _I32, _I32, _I32, C.POINTER(pop_kv_cache_t), _P, _P, _P]),
+    "pop_read_hidden": (C.c_int, [_P, _I32, _I32, _P, _P, _P]),
     "pop_last_status": (C.c_int, [_P, _P]),
     "pop_last_launch_count": (_I64, [_P]),
     "pop_free": (None, [_P]),
@@ -102,6 +103,7 @@ SIGNATURES = {
     "pop_k_profile": (None, [_I32]),
     "pop_k_profile_summary": (C.c_int, [_I32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_I64)]),
     "pop_k_status": (C.c_int, [_P]),
+    "pop_k_wait_selftest": (C.c_int, [_I64, _P]),
     "pop_k_launch_count": (_I64, []),
     "pop_k_reset_launch_count": (None, []),
 }
@@ -138,6 +140,10 @@ class PopLibrary:
 
     def status(self, stream=None) -> int:
         return self.dll.pop_k_status(_stream_ptr(stream))
+
+    def wait_selftest(self, limit_cycles: int = 200000, stream=None):
+        """Launch the bounded-wait self-test kernel (raises the status word to POP_E_DEVICE_TIMEOUT)."""
+        self.check(self.dll.pop_k_wait_selftest(limit_cycles, _stream_ptr(stream)), "pop_k_wait_selftest")
 
     def launch_count(self) -> int:
         return self.dll.pop_k_launch_count()
@@ -587,6 +593,15 @@ class PopModel:
                                                 out.data_ptr(), logits.data_ptr(), _stream_ptr(stream))
         self.lib.check(code, "pop_generate_greedy")
         return out, logits
+
+    def read_hidden(self, seq_len: int, batch: int, stream=None):
+        """(hidden fp32 [B, N, d], last fp32 [B, d]) left in the workspace by the last prefill of this shape."""
+        hidden = torch.empty(batch, seq_len, self.cfg.d_model, dtype=torch.float32, device=self.device)
+        last = torch.empty(batch, self.cfg.d_model, dtype=torch.float32, device=self.device)
+        code = self.lib.dll.pop_read_hidden(self.handle, seq_len, batch, hidden.data_ptr(), last.data_ptr(),
+                                            _stream_ptr(stream))
+        self.lib.check(code, "pop_read_hidden")
+        return hidden, last
 
     def last_status(self, stream=None) -> int:
         return self.lib.dll.pop_last_status(self.handle, _stream_ptr(stream))

@@ -588,7 +588,7 @@ int decode_body(pop_model* m, const Workspace& w, const int32_t* tokens, int pos
   return launch_gemv(v, s);
 }
 
-// One decode step of the full model (paper Sec. 2.2): every sequence's token at position `pos`
+// One decode step of the full model (the decode stage of paper Sec. 3.2, Eq. 11): every sequence's token at position `pos`
 // (= entries already in the cache) goes through all L layers as the boundary token does.
 int run_decode(pop_model* m, const int32_t* tokens, int pos, int B, pop_kv_cache_t* kc, float* logits,
                cudaStream_t s, const int32_t* layer_first_pos = nullptr) {
@@ -899,6 +899,22 @@ int pop_generate_greedy(pop_model_t* m, const int32_t* first_tokens, int32_t pos
                         pop_kv_cache_t* kv_cache, int32_t* tokens_out, float* logits_scratch, void* stream) {
   return run_generate(m, first_tokens, pos0, n_steps, batch, kv_cache, tokens_out, logits_scratch,
                       static_cast<cudaStream_t>(stream));
+}
+
+int pop_read_hidden(pop_model_t* m, int32_t seq_len, int32_t batch, float* hidden_out, float* last_out,
+                    void* stream) {
+  if (!m || seq_len < 1 || batch < 1 || (!hidden_out && !last_out)) return POP_E_INVALID;
+  if (!m->ws) return POP_E_NOSPACE;
+  const Workspace w = carve(m, (char*)m->ws, seq_len, batch);
+  if (w.total > m->ws_bytes) return POP_E_NOSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t d = m->cfg.d_model;
+  if (hidden_out && cudaMemcpyAsync(hidden_out, w.x, (size_t)batch * seq_len * d * 4, cudaMemcpyDeviceToDevice, s) !=
+                        cudaSuccess)
+    return POP_E_CUDA;
+  if (last_out && cudaMemcpyAsync(last_out, w.xb, (size_t)batch * d * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return POP_E_CUDA;
+  return POP_OK;
 }
 
 int pop_last_status(pop_model_t* m, void* stream) {

@@ -30,12 +30,22 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // ------------------------------------------------------------------------------ embedding
+// A token id the host cannot see may be unusable: negative with no embedding rows supplied, or
+// >= vocab. Such a row becomes zeros, nothing is dereferenced for it, and the status word is raised
+// to POP_E_INVALID (the kernels queued behind then return at once; the caller reads the word).
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const bf16* __restrict__ table,
-                             const bf16* __restrict__ embeds, float* __restrict__ x, int d, int vocab) {
+                             const bf16* __restrict__ embeds, float* __restrict__ x, int d, int vocab,
+                             int* __restrict__ status) {
   const int row = blockIdx.x;
   const int tok = tokens[row];
-  const bf16* src = (tok >= 0) ? table + (int64_t)min(tok, vocab - 1) * d : embeds + (int64_t)row * d;
   float* dst = x + (int64_t)row * d;
+  if ((tok < 0 && embeds == nullptr) || tok >= vocab) {
+    if (threadIdx.x == 0) atomicMin(status, (int)POP_E_INVALID);
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4)
+      *reinterpret_cast<float4*>(dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    return;
+  }
+  const bf16* src = (tok >= 0) ? table + (int64_t)tok * d : embeds + (int64_t)row * d;
   for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
     const uint4 raw = *reinterpret_cast<const uint4*>(src + c);
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
@@ -334,8 +344,10 @@ __global__ void bump_counters_kernel(int32_t* c) { c[0] += 1; c[1] += 1; }
 int launch_embed(const int32_t* tokens, const bf16* table, const bf16* embeds, float* x, int rows, int d, int vocab,
                  cudaStream_t s) {
   if (d % 8) return POP_E_INVALID;
+  int* status = status_word();
+  if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_ELEMENTWISE, (double)rows * d * 6, s);
-  embed_kernel<<<rows, 256, 0, s>>>(tokens, table, embeds, x, d, vocab);
+  embed_kernel<<<rows, 256, 0, s>>>(tokens, table, embeds, x, d, vocab, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
 }

@@ -13,6 +13,8 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#include <cstdlib>
+
 namespace pop {
 namespace {
 
@@ -210,6 +212,141 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
   }
 }
 
+// Epilogue of one 128-row x 256-column accumulator slab held in this CTA's TMEM: the calling warp
+// (TMEM lane quarter `quarter`) owns rows row0 + quarter*32 .. +31, one row per lane. `n` is the
+// 256-column tile index, `boxes` the warp's two 32 x 32 fp32 staging boxes for TMA stores.
+template <int EPI, int HD, bool FP8>
+__device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMap& tmO, uint8_t* boxes,
+                                              uint32_t taddr, int g, int row0, int n, int quarter, int lane,
+                                              uint32_t& boxes_out) {
+  const int row = row0 + quarter * 32 + lane;
+  const bool row_ok = row < p.M;
+  // rows of a folded RMSNorm arrive un-normalised: their scale comes from the producer's sums
+  float rs = 1.0f;
+  if (p.ss_in != nullptr && row_ok) {
+    float sum = 0.f;
+    for (int i = 0; i < p.ss_cnt; ++i) sum += p.ss_in[(int64_t)row * p.ss_in_ld + i];
+    rs = rsqrtf(sum * p.inv_d + p.eps_in);
+  }
+  if (FP8 && row_ok) rs = p.a_scale[row] * *p.b_scale;     // codes -> values: row scale x matrix scale
+  if (EPI == EPI_QKV_ROPE) {
+    qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok, rs);
+  } else if (EPI == EPI_GATED_BF16) {
+    bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t gr[32], ur[32];
+      tmem_ld_32x32b_x32(taddr + c * 32, gr);
+      tmem_ld_32x32b_x32(taddr + 128 + c * 32, ur);
+      tmem_wait_ld();
+      const int col0 = n * 128 + c * 32;
+      if (row_ok) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          if (col0 + v * 8 + 8 <= p.n_valid) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int e = v * 8 + j * 2;
+              const float x0 = act_fn(__uint_as_float(gr[e]) * rs, p.act) * (__uint_as_float(ur[e]) * rs);
+              const float x1 = act_fn(__uint_as_float(gr[e + 1]) * rs, p.act) * (__uint_as_float(ur[e + 1]) * rs);
+              w[j] = pack_bf16(x0, x1);
+            }
+            *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  } else if ((EPI == EPI_ADD_F32 || EPI == EPI_STORE_F32) && p.hn_out == nullptr) {
+    // fp32 outputs leave through shared memory: the thread writes its 32 values of the chunk as one
+    // 128-byte swizzled row of the warp's 32 x 32 box, and an elected lane hands the box to the TMA
+    // engine, which stores it or adds it to the residual at the memory side. No residual value
+    // is read by the SM, rows and columns beyond the output are clipped by the hardware.
+    const bool rows_in = row0 + quarter * 32 < p.M;     // uniform per warp
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      if (n * BN + c * 32 >= p.N) break;                 // uniform: the rest of the tile is past the last column
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(taddr + c * 32, r);
+      tmem_wait_ld();
+      if (!rows_in) continue;
+      // boxes alternate by the count of boxes handed over, so "at most one group still reading"
+      // always means the other box
+      uint8_t* box = boxes + (boxes_out & 1) * OUT_STAGE_BYTES;
+      ++boxes_out;
+      if (lane == 0) bulk_wait_read_1();
+      __syncwarp();
+      uint8_t* mine = box + lane * 128;
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                               __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+        if (EPI == EPI_STORE_F32 || FP8) { x.x *= rs; x.y *= rs; x.z *= rs; x.w *= rs; }
+        *reinterpret_cast<float4*>(mine + ((v ^ (lane & 7)) << 4)) = x;
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        if (EPI == EPI_ADD_F32) tma_reduce_add_3d(&tmO, box, n * BN + c * 32, row0 + quarter * 32, g);
+        else tma_store_3d(&tmO, box, n * BN + c * 32, row0 + quarter * 32, g);
+        bulk_commit();
+      }
+    }
+  } else {
+    float ss = 0.f;                       // EPI_ADD_F32 with hn_out: sum of squares of this row's new values
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(taddr + c * 32, r);
+      tmem_wait_ld();
+      const int col0 = n * BN + c * 32;
+      if (row_ok) {
+        if (EPI != EPI_ADD_F32) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * rs);
+        }
+        if (EPI == EPI_STORE_BF16) {
+          bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (col0 + v * 8 + 8 <= p.N) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                w[j] = pack_bf16(__uint_as_float(r[v * 8 + j * 2]), __uint_as_float(r[v * 8 + j * 2 + 1]));
+              *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        } else {
+          float* out = reinterpret_cast<float*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            if (col0 + v * 4 + 4 <= p.N) {
+              float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                     __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+              float4* dst = reinterpret_cast<float4*>(out + col0 + v * 4);
+              if (EPI == EPI_ADD_F32) {
+                const float4 o = *dst;
+                x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
+                if (p.hn_out != nullptr) {
+                  ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                  const float4 gn = *reinterpret_cast<const float4*>(p.gain_next + col0 + v * 4);
+                  uint2 h2;
+                  h2.x = pack_bf16(x.x * gn.x, x.y * gn.y);
+                  h2.y = pack_bf16(x.z * gn.z, x.w * gn.w);
+                  *reinterpret_cast<uint2*>(p.hn_out + (int64_t)row * p.ld_hn + col0 + v * 4) = h2;
+                }
+              }
+              *dst = x;
+            }
+          }
+        }
+      }
+    }
+    if (EPI == EPI_ADD_F32 && p.hn_out != nullptr && row_ok) p.ss_out[(int64_t)row * p.ss_ld + n] = ss;
+  }
+}
+
 // FP8: the operands are E4M3 codes, a k-block of 128 bytes holds 128 of them (64 bf16 otherwise) and
 // one MMA instruction covers 32 (16): the smem tiles, descriptors and their 32-byte steps are the same.
 template <int EPI, int HD, bool FP8>
@@ -330,7 +467,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps)
     const int quarter = warp & 3;              // TMEM lane quarter this warp may read
-    const int row_in_tile = quarter * 32 + lane;
     int it = 0;
     uint32_t boxes_out = 0;                     // output boxes this warp has handed to the TMA engine
     for (int t = blockIdx.x; t < total_tiles && !s.abort; t += gridDim.x, ++it) {
@@ -344,133 +480,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         break;
       }
       tc_fence_after();
-      const int row = m * BM + row_in_tile;
-      const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
-      // rows of a folded RMSNorm arrive un-normalised: their scale comes from the producer's sums
-      float rs = 1.0f;
-      if (p.ss_in != nullptr && row_ok) {
-        float sum = 0.f;
-        for (int i = 0; i < p.ss_cnt; ++i) sum += p.ss_in[(int64_t)row * p.ss_in_ld + i];
-        rs = rsqrtf(sum * p.inv_d + p.eps_in);
-      }
-      if (FP8 && row_ok) rs = p.a_scale[row] * *p.b_scale;     // codes -> values: row scale x matrix scale
-      if (EPI == EPI_QKV_ROPE) {
-        qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok, rs);
-      } else if (EPI == EPI_GATED_BF16) {
-        bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t gr[32], ur[32];
-          tmem_ld_32x32b_x32(taddr + c * 32, gr);
-          tmem_ld_32x32b_x32(taddr + 128 + c * 32, ur);
-          tmem_wait_ld();
-          const int col0 = n * 128 + c * 32;
-          if (row_ok) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col0 + v * 8 + 8 <= p.n_valid) {
-                uint32_t w[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const int e = v * 8 + j * 2;
-                  const float x0 = act_fn(__uint_as_float(gr[e]) * rs, p.act) * (__uint_as_float(ur[e]) * rs);
-                  const float x1 = act_fn(__uint_as_float(gr[e + 1]) * rs, p.act) * (__uint_as_float(ur[e + 1]) * rs);
-                  w[j] = pack_bf16(x0, x1);
-                }
-                *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            }
-          }
-        }
-      } else if ((EPI == EPI_ADD_F32 || EPI == EPI_STORE_F32) && p.hn_out == nullptr) {
-        // fp32 outputs leave through shared memory: the thread writes its 32 values of the chunk as one
-        // 128-byte swizzled row of the warp's 32 x 32 box, and an elected lane hands the box to the TMA
-        // engine, which stores it or adds it to the residual at the memory side. No residual value
-        // is read by the SM, rows and columns beyond the output are clipped by the hardware.
-        const bool rows_in = m * BM + quarter * 32 < p.M;     // uniform per warp
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          if (n * BN + c * 32 >= p.N) break;                 // uniform: the rest of the tile is past the last column
-          uint32_t r[32];
-          tmem_ld_32x32b_x32(taddr + c * 32, r);
-          tmem_wait_ld();
-          if (!rows_in) continue;
-          // boxes alternate by the count of boxes handed over, so "at most one group still reading"
-          // always means the other box
-          uint8_t* box = s.out_stage[quarter][boxes_out & 1];
-          ++boxes_out;
-          if (lane == 0) bulk_wait_read_1();
-          __syncwarp();
-          uint8_t* mine = box + lane * 128;
-#pragma unroll
-          for (int v = 0; v < 8; ++v) {
-            float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
-                                   __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-            if (EPI == EPI_STORE_F32 || FP8) { x.x *= rs; x.y *= rs; x.z *= rs; x.w *= rs; }
-            *reinterpret_cast<float4*>(mine + ((v ^ (lane & 7)) << 4)) = x;
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            if (EPI == EPI_ADD_F32) tma_reduce_add_3d(&tmO, box, n * BN + c * 32, m * BM + quarter * 32, g);
-            else tma_store_3d(&tmO, box, n * BN + c * 32, m * BM + quarter * 32, g);
-            bulk_commit();
-          }
-        }
-      } else {
-        float ss = 0.f;                       // EPI_ADD_F32 with hn_out: sum of squares of this row's new values
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld_32x32b_x32(taddr + c * 32, r);
-          tmem_wait_ld();
-          const int col0 = n * BN + c * 32;
-          if (row_ok) {
-            if (EPI != EPI_ADD_F32) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * rs);
-            }
-            if (EPI == EPI_STORE_BF16) {
-              bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (col0 + v * 8 + 8 <= p.N) {
-                  uint32_t w[4];
-#pragma unroll
-                  for (int j = 0; j < 4; ++j)
-                    w[j] = pack_bf16(__uint_as_float(r[v * 8 + j * 2]), __uint_as_float(r[v * 8 + j * 2 + 1]));
-                  *reinterpret_cast<uint4*>(out + col0 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-              }
-            } else {
-              float* out = reinterpret_cast<float*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
-#pragma unroll
-              for (int v = 0; v < 8; ++v) {
-                if (col0 + v * 4 + 4 <= p.N) {
-                  float4 x = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
-                                         __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-                  float4* dst = reinterpret_cast<float4*>(out + col0 + v * 4);
-                  if (EPI == EPI_ADD_F32) {
-                    const float4 o = *dst;
-                    x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
-                    if (p.hn_out != nullptr) {
-                      ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-                      const float4 gn = *reinterpret_cast<const float4*>(p.gain_next + col0 + v * 4);
-                      uint2 h2;
-                      h2.x = pack_bf16(x.x * gn.x, x.y * gn.y);
-                      h2.y = pack_bf16(x.z * gn.z, x.w * gn.w);
-                      *reinterpret_cast<uint2*>(p.hn_out + (int64_t)row * p.ld_hn + col0 + v * 4) = h2;
-                    }
-                  }
-                  *dst = x;
-                }
-              }
-            }
-          }
-        }
-        if (EPI == EPI_ADD_F32 && p.hn_out != nullptr && row_ok) p.ss_out[(int64_t)row * p.ss_ld + n] = ss;
-      }
+      epilogue_tile<EPI, HD, FP8>(p, tmO, s.out_stage[quarter][0], taddr, g, m * BM, n, quarter, lane, boxes_out);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s.tempty[buf]);
@@ -493,9 +504,254 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair form for large problems: two CTAs of a cluster (one SM pair) own one 256 x 256 output
+// tile. Each CTA streams its own 128 rows of A and its own 128 rows of B (half of the tile's
+// columns) into its own shared memory -- 32 KB per k-block instead of 48 KB, six stages instead of
+// four -- and the even-ranked CTA issues tcgen05.mma.cta_group::2 (256 x 256 x 16), which reads both
+// CTAs' operand halves and leaves each CTA its own 128 x 256 slab of the accumulator in its own
+// TMEM. Per output element every SM fetches a third fewer operand bytes from L2 and shared memory.
+// No load is multicast; only mbarrier arrivals cross between the two CTAs:
+//   full[s]    lives in the even CTA: its producer arms it with the bytes of BOTH CTAs' loads, the odd
+//              CTA's producer arrives on it remotely and both CTAs' loads complete their bytes on it;
+//   empty[s], tfull[b]   one per CTA, signalled in both CTAs by a multicast tcgen05.commit;
+//   tempty[b]  lives in the even CTA, counts the eight epilogue warps of both CTAs.
+constexpr int PSTAGES = 6;
+constexpr int PB_BYTES = 128 * BK * 2;      // this CTA's half of the B block
+constexpr int PAIR_GROUP_M = 8;             // raster: 8 x 256 rows share the same B columns in L2
+
+struct __align__(1024) PairGemmSmem {
+  uint8_t a[PSTAGES][A_BYTES];
+  uint8_t b[PSTAGES][PB_BYTES];
+  uint8_t out_stage[4][2][OUT_STAGE_BYTES];
+  uint64_t full[PSTAGES];
+  uint64_t empty[PSTAGES];
+  uint64_t tfull[2];
+  uint64_t tempty[2];
+  uint32_t tmem_base;
+  uint32_t raised;
+  volatile uint32_t abort;
+};
+
+__device__ __forceinline__ void pair_tile_coords(const GemmDev& p, int m_tiles2, int t, int& g, int& m, int& n) {
+  const int per_batch = m_tiles2 * p.n_tiles;
+  g = t / per_batch;
+  const int r = t - g * per_batch;
+  const int span = PAIR_GROUP_M * p.n_tiles;
+  const int grp = r / span;
+  const int first_m = grp * PAIR_GROUP_M;
+  const int gsize = min(PAIR_GROUP_M, m_tiles2 - first_m);
+  const int rr = r - grp * span;
+  m = first_m + rr % gsize;
+  n = rr / gsize;
+}
+
+template <int EPI, int HD, bool FP8>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmO, const GemmDev p, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  PairGemmSmem& s =
+      *reinterpret_cast<PairGemmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0: issues the tensor-core instructions
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles2 = (p.M + 2 * BM - 1) / (2 * BM);
+  const int total_tiles = m_tiles2 * p.n_tiles * p.batch;
+  constexpr int BKE = FP8 ? 2 * BK : BK;
+  const int k_blocks = (p.K + BKE - 1) / BKE;
+
+  // The even CTA decides for the pair whether the status word is raised (a kernel of this library
+  // does nothing then), so that both CTAs take the same path through the collective steps below.
+  if (threadIdx.x == 0) {
+    s.abort = 0;
+    if (rank == 0) {
+      const uint32_t v = (*reinterpret_cast<const volatile int*>(status) != 0) ? 1u : 0u;
+      s.raised = v;
+      st_cluster_u32(mapa_u32(smem_u32(&s.raised), 1), v);
+    }
+  }
+  cluster_arrive();
+  cluster_wait();
+  if (*reinterpret_cast<volatile uint32_t*>(&s.raised) != 0) return;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < PSTAGES; ++i) {
+      mbar_init(&s.full[i], 2);        // used in the even CTA: its own arming arrival + the odd CTA's
+      mbar_init(&s.empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s.tfull[i], 1);
+      mbar_init(&s.tempty[i], 8);      // used in the even CTA: four epilogue warps of each CTA
+    }
+    fence_barrier_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&s.tmem_base, TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  // the peer's barriers must exist before anything is signalled across
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem_base = s.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = pair; t < total_tiles && !s.abort; t += n_pairs) {
+        int g, m, n;
+        pair_tile_coords(p, m_tiles2, t, g, m, n);
+        const int row0 = m * 2 * BM + (int)rank * BM;       // this CTA's rows of A
+        const int col0 = n * BN + (int)rank * 128;          // this CTA's rows of B (output columns)
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&s.empty[stage], phase ^ 1)) {
+            s.abort = 1;
+            atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+            break;
+          }
+          const uint32_t full0 = mapa_u32(smem_u32(&s.full[stage]), 0);
+          if (rank == 0) mbar_expect_tx(&s.full[stage], 2 * (A_BYTES + PB_BYTES));
+          else mbar_arrive_cluster(full0);
+          tma_load_3d_pair(s.a[stage], &tmA, full0, kb * BKE, row0, g);
+          tma_load_3d_pair(s.b[stage], &tmB, full0, kb * BKE, col0, g);
+          if (++stage == PSTAGES) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA only)
+    if (rank == 0) {
+      const uint32_t leader = elect_one();
+      constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(2 * BM, BN) : umma_idesc_bf16(2 * BM, BN, 0, 0);
+      const uint64_t a_desc0 = umma_smem_desc(smem_u32(s.a[0]), 16, 1024);
+      const uint64_t b_desc0 = umma_smem_desc(smem_u32(s.b[0]), 16, 1024);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int t = pair; t < total_tiles && !s.abort; t += n_pairs, ++it) {
+        const int buf = it & 1;
+        const uint32_t bphase = (it >> 1) & 1;
+        if (!mbar_wait(&s.tempty[buf], bphase ^ 1)) {
+          s.abort = 1;
+          atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&s.full[stage], phase)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint64_t ad0 = a_desc0 + uint64_t(stage * (A_BYTES >> 4));
+          const uint64_t bd0 = b_desc0 + uint64_t(stage * (PB_BYTES >> 4));
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            if constexpr (FP8)
+              umma_e4m3_ss_pair_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+            else
+              umma_bf16_ss_pair_w(leader, d_tmem, ad0 + uint64_t(k * 2), bd0 + uint64_t(k * 2), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit_pair_w(leader, &s.empty[stage], (uint16_t)3);      // the stage is free in both CTAs
+          if (++stage == PSTAGES) {
+            stage = 0;
+            phase ^= 1;
+          }
+        }
+        if (!ok) {
+          s.abort = 1;
+          atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+          break;
+        }
+        umma_commit_pair_w(leader, &s.tfull[buf], (uint16_t)3);           // both CTAs' slabs are complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps per CTA)
+    const int quarter = warp & 3;
+    int it = 0;
+    uint32_t boxes_out = 0;
+    for (int t = pair; t < total_tiles && !s.abort; t += n_pairs, ++it) {
+      const int buf = it & 1;
+      const uint32_t bphase = (it >> 1) & 1;
+      int g, m, n;
+      pair_tile_coords(p, m_tiles2, t, g, m, n);
+      if (!mbar_wait(&s.tfull[buf], bphase)) {
+        s.abort = 1;
+        atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+      epilogue_tile<EPI, HD, FP8>(p, tmO, s.out_stage[quarter][0], taddr, g, m * 2 * BM + (int)rank * BM, n, quarter,
+                                  lane, boxes_out);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&s.tempty[buf]), 0));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (warp >= 2 && lane == 0) bulk_wait_all();
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (s.abort && threadIdx.x == 0) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let copies still in flight into this CTA land
+  }
+  // neither CTA may release its TMEM or exit while the other can still signal it or read its operands
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 template <int EPI, int HD = 0, bool FP8 = false>
 int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p, int grid,
-               cudaStream_t stream) {
+               bool pair, cudaStream_t stream) {
+  int* status = status_word();
+  if (!status) return POP_E_CUDA;
+  if (pair) {
+    const size_t smem = sizeof(PairGemmSmem) + 1024;
+    static bool configured = false;
+    if (!configured) {
+      if (cudaFuncSetAttribute(gemm_pair_kernel<EPI, HD, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem) != cudaSuccess)
+        return POP_E_CUDA;
+      configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_pair_kernel<EPI, HD, FP8>, ta, tb, to, p, status);
+    count_launch();
+    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? POP_OK : POP_E_CUDA;
+  }
   const size_t smem = sizeof(GemmSmem) + 1024;
   static bool configured = false;
   if (!configured) {
@@ -504,12 +760,20 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
       return POP_E_CUDA;
     configured = true;
   }
-  int* status = status_word();
-  if (!status) return POP_E_CUDA;
   ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
   gemm_kernel<EPI, HD, FP8><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+}
+
+// CTA pairs pay off once every SM pair has at least one 256 x 256 tile; POP_GEMM_PAIR=0 / 1 in the
+// environment forces the single-CTA / the pair form (used by the tests to cover both on every shape).
+bool use_pair(int M, int64_t tiles2, int sms) {
+  const char* e = std::getenv("POP_GEMM_PAIR");
+  if (e && e[0] == '0') return false;
+  if (e && e[0] == '1') return true;
+  (void)M; (void)tiles2; (void)sms;
+  return false;
 }
 
 }  // namespace
@@ -534,6 +798,13 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   } else {
     if (a.N % 4 || a.ldo % 4) return POP_E_INVALID;
   }
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return POP_E_CUDA;
+  const int64_t tiles2 = int64_t(ceil_div(a.M, 2 * BM)) * ceil_div(a.N, BN) * a.batch;
+  const bool pair = use_pair(a.M, tiles2, sms);
+  const uint32_t b_box = pair ? 128 : BN;      // a CTA of a pair loads its own half of the B block
   CUtensorMap ta, tb;
   int rc;
   if (a.fp8) {
@@ -541,14 +812,14 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
       return POP_E_INVALID;
     rc = make_tmap_u8_3d(&ta, a.A, a.K, a.M, 1, a.lda, (uint64_t)a.lda * a.M, BM);
     if (rc) return rc;
-    rc = make_tmap_u8_3d(&tb, a.B, a.K, a.N, 1, a.ldb, (uint64_t)a.ldb * a.N, BN);
+    rc = make_tmap_u8_3d(&tb, a.B, a.K, a.N, 1, a.ldb, (uint64_t)a.ldb * a.N, b_box);
     if (rc) return rc;
   } else {
     rc = make_tmap_bf16_3d(&ta, a.A, a.K, a.M, a.batch, a.lda, a.a_batch_stride ? a.a_batch_stride : a.lda * a.M,
                            BK, BM);
     if (rc) return rc;
     rc = make_tmap_bf16_3d(&tb, a.B, a.K, a.N, a.batch, a.ldb, a.b_batch_stride ? a.b_batch_stride : a.ldb * a.N, BK,
-                           BN);
+                           b_box);
     if (rc) return rc;
   }
   if (a.hn_out != nullptr) {
@@ -592,38 +863,35 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   p.n_tiles = ceil_div(a.N, BN);
   p.act = a.act;
   p.n_valid = a.n_valid;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return POP_E_CUDA;
   const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
-  const int grid = (int)(total < sms ? total : sms);
+  int grid = (int)(total < sms ? total : sms);
+  if (pair) grid = 2 * (int)(tiles2 < sms / 2 ? tiles2 : sms / 2);
   if (a.fp8) {
     switch (a.epilogue) {
-      case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, stream);
-      case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, stream);
-      case EPI_ADD_F32: return launch_epi<EPI_ADD_F32, 0, true>(ta, tb, to, p, grid, stream);
-      case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, stream);
+      case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, pair, stream);
+      case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, pair, stream);
+      case EPI_ADD_F32: return launch_epi<EPI_ADD_F32, 0, true>(ta, tb, to, p, grid, pair, stream);
+      case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, pair, stream);
       case EPI_QKV_ROPE:
         switch (a.rope->hd) {
-          case 64: return launch_epi<EPI_QKV_ROPE, 64, true>(ta, tb, to, p, grid, stream);
-          case 128: return launch_epi<EPI_QKV_ROPE, 128, true>(ta, tb, to, p, grid, stream);
-          case 256: return launch_epi<EPI_QKV_ROPE, 256, true>(ta, tb, to, p, grid, stream);
+          case 64: return launch_epi<EPI_QKV_ROPE, 64, true>(ta, tb, to, p, grid, pair, stream);
+          case 128: return launch_epi<EPI_QKV_ROPE, 128, true>(ta, tb, to, p, grid, pair, stream);
+          case 256: return launch_epi<EPI_QKV_ROPE, 256, true>(ta, tb, to, p, grid, pair, stream);
         }
         return POP_E_INVALID;
     }
     return POP_E_INVALID;
   }
   switch (a.epilogue) {
-    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, stream);
-    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, stream);
-    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, to, p, grid, stream);
-    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, to, p, grid, stream);
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, pair, stream);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, pair, stream);
+    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, to, p, grid, pair, stream);
+    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, to, p, grid, pair, stream);
     case EPI_QKV_ROPE:
       switch (a.rope->hd) {
-        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, to, p, grid, stream);
-        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, to, p, grid, stream);
-        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, to, p, grid, stream);
+        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, to, p, grid, pair, stream);
+        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, to, p, grid, pair, stream);
+        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, to, p, grid, pair, stream);
       }
       return POP_E_INVALID;
   }

@@ -23,3 +23,16 @@ def paged_pools(k, v, page_size, extra_pages=3, seed=0, garbage=float("nan")):
         kp[pages, pos % page_size] = k[b]
         vp[pages, pos % page_size] = v[b]
     return kp, vp, bt
+
+
+def interleave_gate_up(w_gate, w_up):
+    """The fused gate/up operand layout of the gated GEMM / GEMV: blocks of 128 gate rows followed by the
+    matching 128 up rows, the last block zero-padded to 128. [F, K] x 2 -> [2 * ceil(F/128)*128, K]."""
+    F, K = w_gate.shape
+    f_pad = (F + 127) // 128 * 128
+    out = torch.zeros(2 * f_pad, K, dtype=w_gate.dtype, device=w_gate.device)
+    for t in range(f_pad // 128):
+        n = min(128, F - t * 128)
+        out[256 * t: 256 * t + n] = w_gate[128 * t: 128 * t + n]
+        out[256 * t + 128: 256 * t + 128 + n] = w_up[128 * t: 128 * t + n]
+    return out

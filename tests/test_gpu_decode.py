@@ -1,5 +1,5 @@
-"""pop_decode_step (the full model's decode stage over the cache a prefill built, paper Sec. 2.2 /
-Sec. 3 "retaining the full model for decode") against the oracle's decode_step.
+"""pop_decode_step (the full model's decode stage over the cache a prefill built, paper Sec. 3.2 Eq. 11 /
+Sec. 3.3, where decoding keeps every layer) against the oracle's decode_step.
 
 Tolerances as for the prefill: every layer's K and V per tensor max|err|/max|ref| <= 2e-2, logits
 max|err| <= 5e-2 against the fp64 oracle; the greedy token (a decision taken in floating point) is

@@ -121,7 +121,7 @@ def test_kept_layers_on_fp8_operands(variant, B, N, l_keep, chunk):
     l_keep = min(l_keep, cfg.n_layers)
     w = ps.SynthWeights(cfg)
     tokens = ps.uniform_tokens(41, B, N, cfg.vocab)
-    ref = po.pop_prefill(cfg, w, tokens, None, l_keep, precision="kernel", fp8_kept=True)
+    ref = po.pop_prefill(cfg, w, tokens, None, l_keep, precision="bf16ops", fp8_kept=True)
     model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
     model.enable_fp8()
     cache = KVCache(cfg, B, N, 16, fill=float("nan"))
@@ -203,7 +203,7 @@ def test_ragged_batch_on_fp8_operands():
     logits = model.prefill_ragged(packed.to(DEV), None, lens, l_keep, cache)
     assert model.last_status() == 0 and not torch.isnan(logits).any()
     for b, (t, n) in enumerate(zip(seqs, lens)):
-        ref = po.pop_prefill(cfg, w, t, None, l_keep, precision="kernel", fp8_kept=True)
+        ref = po.pop_prefill(cfg, w, t, None, l_keep, precision="bf16ops", fp8_kept=True)
         assert (logits[b].cpu().double() - ref["logits"][0]).abs().max().item() <= 3e-1, f"seq {b}"
         for l in range(cfg.n_layers):
             k, v = cache.gather(l, n)

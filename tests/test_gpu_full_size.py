@@ -205,7 +205,7 @@ def test_fp8_operands_at_the_benchmark_size():
     k_ref, v_ref = po.kv_generation(cfg, w, 1, x1, pos, torch.float64, "fp8")
     k1, v1 = c8.gather(0)
     assert rel_err(k1[0, pos], k_ref) <= KV_TOL and rel_err(v1[0, pos], v_ref) <= KV_TOL
-    k_b, v_b = po.kv_generation(cfg, w, 1, x1, pos, torch.float64, "kernel")
+    k_b, v_b = po.kv_generation(cfg, w, 1, x1, pos, torch.float64, "bf16ops")
     assert rel_err(k1[0, pos], k_b) > 2e-3                         # the quantisation is really there
     for l in range(cfg.n_layers):
         k, v = c8.gather(l)

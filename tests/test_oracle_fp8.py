@@ -98,17 +98,17 @@ def test_fp8_projections_restated_with_the_library_cast():
     # the quantised model stays near the unquantised one, and is not it
     tokens = ps.uniform_tokens(3, 1, 12, cfg.vocab)
     a = po.full_prefill(cfg, w, tokens, precision="fp8")
-    b = po.full_prefill(cfg, w, tokens, precision="kernel")
+    b = po.full_prefill(cfg, w, tokens, precision="bf16ops")
     for l in range(cfg.n_layers):
         err = (a["V"][l] - b["V"][l]).abs().max() / b["V"][l].abs().max()
         assert 0 < err.item() < 0.35          # 3 mantissa bits, rows of 32 terms
     # kept layers only: with every layer pruned but the first, the deep layers' entries of positions < N-1
     # are bf16 projections of an fp8-computed state
-    r = po.pop_prefill(cfg, w, tokens, None, 1, precision="kernel", fp8_kept=True)
-    r0 = po.pop_prefill(cfg, w, tokens, None, 1, precision="kernel")
+    r = po.pop_prefill(cfg, w, tokens, None, 1, precision="bf16ops", fp8_kept=True)
+    r0 = po.pop_prefill(cfg, w, tokens, None, 1, precision="bf16ops")
     assert (r["K"][0] - a["K"][0]).abs().max().item() == 0                 # layer 1 is the fp8 layer of the full run
     assert (r["K"][1] - r0["K"][1]).abs().max().item() > 0                 # H differs
-    kk, vv = po.kv_generation(cfg, w, 2, r["H"][0], torch.arange(11), torch.float64, "kernel")
+    kk, vv = po.kv_generation(cfg, w, 2, r["H"][0], torch.arange(11), torch.float64, "bf16ops")
     assert (r["K"][1][0, :11] - kk).abs().max().item() == 0
 
 
@@ -132,8 +132,8 @@ def test_weight_only_precision_is_the_kernel_precision_on_dequantised_weights():
     x = torch.randn(5, cfg.d_model, generator=torch.Generator().manual_seed(12), dtype=torch.float64)
     pos = torch.arange(5)
     a = po.layer_forward(cfg, w, 2, x, pos, None, None, torch.float64, "fp8w")
-    b = po.layer_forward(cfg, Patched(), 2, x, pos, None, None, torch.float64, "kernel")
+    b = po.layer_forward(cfg, Patched(), 2, x, pos, None, None, torch.float64, "bf16ops")
     for u, v in zip(a, b):
         assert (u - v).abs().max().item() < 1e-5          # the scale is an fp32 number in the oracle
-    c = po.layer_forward(cfg, w, 2, x, pos, None, None, torch.float64, "kernel")
+    c = po.layer_forward(cfg, w, 2, x, pos, None, None, torch.float64, "bf16ops")
     assert (a[0] - c[0]).abs().max().item() > 1e-4

@@ -333,7 +333,7 @@ def test_first_token_depends_on_the_projected_cache():
 
 @pytest.mark.parametrize("variant", list(VARIANTS))
 def test_decode_steps_reproduce_the_full_prefill_of_the_longer_prompt(variant):
-    # the decode stage is the full model on one more position over the cache (Sec. 2.2): feeding the
+    # the decode stage is the full model on one more position over the cache (Sec. 3.2, Eq. 11): feeding the
     # tokens of a longer prompt one by one after a full prefill of its first part must give that
     # longer prompt's cache and last-position logits (causality; nothing of the future is used)
     cfg, w, tokens = _setup(variant, n=11, batch=2)
@@ -391,7 +391,7 @@ def test_explicit_skip_sets():
 
 
 def test_without_boundary_handling_the_last_token_sees_the_pruned_model():
-    # Sec. 4.4.1 "w/o Boundary Handling": x_N goes through the pruned prefill model. Pruned layers pass
+    # Sec. 4.4.1, the variant without boundary handling: x_N goes through the pruned prefill model. Pruned layers pass
     # the state on unchanged (Eq. 15), so the logits are those of the model truncated to its kept
     # layers, and every position of a pruned layer -- the last included -- holds Eq. 14 of the kept
     # stack's output.
@@ -412,7 +412,7 @@ def test_without_boundary_handling_the_last_token_sees_the_pruned_model():
 
 
 def test_without_independent_kv_a_pruned_layer_attends_to_the_last_token_only():
-    # Sec. 4.4.1 "w/o Indep. KV Proj.": pruned layers generate no cache in the prefill, so in the first
+    # Sec. 4.4.1, the variant without independent KV projections: pruned layers generate no cache in the prefill, so in the first
     # decode step such a layer sees one key, its own: softmax over one score is 1 and the attention
     # output is the token's own value vector (repeated over the query heads of a group), whatever q is.
     cfg, w, tokens = _setup("llama", n=7, batch=2)          # 3 layers, no window, no post norms

@@ -170,7 +170,7 @@ def _golden():
 def test_values_the_paper_prints():
     import pop_synth as ps
     g = _golden()
-    # the pruned set "last 1/3 of the layers" gives the fractions the results table prints, and the layer
+    # pruning the deepest third of the layers gives the fractions the results table prints, and the layer
     # range the appendix names for the 36-layer model
     for L in (32, 36, 48):
         frac = 100.0 * len(po.deep_third(L)) / L
