@@ -180,7 +180,7 @@ int full_layer(pop_model* m, const Workspace& w, int l, int N, int B, const pop_
   r.q_out = w.q; r.ldq = m->q_dim;
   r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
   r.layer0 = l - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
-  r.page_size = kc->page_size;
+  r.page_size = kc->page_size; r.num_pages = kc->num_pages;
   r.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   // the epilogue indexes the table by absolute position: hand it the address row 0 would have
@@ -270,7 +270,7 @@ int pruned_kv(pop_model* m, const Workspace& w, int l0, int n, int N, int B, con
   r.q_out = nullptr; r.ldq = 0;
   r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
   r.layer0 = l0 - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
-  r.page_size = kc->page_size;
+  r.page_size = kc->page_size; r.num_pages = kc->num_pages;
   r.q_gain = nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l0, m->lo.k_norm) : nullptr;
   r.gain_group_stride = (int64_t)(m->layer_stride / 4);
@@ -310,7 +310,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   r.in = w.qkvb; r.ld_in = m->qkv_dim; r.q_out = w.qb; r.ldq = m->q_dim;
   r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
   r.layer0 = l - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
-  r.page_size = kc->page_size;
+  r.page_size = kc->page_size; r.num_pages = kc->num_pages;
   r.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
   r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   r.table = table; r.table_pos0 = table_pos0; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
@@ -325,7 +325,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.partial = w.partial; a.out = w.ob; a.ldo = m->q_dim;
   a.batch = B; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads; a.head_dim = c.head_dim; a.kv_len = N;
   a.cu_seqlens = cu; a.pos_dev = pos_dev; a.counters = w.dec_ctr;
-  a.kv_first = kv_first;
+  a.kv_first = kv_first; a.num_pages = kc->num_pages;
   a.window = layer_window(c, l);
   POP_TRY(launch_decode_attention(a, s));
   v = GemvArgs{};

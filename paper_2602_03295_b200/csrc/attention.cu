@@ -76,6 +76,7 @@ struct AttnDev {
   int kv_len;           // valid cache positions per sequence
   int n_q_heads, n_kv_heads;
   int window;
+  int num_pages;        // block-table entries are checked against it
   int q_tiles;
   float scale_log2;     // log2(e) / sqrt(hd)
   const int32_t* cu;    // ragged batches: packed-row prefix sums [batch + 1], or null
@@ -191,6 +192,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         for (int r = 0; r < n_loads; ++r) {
           const int pos = kv0 + r * p.rows_per_load;
           const int page = bt[pos / p.page_size];
+          // an entry outside the pool cannot fault here (the tensor map clips), but it is an error
+          if ((unsigned)page >= (unsigned)p.num_pages) atomicMin(status, (int)POP_E_INVALID);
           const int slot = pos % p.page_size;
           for (int c = 0; c < HD / 64; ++c)
             tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
@@ -571,6 +574,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int r = 0; r < n_loads; ++r) {
           const int pos = kv0 + r * p.rows_per_load;
           const int page = bt[pos / p.page_size];
+          // an entry outside the pool cannot fault here (the tensor map clips), but it is an error
+          if ((unsigned)page >= (unsigned)p.num_pages) atomicMin(status, (int)POP_E_INVALID);
           const int slot = pos % p.page_size;
           for (int c = 0; c < HD / 64; ++c)
             tma_load_4d(s.kv[stage] + c * C::KV_SUB_BYTES + r * p.rows_per_load * 128, tm, &s.kv_full[stage],
@@ -826,6 +831,7 @@ int launch_t(const AttnArgs& a, cudaStream_t stream) {
   p.n_q_heads = a.n_q_heads;
   p.n_kv_heads = a.n_kv_heads;
   p.window = a.window;
+  p.num_pages = a.num_pages;
   p.q_tiles = ceil_div(a.seq_len, 128);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.cu = a.cu_seqlens;

@@ -174,6 +174,10 @@ struct RopeArgs {
   // boundary / decode rows only: the position is read from device memory at run time (a step that is
   // replayed from a captured graph with an advancing position); the table then holds that one row
   const int32_t* pos_dev;
+  // pages per layer of the pools. Block-table entries live on the device, so only the kernel can
+  // check them: with num_pages > 0 an entry outside [0, num_pages) is never turned into an address;
+  // the row is skipped and the status word raised to POP_E_INVALID. 0 = unknown (no check).
+  int num_pages;
 };
 int launch_rope_cache(const RopeArgs& a, cudaStream_t s);
 int launch_gather_rows(const float* src, float* dst, int batch, int d, int rows_per_seq, int row, cudaStream_t s);
@@ -221,6 +225,7 @@ struct DecAttnArgs {
   // optional [batch][n_kv] int32, all zero before the call and all zero again after it: with it the
   // attention kernel merges its own splits (one launch); without, a second kernel does
   int32_t* counters;
+  int num_pages;               // pages in the pool, for the device-side block-table check (0 = no check)
 };
 int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

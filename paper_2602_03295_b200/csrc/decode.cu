@@ -259,6 +259,8 @@ struct DecAttnDev {
   // [B][n_kv] arrival counters, zero before the launch and zero again after it: the last CTA of a
   // (sequence, kv head) to finish merges the splits itself. Null: the combine kernel does it.
   unsigned int* counters;
+  int num_pages;                           // block-table entries are checked against it when > 0
+  int* status;                             // device status word
 };
 
 constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of one MMA
@@ -394,7 +396,13 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
     // lanes 0..15 (and again 16..31) each find the pool row of one key of the group; -1 past the chunk
     const int jk = jg + (lane & 15);
     int row = -1;
-    if (jk < j1) row = bt[jk / p.page_size] * p.page_size + jk % p.page_size;
+    if (jk < j1) {
+      const int page = bt[jk / p.page_size];
+      if (p.num_pages > 0 && (unsigned)page >= (unsigned)p.num_pages)
+        atomicMin(p.status, (int)POP_E_INVALID);     // never turned into an address: the key reads as zeros
+      else
+        row = page * p.page_size + jk % p.page_size;
+    }
 #pragma unroll
     for (int i = 0; i < KT * CH / 32; ++i) {
       const int idx = i * 32 + lane;
@@ -658,6 +666,9 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   p.cu = a.cu_seqlens;
   p.pos_dev = a.pos_dev;
   p.counters = reinterpret_cast<unsigned int*>(a.counters);
+  p.num_pages = a.num_pages;
+  p.status = status_word();
+  if (!p.status) return POP_E_CUDA;
   p.splits = decode_attn_splits(a.pos_dev ? 0 : a.kv_len, a.window, a.n_kv, a.batch);
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)a.head_dim);
   const int span = (a.window > 0 && a.window < a.kv_len) ? a.window : a.kv_len;
@@ -734,6 +745,8 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.q = static_cast<const bf16*>(q); p.ldq = ldq;
   p.k_pool = static_cast<const bf16*>(k_pool); p.v_pool = static_cast<const bf16*>(v_pool);
   p.block_table = block_table; p.max_pages_per_seq = max_pages_per_seq; p.page_size = page_size;
+  p.num_pages = 0;
+  p.status = nullptr;
   p.partial = scratch;
   p.out = static_cast<bf16*>(out); p.ldo = ldo;
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;

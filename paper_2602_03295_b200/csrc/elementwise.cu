@@ -213,6 +213,8 @@ struct RopeDev {
   float eps;
   const int32_t* cu;      // boundary rows of a ragged batch: row b sits at position cu[b+1] - cu[b] - 1
   const int32_t* pos_dev; // run-time position of all rows; table row 0 is that position
+  int num_pages;          // block-table entries are checked against it when > 0
+  int* status;            // device status word
 };
 
 template <int HD>
@@ -272,6 +274,10 @@ __global__ void rope_cache_kernel(const RopeDev p) {
   } else {
     const int kvh = is_v ? h - p.n_q - p.n_kv : h - p.n_q;
     const int page = p.block_table[(int64_t)b * p.max_pages_per_seq + pos / p.page_size];
+    if (p.num_pages > 0 && (unsigned)page >= (unsigned)p.num_pages) {
+      if (lane == 0) atomicMin(p.status, (int)POP_E_INVALID);     // never turned into an address
+      return;
+    }
     const int slot = pos % p.page_size;
     bf16* pool = (is_v ? p.v_pool : p.k_pool) + (int64_t)(p.layer0 + g) * p.pool_layer_stride;
     dst = pool + (((int64_t)page * p.page_size + slot) * p.n_kv + kvh) * HD;
@@ -399,6 +405,9 @@ int launch_rope_cache(const RopeArgs& a, cudaStream_t s) {
   p.eps = a.eps;
   p.cu = a.cu_seqlens;
   p.pos_dev = a.pos_dev;
+  p.num_pages = a.num_pages;
+  p.status = status_word();
+  if (!p.status) return POP_E_CUDA;
   if ((a.cu_seqlens != nullptr || a.pos_dev != nullptr) && a.rows_per_seq != 1) return POP_E_INVALID;
   const int heads = a.n_q + 2 * a.n_kv;
   const int64_t items = (int64_t)a.rows * heads;

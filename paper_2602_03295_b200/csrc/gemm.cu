@@ -51,6 +51,7 @@ struct RopeEpi {
   int rows_per_seq, rows_written, pos0;
   float eps;
   const int32_t* cu; int batch; int skip_last;    // ragged batches (see RopeArgs)
+  int num_pages;                                  // block-table entries are checked against it when > 0
 };
 
 struct GemmDev {
@@ -63,6 +64,7 @@ struct GemmDev {
   bf16* hn_out; int64_t ld_hn; const float* gain_next; float* ss_out; int ss_ld;
   const float* ss_in; int ss_cnt; int ss_in_ld; float inv_d; float eps_in;
   const float* a_scale; const float* b_scale;      // FP8 operands: accumulator scale a_scale[row] * *b_scale
+  int* status;                                     // device status word
 };
 
 __device__ __forceinline__ void tile_coords(const GemmDev& p, int t, int& g, int& m, int& n) {
@@ -121,7 +123,12 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
   int64_t cache_row = 0;
   if (active) {
     const int page = r.block_table[(int64_t)b * r.max_pages_per_seq + pos / r.page_size];
-    cache_row = (int64_t)page * r.page_size + pos % r.page_size;
+    if (r.num_pages > 0 && (unsigned)page >= (unsigned)r.num_pages) {
+      atomicMin(p.status, (int)POP_E_INVALID);       // never turned into an address
+      active = false;
+    } else {
+      cache_row = (int64_t)page * r.page_size + pos % r.page_size;
+    }
   }
   const float2* tab = r.table + (int64_t)pos * (HD / 2);
 #pragma unroll 1
@@ -512,8 +519,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // CTAs' operand halves and leaves each CTA its own 128 x 256 slab of the accumulator in its own
 // TMEM. Per output element every SM fetches a third fewer operand bytes from L2 and shared memory.
 // No load is multicast; only mbarrier arrivals cross between the two CTAs:
-//   full[s]    lives in the even CTA: its producer arms it with the bytes of BOTH CTAs' loads, the odd
-//              CTA's producer arrives on it remotely and both CTAs' loads complete their bytes on it;
+//   full[s]    lives in the even CTA: its producer arms it with the bytes of BOTH CTAs' loads and both
+//              CTAs' loads complete their bytes on it;
 //   empty[s], tfull[b]   one per CTA, signalled in both CTAs by a multicast tcgen05.commit;
 //   tempty[b]  lives in the even CTA, counts the eight epilogue warps of both CTAs.
 constexpr int PSTAGES = 6;
@@ -564,6 +571,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   // The even CTA decides for the pair whether the status word is raised (a kernel of this library
   // does nothing then), so that both CTAs take the same path through the collective steps below.
+  cluster_arrive();      // both CTAs are running: the peer's shared memory may be written from here on
+  cluster_wait();
   if (threadIdx.x == 0) {
     s.abort = 0;
     if (rank == 0) {
@@ -577,7 +586,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (*reinterpret_cast<volatile uint32_t*>(&s.raised) != 0) return;
   if (threadIdx.x == 0) {
     for (int i = 0; i < PSTAGES; ++i) {
-      mbar_init(&s.full[i], 2);        // used in the even CTA: its own arming arrival + the odd CTA's
+      mbar_init(&s.full[i], 1);        // used in the even CTA, armed by its producer for both CTAs' bytes
       mbar_init(&s.empty[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -616,8 +625,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             break;
           }
           const uint32_t full0 = mapa_u32(smem_u32(&s.full[stage]), 0);
+          // The even CTA's one arrival arms the barrier with the bytes of both CTAs' loads; the odd CTA
+          // only sends its bytes there. Its loads for this phase cannot start before the phase opens:
+          // its empty[stage] fires when the tensor core has finished reading the previous contents,
+          // which is after the previous phase completed. Bytes that land before the arming arrival
+          // are accounted for when it comes (the pending arrival keeps the phase open).
           if (rank == 0) mbar_expect_tx(&s.full[stage], 2 * (A_BYTES + PB_BYTES));
-          else mbar_arrive_cluster(full0);
           tma_load_3d_pair(s.a[stage], &tmA, full0, kb * BKE, row0, g);
           tma_load_3d_pair(s.b[stage], &tmB, full0, kb * BKE, col0, g);
           if (++stage == PSTAGES) {
@@ -722,10 +735,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 }
 
 template <int EPI, int HD = 0, bool FP8 = false>
-int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p, int grid,
+int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p_in, int grid,
                bool pair, cudaStream_t stream) {
   int* status = status_word();
   if (!status) return POP_E_CUDA;
+  GemmDev p = p_in;
+  p.status = status;
   if (pair) {
     const size_t smem = sizeof(PairGemmSmem) + 1024;
     static bool configured = false;
@@ -772,8 +787,7 @@ bool use_pair(int M, int64_t tiles2, int sms) {
   const char* e = std::getenv("POP_GEMM_PAIR");
   if (e && e[0] == '0') return false;
   if (e && e[0] == '1') return true;
-  (void)M; (void)tiles2; (void)sms;
-  return false;
+  return M > BM && tiles2 >= sms / 2;
 }
 
 }  // namespace
@@ -854,6 +868,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     p.rope.rows_per_seq = r.rows_per_seq; p.rope.rows_written = r.rows_written; p.rope.pos0 = r.pos0;
     p.rope.eps = r.eps;
     p.rope.cu = r.cu_seqlens; p.rope.batch = r.batch; p.rope.skip_last = r.skip_last;
+    p.rope.num_pages = r.num_pages;
   }
   p.out = a.out;
   p.ldo = a.ldo;

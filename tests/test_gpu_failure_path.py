@@ -71,3 +71,22 @@ def test_an_unusable_token_id_is_reported_not_dereferenced(bad):
     model.decode_step(torch.tensor([bad], dtype=torch.int32, device=DEV), 40, KVCache(cfg, 1, 41, 16))
     assert model.last_status() == POP_E_INVALID
     assert model.last_status() == 0
+
+
+def test_a_block_table_entry_outside_the_pool_is_reported_not_dereferenced():
+    # the block table lives on the device: the kernels that turn its entries into addresses check them
+    from paper_2602_03295_b200 import POP_E_INVALID
+    from paper_2602_03295_b200.binding import KVCache, PopModel
+    cfg = ps.C1_TINY
+    model = PopModel(cfg, ps.SynthWeights(cfg, device=DEV))
+    tokens = ps.uniform_tokens(6, 1, 40, cfg.vocab).to(DEV)
+    for bad in (-1, 3, 10 ** 6):
+        bt = torch.tensor([[0, bad, 2]], dtype=torch.int32)
+        cache = KVCache(cfg, 1, 40, 16, block_table=bt, num_pages=3, fill=5.0)
+        model.prefill(tokens, None, 3, cache)
+        assert model.last_status() == POP_E_INVALID, bad
+        assert model.last_status() == 0
+        assert (cache.k[:, [0, 2]] == 5.0).sum() < cache.k[:, [0, 2]].numel()     # valid pages were written
+    cache = KVCache(cfg, 1, 40, 16, fill=float("nan"))
+    logits = model.prefill(tokens, None, 3, cache)
+    assert model.last_status() == 0 and torch.isfinite(logits).all()

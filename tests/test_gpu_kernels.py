@@ -23,15 +23,24 @@ def L():
     return pk.lib()
 
 
+@pytest.fixture(params=["single", "pair"])
+def gemm_form(request, monkeypatch):
+    """Runs a GEMM test twice: with one CTA per 128 x 256 tile and with a CTA pair per 256 x 256 tile
+    (POP_GEMM_PAIR forces either form whatever the problem size)."""
+    monkeypatch.setenv("POP_GEMM_PAIR", "1" if request.param == "pair" else "0")
+    return request.param
+
+
 def _bf(shape, seed, std=0.5):
     g = torch.Generator().manual_seed(seed)
     return (torch.randn(*shape, generator=g) * std).bfloat16()
 
 
 @pytest.mark.parametrize("M,N,K,G", [(128, 256, 64, 1), (300, 264, 136, 1), (1000, 1024, 4096, 1),
-                                     (200, 512, 128, 3), (1, 8, 8, 1), (129, 2056, 72, 2)])
+                                     (200, 512, 128, 3), (1, 8, 8, 1), (129, 2056, 72, 2), (385, 520, 200, 1),
+                                     (2100, 5000, 328, 1)])
 @pytest.mark.parametrize("epi", [0, 1, 2])
-def test_gemm_plain_epilogues(L, M, N, K, G, epi):
+def test_gemm_plain_epilogues(L, gemm_form, M, N, K, G, epi):
     A, B = _bf((G, M, K), 1), _bf((G, N, K), 2)
     ref = torch.matmul(A.double(), B.double().transpose(1, 2))
     if epi == 0:
@@ -47,7 +56,7 @@ def test_gemm_plain_epilogues(L, M, N, K, G, epi):
 
 
 @pytest.mark.parametrize("M,F,K,act", [(384, 256, 320, 0), (130, 688, 256, 0), (257, 1000, 136, 1)])
-def test_gemm_gated_epilogue(L, M, F, K, act):
+def test_gemm_gated_epilogue(L, gemm_form, M, F, K, act):
     # gate/up rows interleaved in blocks of 128 with zero padding of the last block, as the
     # library's weight repacking lays them out
     Wg, Wu, A = _bf((F, K), 4), _bf((F, K), 5), _bf((M, K), 6)
@@ -164,7 +173,7 @@ def test_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm):
 
 
 @pytest.mark.parametrize("M,d,K,F", [(300, 520, 136, 688), (129, 256, 72, 264)])
-def test_rmsnorm_folded_around_the_gemms(L, M, d, K, F):
+def test_rmsnorm_folded_around_the_gemms(L, gemm_form, M, d, K, F):
     # residual GEMM that also emits the next operand and row sums of squares, then a gated and a
     # plain GEMM that consume them: together they must equal residual add -> RMSNorm -> GEMM
     eps = 1e-5
@@ -203,7 +212,7 @@ def test_rmsnorm_folded_around_the_gemms(L, M, d, K, F):
 
 @pytest.mark.parametrize("hd,n_q,n_kv,qk_norm,groups", [(64, 4, 2, 0, 1), (128, 4, 1, 1, 1), (256, 2, 2, 1, 1),
                                                         (128, 0, 2, 1, 3), (64, 3, 3, 0, 1)])
-def test_fused_qkv_projection_rope_and_cache_write(L, hd, n_q, n_kv, qk_norm, groups):
+def test_fused_qkv_projection_rope_and_cache_write(L, gemm_form, hd, n_q, n_kv, qk_norm, groups):
     # the projection GEMM with norm, RoPE and the paged-cache write in its epilogue, against the
     # oracle's statement of Eq. 2-3 (fp64); several m tiles with a ragged tail, several n tiles
     B, N, K, page, theta, eps, layers = 2, 150, 136, 16, 500000.0, 1e-6, 5

@@ -32,6 +32,12 @@ def L():
     return pk.lib()
 
 
+@pytest.fixture(params=["single", "pair"])
+def gemm_form(request, monkeypatch):
+    monkeypatch.setenv("POP_GEMM_PAIR", "1" if request.param == "pair" else "0")
+    return request.param
+
+
 def _randn_bf16(shape, seed, std=1.0):
     g = torch.Generator(device=DEV).manual_seed(seed)
     return (torch.randn(*shape, generator=g, device=DEV) * std).bfloat16()
@@ -80,7 +86,7 @@ M_FULL = 8192
 
 @pytest.mark.parametrize("name,N,K,epi", [("qkv-shape", 6144, 4096, 0), ("o-proj", 4096, 4096, 2),
                                           ("down", 4096, 14336, 2), ("store-f32", 4096, 4096, 1)])
-def test_gemm_at_the_config2_shapes(L, name, N, K, epi):
+def test_gemm_at_the_config2_shapes(L, gemm_form, name, N, K, epi):
     A = _randn_bf16((M_FULL, K), 201, 0.5)
     B = _randn_bf16((N, K), 202, 0.05)
     rows = _rows(M_FULL, 256, 11)
@@ -98,7 +104,7 @@ def test_gemm_at_the_config2_shapes(L, name, N, K, epi):
     assert rel_err(out[rows.to(DEV)], ref) < (1e-2 if epi == 0 else 1e-4)
 
 
-def test_gated_gemm_at_the_config2_shape(L):
+def test_gated_gemm_at_the_config2_shape(L, gemm_form):
     F, K = 14336, 4096
     A = _randn_bf16((M_FULL, K), 211, 0.5)
     Wg, Wu = _randn_bf16((F, K), 212, 0.03), _randn_bf16((F, K), 213, 0.03)
@@ -113,7 +119,7 @@ def test_gated_gemm_at_the_config2_shape(L):
     assert rel_err(out[rows.to(DEV)], ref) < 1e-2
 
 
-def test_batched_pruned_layer_projection_at_the_config2_shape(L):
+def test_batched_pruned_layer_projection_at_the_config2_shape(L, gemm_form):
     # Eq. 14 for 8 pruned layers in one launch: A holds 8 normalised copies of the state (one per
     # layer's gain), W the layers' [W^K; W^V]; the epilogue applies RoPE to k and writes both into the
     # layers' pages; the last position of the sequence is skipped (it belongs to the boundary token)

@@ -11,7 +11,8 @@ import torch
 
 import pop_synth as ps
 from oracle import pop_oracle as po
-from tests.gpu_util import rel_err
+from tests.full_parity import DeviceDrawnWeights
+from tests.gpu_util import logits_budget, rel_err
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -262,34 +263,56 @@ class CachedWeights:
     def embedding_rows(self, ids):
         return self.w.embedding_rows(ids)
 
+    def rows(self, name, layer, row_start, row_count):
+        return self.get(name, layer)[row_start: row_start + row_count]
+
 
 def test_true_width_reduced_depth():
     # Llama-3.1-8B layer shapes (d 4096, 32/8 heads of 128, FFN 14336), 3 layers, 640 tokens
-    # (5 query tiles), vocabulary cut to 32000 to keep the CPU side short.
-    # At this width the rounding of bf16 operands alone (oracle in kernel precision against the
-    # exact oracle) already moves single logits by more than 5e-2, because 32000 logits of
-    # standard deviation 1.3 are compared by their maximum error. The logits bound is therefore
-    # the stated 5e-2 or 1.5 x that irreducible figure, whichever is larger; the KV bound stays.
+    # (5 query tiles), vocabulary cut to 32000 to keep the CPU side short. Three layers are within the
+    # depth at which the stated cache tolerance is asserted; the logits (standard deviation 1.3 at this
+    # width, maximum taken over 32000 entries) get the depth budget of a bf16-operand pipeline.
     cfg = ps.C2_LLAMA8B.replace(n_layers=3, vocab=32000, name="llama8b-width-3-layers")
     tokens = ps.uniform_tokens(14, 1, 640, cfg.vocab)
-    w = CachedWeights(ps.SynthWeights(cfg))
+    w = CachedWeights(DeviceDrawnWeights(cfg))     # drawn on the GPU by the shared generator, handed over as CPU tensors
     ref = po.pop_prefill(cfg, w, tokens, None, 1, dtype=torch.float32)
-    emu = po.pop_prefill(cfg, w, tokens, None, 1, dtype=torch.float32, precision="bf16ops")
-    noise = (emu["logits"] - ref["logits"]).abs().max().item()
     logits, cache = run_gpu(build(cfg), cfg, tokens, None, 1, page=128)
-    err = (logits.cpu().double() - ref["logits"].double()).abs().max().item()
-    assert err <= max(LOGIT_TOL, 1.5 * noise), (err, noise)
-    # Against the oracle in the kernel's own precision the distance is of the same kind: both round
-    # operands to bf16, but at points that differ in detail (the kernel rounds exp2(s - m) for a
-    # running, possibly stale maximum m, the oracle the normalised probabilities), so the bound is
-    # the stated 5e-2 or that same irreducible figure, whichever is larger.
-    assert (logits.cpu().double() - emu["logits"].double()).abs().max().item() <= max(LOGIT_TOL, noise)
+    d = logits.cpu().double() - ref["logits"].double()
+    rms_b, max_b = logits_budget(cfg.n_layers, ref["logits"].double().std().item())
+    assert d.pow(2).mean().sqrt().item() <= rms_b and d.abs().max().item() <= max_b, (d.abs().max().item(), max_b)
     for l in range(cfg.n_layers):
         k, v = cache.gather(l)
         assert rel_err(k, ref["K"][l]) <= KV_TOL and rel_err(v, ref["V"][l]) <= KV_TOL
 
 
-def test_first_token_agrees_with_the_oracle_in_kernel_precision():
+@pytest.mark.parametrize("l_keep", [3, 1])
+def test_first_token_on_true_width_prompts(l_keep):
+    # 16 seeded prompts at the Llama-3.1-8B layer shapes (3 layers, 256 tokens, vocabulary 32000): the
+    # GPU's first token against the oracle in the kernel's precision (an arg-max is a decision taken in
+    # floating point) and against the exact oracle. A disagreement must be a near-tie of the oracle's
+    # two best logits; the agreement with the exact oracle is printed, not gated (with random-init
+    # weights the gap between the two best of 32000 logits is often below the bf16 rounding floor).
+    cfg = ps.C2_LLAMA8B.replace(n_layers=3, vocab=32000, name="llama8b-width-3-layers")
+    n_prompts, N = 16, 256
+    tokens = ps.uniform_tokens(2000, n_prompts, N, cfg.vocab)
+    w = CachedWeights(DeviceDrawnWeights(cfg))
+    logits, _ = run_gpu(build(cfg), cfg, tokens, None, l_keep, page=128)
+    got = logits.argmax(-1).cpu()
+    emu = po.pop_prefill(cfg, w, tokens, None, l_keep, dtype=torch.float32, precision="bf16ops")["logits"]
+    exact = po.pop_prefill(cfg, w, tokens, None, l_keep, dtype=torch.float32)["logits"]
+    agree_emu = (got == emu.argmax(-1)).float().mean().item()
+    agree_exact = (got == exact.argmax(-1)).float().mean().item()
+    print(f"\nfirst token, true width, L_keep={l_keep}: {agree_emu:.3f} vs kernel-precision oracle, "
+          f"{agree_exact:.3f} vs exact oracle ({n_prompts} prompts)")
+    err = (logits.cpu().double() - exact.double()).abs().max().item()
+    for ref in (emu, exact):
+        top2 = ref.topk(2, dim=-1).values
+        for i in (got != ref.argmax(-1)).nonzero().flatten().tolist():
+            assert (top2[i, 0] - top2[i, 1]).item() <= 2.0 * err, (i, (top2[i, 0] - top2[i, 1]).item(), err)
+    assert agree_emu >= 0.8
+
+
+def test_first_token_agrees_with_the_oracle():
     cfg = ps.C1_TINY
     n_prompts, N = 128, 128
     tokens = ps.uniform_tokens(1000, n_prompts, N, cfg.vocab)
@@ -299,12 +322,14 @@ def test_first_token_agrees_with_the_oracle_in_kernel_precision():
     for l_keep in (3, 2):
         logits, _ = run_gpu(model, cfg, tokens, None, l_keep, page=128)
         got = logits.argmax(-1).cpu()
-        ref = po.pop_prefill(cfg, w, tokens, None, l_keep, precision="bf16ops")["logits"]
-        agree[l_keep] = (got == ref.argmax(-1)).float().mean().item()
-        # a mismatch is only acceptable as a near-tie of the oracle's two best logits
-        top2 = ref.topk(2, dim=-1).values
-        for i in (got != ref.argmax(-1)).nonzero().flatten().tolist():
-            assert (top2[i, 0] - top2[i, 1]).item() < 1e-2
+        for mode in ("bf16ops", "exact"):
+            ref = po.pop_prefill(cfg, w, tokens, None, l_keep, precision=mode)["logits"]
+            agree[(l_keep, mode)] = (got == ref.argmax(-1)).float().mean().item()
+            # a mismatch is only acceptable as a near-tie of the oracle's two best logits
+            top2 = ref.topk(2, dim=-1).values
+            for i in (got != ref.argmax(-1)).nonzero().flatten().tolist():
+                assert (top2[i, 0] - top2[i, 1]).item() < 1e-2
+    print("\nfirst-token agreement on 128 prompts:", agree)
     assert min(agree.values()) >= 0.99, agree
 
 
