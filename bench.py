@@ -72,9 +72,9 @@ def resolve_workload(a) -> ps.Workload:
 
 
 # DRAM read+write bytes of one down-projection GEMM launch at the c2 layer shape, from the ncu capture
-# summarised in profiles/gemm_kernel_residual_proj_c2.md; valid only for the kernel source it was taken on.
-GEMM_TRAFFIC = {"bytes_per_launch": 1.345e9, "launch": "down projection, M 8192 N 4096 K 14336",
-                "gemm_cu_sha256": "b020e6f3dc461ff535a8595aa3cb4c3e2e020095c472c6b99ae5e15467c0139e"}
+# summarised in profiles/gemm_pair_kernel_c2.md; valid only for the kernel source it was taken on.
+GEMM_TRAFFIC = {"bytes_per_launch": 1.347e9, "launch": "down projection, M 8192 N 4096 K 14336 (CTA-pair form)",
+                "gemm_cu_sha256": "68800108d86750aba29104539d973f3f692986ddd9e11858b4cb80cc247c5f56"}
 
 
 def gemm_traffic():
@@ -419,7 +419,7 @@ def run_ours(a, wl):
                       "weight_stream_gbs": weight_bytes / (dec_ms * 1e-3) / 1e9,
                       "frac_of_measured_hbm": weight_bytes / (dec_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"]},
            "gpu_launches": int(launches * a.steps),
-           "roofline": {"kernel": "gemm_kernel (tcgen05 projection GEMM, all epilogues)", "bound": "tensor",
+           "roofline": {"kernel": "gemm_pair_kernel / gemm_kernel (tcgen05 projection GEMM, all epilogues)", "bound": "tensor",
                         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                         "frac": achieved_tf / peak_tf if peak_tf else None,
                         "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']})"

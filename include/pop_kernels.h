@@ -156,7 +156,10 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
  *  - All calls share the one array, which keeps whatever the previous call left. Each call
  *    overwrites every slot it later reads, so no clearing is needed, but two calls whose kernels
  *    may overlap on the GPU (different streams without an ordering between them) race on it:
- *    serialise them. Calls on one stream are safe.
+ *    serialise them. Calls on one stream are safe. The arrival counters of the split merge sit in a
+ *    second fixed array (4096 entries, one per sequence and kv head; with more than that a second
+ *    kernel merges the splits instead); it is not reachable from the host, starts at zero when the
+ *    library is loaded and every launch leaves it at zero again.
  * Errors: POP_E_INVALID (null pointer, bad head_dim or head counts), POP_E_NOSPACE (over the limit,
  * or block table too short), POP_E_CUDA. */
 #define POP_STATIC_SCRATCH_FLOATS (4 * 1024 * 1024)

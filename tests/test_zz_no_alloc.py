@@ -10,6 +10,7 @@ run alone in a fresh process (the first call on a device performs the one-time a
 import pytest
 import torch
 
+from oracle import pop_oracle as po
 from tests.gpu_util import paged_pools, rel_err
 
 pytestmark = pytest.mark.gpu
@@ -35,6 +36,10 @@ def _both(L, B, S, n_q, n_kv, hd, page, window, seed):
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated() == before      # torch's allocator was not touched either
     assert L.status() == 0
+    # and the arithmetic itself, not only the sibling: the oracle's attention of the same inputs (fp64)
+    ref = torch.stack([po.attention(q[b].cpu().double().reshape(1, n_q, hd), k[b].double(), v[b].double(),
+                                    torch.tensor([S - 1]), window).reshape(-1) for b in range(B)])
+    assert rel_err(got, ref) < 1e-2
     return got, want
 
 
