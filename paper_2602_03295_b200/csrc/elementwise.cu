@@ -72,7 +72,10 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, int64_t ldx, const f
   constexpr int RN_CACHE = 4;
   __shared__ float red[32];
   chain_trigger();
-  const int row = blockIdx.x, g = blockIdx.y;
+  // Rows are walked from the last to the first: the kernel that produced x wrote its highest rows last,
+  // so those are the ones still in L2, and the GEMM that consumes the output starts at row 0, which this
+  // order writes last.
+  const int row = gridDim.x - 1 - blockIdx.x, g = blockIdx.y;
   const float* xr = x + (int64_t)row * ldx;
   const float* gr = gain + (int64_t)g * gain_stride;
   const int step = blockDim.x * 4;

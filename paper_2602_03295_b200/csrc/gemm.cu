@@ -65,6 +65,7 @@ struct GemmDev {
   const float* ss_in; int ss_cnt; int ss_in_ld; float inv_d; float eps_in;
   const float* a_scale; const float* b_scale;      // FP8 operands: accumulator scale a_scale[row] * *b_scale
   int* status;                                     // device status word
+  int group_m;                                     // pair form: 256-row tiles per raster group
 };
 
 __device__ __forceinline__ void tile_coords(const GemmDev& p, int t, int& g, int& m, int& n) {
@@ -525,7 +526,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 //   tempty[b]  lives in the even CTA, counts the eight epilogue warps of both CTAs.
 constexpr int PSTAGES = 6;
 constexpr int PB_BYTES = 128 * BK * 2;      // this CTA's half of the B block
-constexpr int PAIR_GROUP_M = 8;             // raster: 8 x 256 rows share the same B columns in L2
 
 struct __align__(1024) PairGemmSmem {
   uint8_t a[PSTAGES][A_BYTES];
@@ -540,14 +540,17 @@ struct __align__(1024) PairGemmSmem {
   volatile uint32_t abort;
 };
 
+// Raster of the pair form: groups of group_m tile rows; inside a group the tile rows vary fastest, so
+// the CTA pairs working at any one time share a few B column panels and the group's A panel, which
+// stays in L2 while the group sweeps over all column tiles.
 __device__ __forceinline__ void pair_tile_coords(const GemmDev& p, int m_tiles2, int t, int& g, int& m, int& n) {
   const int per_batch = m_tiles2 * p.n_tiles;
   g = t / per_batch;
   const int r = t - g * per_batch;
-  const int span = PAIR_GROUP_M * p.n_tiles;
+  const int span = p.group_m * p.n_tiles;
   const int grp = r / span;
-  const int first_m = grp * PAIR_GROUP_M;
-  const int gsize = min(PAIR_GROUP_M, m_tiles2 - first_m);
+  const int first_m = grp * p.group_m;
+  const int gsize = min(p.group_m, m_tiles2 - first_m);
   const int rr = r - grp * span;
   m = first_m + rr % gsize;
   n = rr / gsize;
@@ -783,6 +786,14 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
 
 // CTA pairs pay off once every SM pair has at least one 256 x 256 tile; POP_GEMM_PAIR=0 / 1 in the
 // environment forces the single-CTA / the pair form (used by the tests to cover both on every shape).
+// Tile rows per raster group of the pair form. POP_GEMM_GROUP_M overrides (measurements).
+int pair_group_m(int K) {
+  const char* e = std::getenv("POP_GEMM_GROUP_M");
+  if (e && atoi(e) > 0) return atoi(e);
+  (void)K;
+  return 16;
+}
+
 bool use_pair(int M, int64_t tiles2, int sms) {
   const char* e = std::getenv("POP_GEMM_PAIR");
   if (e && e[0] == '0') return false;
@@ -881,6 +892,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
   int grid = (int)(total < sms ? total : sms);
   if (pair) grid = 2 * (int)(tiles2 < sms / 2 ? tiles2 : sms / 2);
+  p.group_m = pair_group_m(a.K);
   if (a.fp8) {
     switch (a.epilogue) {
       case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, pair, stream);
