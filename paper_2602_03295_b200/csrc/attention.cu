@@ -321,20 +321,50 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           if (!(j <= pos && j > lo)) sv[i] = -INFINITY;
         }
       }
-      float mx0 = sv[0], mx1 = sv[1], mx2 = sv[2], mx3 = sv[3];
+      // P = exp2(S * scale - m) with packed fp32 pairs, summed on two chains, rounded to bf16 (key 2c in
+      // the low half of packed column c, key 2c+1 in the high half). The exponentials are taken against
+      // the maximum the row already has: nothing in them depends on this tile's own maximum, which is
+      // reduced alongside (four chains of three-input max) and only checked afterwards.
+      float2 acc0, acc1;
+      uint32_t pk[BKV / 2];
+      float mx0, mx1, mx2, mx3;
+      auto exps = [&](float m_use) {
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+        const float2 nm2 = make_float2(-m_use, -m_use);
+        acc0 = make_float2(0.f, 0.f);
+        acc1 = make_float2(0.f, 0.f);
+        mx0 = sv[0]; mx1 = sv[2]; mx2 = sv[4]; mx3 = sv[6];
 #pragma unroll
-      for (int i = 4; i + 8 <= BKV; i += 8) {
-        mx0 = max3(mx0, sv[i], sv[i + 1]);
-        mx1 = max3(mx1, sv[i + 2], sv[i + 3]);
-        mx2 = max3(mx2, sv[i + 4], sv[i + 5]);
-        mx3 = max3(mx3, sv[i + 6], sv[i + 7]);
-      }
-      mx0 = max3(mx0, sv[BKV - 4], sv[BKV - 3]);
-      mx1 = max3(mx1, sv[BKV - 2], sv[BKV - 1]);
+        for (int c = 0; c < BKV / 8; ++c) {
+          float2 x0 = __ffma2_rn(make_float2(sv[c * 8 + 0], sv[c * 8 + 1]), sc2, nm2);
+          float2 x1 = __ffma2_rn(make_float2(sv[c * 8 + 2], sv[c * 8 + 3]), sc2, nm2);
+          float2 x2 = __ffma2_rn(make_float2(sv[c * 8 + 4], sv[c * 8 + 5]), sc2, nm2);
+          float2 x3 = __ffma2_rn(make_float2(sv[c * 8 + 6], sv[c * 8 + 7]), sc2, nm2);
+          mx0 = max3(mx0, sv[c * 8 + 0], sv[c * 8 + 1]);
+          mx1 = max3(mx1, sv[c * 8 + 2], sv[c * 8 + 3]);
+          mx2 = max3(mx2, sv[c * 8 + 4], sv[c * 8 + 5]);
+          mx3 = max3(mx3, sv[c * 8 + 6], sv[c * 8 + 7]);
+          x0.x = ex2(x0.x); x0.y = ex2(x0.y);
+          x1.x = ex2(x1.x); x1.y = ex2(x1.y);
+          x2.x = ex2(x2.x); x2.y = ex2(x2.y);
+          x3.x = ex2(x3.x); x3.y = ex2(x3.y);
+          acc0 = __fadd2_rn(acc0, x0);
+          acc1 = __fadd2_rn(acc1, x1);
+          acc0 = __fadd2_rn(acc0, x2);
+          acc1 = __fadd2_rn(acc1, x3);
+          pk[c * 4 + 0] = pack2(x0.x, x0.y);
+          pk[c * 4 + 1] = pack2(x1.x, x1.y);
+          pk[c * 4 + 2] = pack2(x2.x, x2.y);
+          pk[c * 4 + 3] = pack2(x3.x, x3.y);
+        }
+      };
+      exps(m_run == -INFINITY ? 0.f : m_run);
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;   // log2 domain
       const float m_new = fmaxf(m_run, mx);
       const bool need = (m_new - m_run > 8.0f) || (m_run == -INFINITY && m_new > -INFINITY);
       if (__any_sync(0xffffffffu, need)) {
+        // the maximum grew by more than 2^8 somewhere in this warp (in practice: a row's first tiles):
+        // rescale the accumulator to the new maximum and take the exponentials again
         const float factor = (m_new == -INFINITY) ? 1.0f : ex2(m_run - m_new);   // ex2(-inf) = 0
         if (jj > 0) {
           if (!wait_pv(jj - 1)) { ok = false; break; }
@@ -352,32 +382,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         l_run *= factor;
         m_run = m_new;
-      }
-      // P = exp2(S * scale - m) with packed fp32 pairs, summed on four chains, rounded to bf16
-      // (key 2c in the low half of packed column c, key 2c+1 in the high half)
-      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-      const float2 nm2 = make_float2(-m_use, -m_use);
-      float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-      uint32_t pk[BKV / 2];
-#pragma unroll
-      for (int c = 0; c < BKV / 8; ++c) {
-        float2 x0 = __ffma2_rn(make_float2(sv[c * 8 + 0], sv[c * 8 + 1]), sc2, nm2);
-        float2 x1 = __ffma2_rn(make_float2(sv[c * 8 + 2], sv[c * 8 + 3]), sc2, nm2);
-        float2 x2 = __ffma2_rn(make_float2(sv[c * 8 + 4], sv[c * 8 + 5]), sc2, nm2);
-        float2 x3 = __ffma2_rn(make_float2(sv[c * 8 + 6], sv[c * 8 + 7]), sc2, nm2);
-        x0.x = ex2(x0.x); x0.y = ex2(x0.y);
-        x1.x = ex2(x1.x); x1.y = ex2(x1.y);
-        x2.x = ex2(x2.x); x2.y = ex2(x2.y);
-        x3.x = ex2(x3.x); x3.y = ex2(x3.y);
-        acc0 = __fadd2_rn(acc0, x0);
-        acc1 = __fadd2_rn(acc1, x1);
-        acc0 = __fadd2_rn(acc0, x2);
-        acc1 = __fadd2_rn(acc1, x3);
-        pk[c * 4 + 0] = pack2(x0.x, x0.y);
-        pk[c * 4 + 1] = pack2(x1.x, x1.y);
-        pk[c * 4 + 2] = pack2(x2.x, x2.y);
-        pk[c * 4 + 3] = pack2(x3.x, x3.y);
+        exps(m_run == -INFINITY ? 0.f : m_run);
       }
       l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
       tmem_st_32x32b_x32(sp_addr, pk);      // over the scores this thread has just consumed
