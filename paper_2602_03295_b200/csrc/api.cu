@@ -44,7 +44,6 @@ struct Workspace {
   int32_t* tok;      // [B] current token of every sequence in the greedy loop
   int32_t* dec_ctr;  // [B][n_kv] arrival counters of the decode attention's split merge (zero between launches)
   float* a_scale;    // [M] row scales of FP8 activations
-  unsigned int* fuse_sync;   // [2] grid-barrier arrivals and abort flag of the fused decode kernel
   size_t total;
 };
 
@@ -150,7 +149,6 @@ Workspace carve(const pop_model* m, char* base, int N, int B) {
   w.tok = (int32_t*)take((size_t)B * 4);
   w.dec_ctr = (int32_t*)take((size_t)B * c.n_kv_heads * 4);
   w.a_scale = (float*)take(M * 4);
-  w.fuse_sync = (unsigned int*)take(2 * 4);
   w.total = o;
   return w;
 }
@@ -365,41 +363,6 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   return POP_OK;
 }
 
-// Layers first1 .. last1 (1-based) for the boundary token / a decode step. One sequence of a
-// configuration the fused kernel covers takes them in a single launch; everything else goes layer
-// by layer through the chain of single kernels.
-int boundary_layers(pop_model* m, const Workspace& w, int first1, int last1, int N, int B, const pop_kv_cache_t* kc,
-                    const float2* table, int table_pos0, cudaStream_t s, const int32_t* pos_dev = nullptr,
-                    const int32_t* layer_first_pos = nullptr) {
-  if (first1 > last1) return POP_OK;
-  const pop_config_t& c = m->cfg;
-  if (layer_first_pos == nullptr && decode_fused_supported(c, B, m->fp8 != nullptr)) {
-    FusedDecodeArgs a{};
-    a.layer_base = m->arena; a.layer_stride = (int64_t)m->layer_stride;
-    a.off_ln_in = (int64_t)m->lo.ln_in; a.off_wqkv = (int64_t)m->lo.wqkv; a.off_qn = (int64_t)m->lo.q_norm;
-    a.off_kn = (int64_t)m->lo.k_norm; a.off_wo = (int64_t)m->lo.wo; a.off_ln_ffn = (int64_t)m->lo.ln_ffn;
-    a.off_wgu = (int64_t)m->lo.wgu; a.off_wd = (int64_t)m->lo.wd;
-    a.layer_first = first1 - 1; a.n_layers = last1 - first1 + 1;
-    a.d = c.d_model; a.d_ffn = c.d_ffn; a.n_q = c.n_q_heads; a.n_kv = c.n_kv_heads;
-    a.q_dim = m->q_dim; a.kv_dim = m->kv_dim; a.qkv_dim = m->qkv_dim; a.act = c.act; a.qk_norm = c.qk_norm;
-    a.window = c.window; a.global_every = c.global_every; a.eps = c.rms_eps;
-    a.xb = w.xb; a.qkv = w.qkvb; a.ob = w.ob; a.ab = w.ab; a.partial = w.partial;
-    a.rope_row = pos_dev ? table : table + (int64_t)(N - 1 - table_pos0) * (c.head_dim / 2);
-    a.k_pool = (bf16*)kc->k_pool; a.v_pool = (bf16*)kc->v_pool;
-    a.pool_layer_stride = (int64_t)kc->num_pages * kc->page_size * m->kv_dim;
-    a.block_table = kc->block_table; a.page_size = kc->page_size; a.num_pages = kc->num_pages;
-    a.pos = N - 1; a.pos_dev = pos_dev;
-    a.counters = reinterpret_cast<unsigned int*>(w.dec_ctr);
-    a.sync = w.fuse_sync;
-    if (cudaMemsetAsync(w.fuse_sync, 0, 2 * sizeof(unsigned int), s) != cudaSuccess) return POP_E_CUDA;
-    return launch_decode_fused(a, s);
-  }
-  for (int l = first1; l <= last1; ++l)
-    POP_TRY(boundary_layer(m, w, l, N, B, kc, table, table_pos0, s, nullptr, pos_dev,
-                           layer_first_pos ? layer_first_pos[l - 1] : 0));
-  return POP_OK;
-}
-
 int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, pop_kv_cache_t* kc, float* logits,
                 cudaStream_t s) {
   if (!m || !in || !in->tokens || !kc || !kc->k_pool || !kc->v_pool || !kc->block_table || !logits)
@@ -430,7 +393,7 @@ int run_prefill(pop_model* m, const pop_input_t* in, int N, int B, int L_keep, p
       }
     }
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
-    POP_TRY(boundary_layers(m, w, L_keep + 1, c.n_layers, N, B, kc, w.rope, 0, s));
+    for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, 0, s));
   } else {
     POP_TRY(launch_gather_rows(w.x, w.xb, B, d, N, N - 1, s));
   }
@@ -486,7 +449,7 @@ int run_prefill_chunked(pop_model* m, const pop_input_t* in, int N, int B, int L
     }
     if (last) {
       POP_TRY(launch_gather_rows(w.x, w.xb, B, d, n, n - 1, s));
-      POP_TRY(boundary_layers(m, w, L_keep + 1, c.n_layers, N, B, kc, w.rope, p0, s));
+      for (int l = L_keep + 1; l <= c.n_layers; ++l) POP_TRY(boundary_layer(m, w, l, N, B, kc, w.rope, p0, s));
     }
   }
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
@@ -614,7 +577,9 @@ int decode_body(pop_model* m, const Workspace& w, const int32_t* tokens, int pos
   const int d = c.d_model;
   POP_TRY(launch_rope_table(w.rope1, 1, c.head_dim, c.rope_theta, s, pos, pos_dev));
   POP_TRY(launch_embed(tokens, (const bf16*)(m->arena + m->off_embed), nullptr, w.xb, B, d, c.vocab, s));
-  POP_TRY(boundary_layers(m, w, 1, c.n_layers, pos + 1, B, kc, w.rope1, pos, s, pos_dev, layer_first_pos));
+  for (int l = 1; l <= c.n_layers; ++l)
+    POP_TRY(boundary_layer(m, w, l, pos + 1, B, kc, w.rope1, pos, s, nullptr, pos_dev,
+                           layer_first_pos ? layer_first_pos[l - 1] : 0));
   POP_TRY(launch_rmsnorm(w.xb, d, (const float*)(m->arena + m->off_final_norm), 0, w.hb32, d, 0, B, d, 1, c.rms_eps,
                          true, s));
   GemvArgs v{};

@@ -230,32 +230,4 @@ struct DecAttnArgs {
 int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);
 
-// One position of one sequence through layers layer_first .. layer_first + n_layers - 1 in a single
-// cooperative kernel (decode_fused.cu). decode_fused_supported() says whether a configuration qualifies;
-// the caller zeroes `sync` (two words) and `counters` on the stream before the launch.
-struct FusedDecodeArgs {
-  const char* layer_base;       // arena address of layer 0's block
-  int64_t layer_stride;         // bytes
-  int64_t off_ln_in, off_wqkv, off_qn, off_kn, off_wo, off_ln_ffn, off_wgu, off_wd;
-  int layer_first, n_layers;    // layers layer_first .. layer_first + n_layers - 1 (0-based)
-  int d, d_ffn, n_q, n_kv, q_dim, kv_dim, qkv_dim, act, qk_norm;
-  int window, global_every;
-  float eps, scale_log2;
-  float* xb;                    // [d] residual stream of the position
-  float* qkv;                   // [qkv_dim]
-  bf16* ob;                     // [q_dim]
-  bf16* ab;                     // [d_ffn]
-  float* partial;               // [n_q][splits][hd + 2]
-  const float2* rope_row;       // [hd/2] cos, sin of the position
-  bf16* k_pool; bf16* v_pool; int64_t pool_layer_stride;
-  const int32_t* block_table; int page_size; int num_pages;
-  int pos; const int32_t* pos_dev;
-  unsigned int* counters;       // [n_kv], zero before and after
-  unsigned int* sync;           // [0] arrivals at the grid barriers, [1] abort flag; both zero at launch
-  int* status;
-  int splits;
-};
-bool decode_fused_supported(const pop_config_t& c, int batch, bool fp8);
-int launch_decode_fused(const FusedDecodeArgs& a, cudaStream_t s);
-
 }  // namespace pop
