@@ -19,13 +19,14 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// 8 bf16 -> fp32 with a shift and a mask per pair: a bf16 is the upper half of the fp32 of the same
+// value, and the integer pipe is wider than the conversion unit
 __device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
-  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float2 t = __bfloat1622float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
 }
 
