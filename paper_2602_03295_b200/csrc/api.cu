@@ -306,19 +306,12 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   const float* sc8 = m->fp8 ? m->fp8_scales + 4 * (l - 1) : nullptr;
   if (w8) { v.w = w8; v.w_fp8 = true; v.w_scale = sc8; }
   POP_TRY(launch_gemv(v, s));
-  RopeArgs r{};
-  r.in = w.qkvb; r.ld_in = m->qkv_dim; r.q_out = w.qb; r.ldq = m->q_dim;
-  r.k_pool = (bf16*)kc->k_pool; r.v_pool = (bf16*)kc->v_pool; r.pool_layer_stride = pool_layer_stride;
-  r.layer0 = l - 1; r.block_table = kc->block_table; r.max_pages_per_seq = kc->max_pages_per_seq;
-  r.page_size = kc->page_size; r.num_pages = kc->num_pages;
-  r.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
-  r.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
-  r.table = table; r.table_pos0 = table_pos0; r.n_q = c.n_q_heads; r.n_kv = c.n_kv_heads; r.hd = c.head_dim;
-  r.rows = B; r.rows_per_seq = 1; r.rows_written = 1; r.pos0 = N - 1; r.groups = 1; r.eps = c.rms_eps;
-  r.cu_seqlens = cu; r.batch = B; r.pos_dev = pos_dev;
-  POP_TRY(launch_rope_cache(r, s));
+  // per-head norm, RoPE and the cache append of the new position happen inside the attention kernel
   DecAttnArgs a{};
-  a.q = w.qb; a.ldq = m->q_dim;
+  a.qkv = w.qkvb; a.ld_qkv = m->qkv_dim;
+  a.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
+  a.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
+  a.table = table; a.table_pos0 = table_pos0; a.eps = c.rms_eps;
   a.k_pool = (const bf16*)kc->k_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.v_pool = (const bf16*)kc->v_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.block_table = kc->block_table; a.max_pages_per_seq = kc->max_pages_per_seq; a.page_size = kc->page_size;

@@ -226,6 +226,15 @@ struct DecAttnArgs {
   // attention kernel merges its own splits (one launch); without, a second kernel does
   int32_t* counters;
   int num_pages;               // pages in the pool, for the device-side block-table check (0 = no check)
+  // Optional: finish the projection inside the attention kernel instead of a kernel of its own. With
+  // `qkv` set (fp32 rows [q heads | k heads | v heads] * hd, one per sequence, straight from the QKV
+  // GEMV) every CTA applies the per-head norm (gains or null) and the rotary row to its own query
+  // heads, and the CTA whose key range holds the newest position does the same for that position's
+  // key, appends key and value to the (then writable) pools and takes them from there; `q` is unused.
+  const float* qkv; int64_t ld_qkv;
+  const float* q_gain; const float* k_gain;
+  const float2* table; int table_pos0;   // as in RopeArgs
+  float eps;
 };
 int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

@@ -262,6 +262,11 @@ struct DecAttnDev {
   unsigned int* counters;
   int num_pages;                           // block-table entries are checked against it when > 0
   int* status;                             // device status word
+  // projection finished in this kernel (see DecAttnArgs::qkv); null = q holds finished queries
+  const float* qkv; int64_t ld_qkv;
+  const float* q_gain; const float* k_gain;
+  const float2* table; int table_pos0;
+  float eps;
 };
 
 constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of one MMA
@@ -371,11 +376,79 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   const int n_groups = j1 > j0 ? (j1 - j0 + KT - 1) / KT : 0;
   const int n_mine = n_groups > warp ? (n_groups - warp + WARPS - 1) / WARPS : 0;
 
+  const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
+  __shared__ __align__(16) bf16 q_fin[DEC_MAXG * HD];
+  if (p.qkv != nullptr) {
+    // Finish the projection here: per-head norm, rotary row of the newest position kv_len - 1. Every
+    // CTA does its own G query heads (to shared memory); the CTA whose range holds that position also
+    // does the key, and writes key and value into the cache before any of its warps loads that range.
+    constexpr int PER = HD / 64;
+    const int pos = kv_len - 1;
+    const bool owner = pos >= j0 && pos < j1;
+    const float* row = p.qkv + (int64_t)b * p.ld_qkv;
+    const int q_dim = p.n_q * HD, kv_dim = p.n_kv * HD;
+    const float2* trow = p.table + (int64_t)(p.pos_dev ? 0 : pos - p.table_pos0) * (HD / 2);
+    for (int it = warp; it < G + (owner ? 2 : 0); it += WARPS) {
+      const bool is_q = it < G, is_k = it == G;
+      const float* src = row + (is_q ? (int64_t)(kvh * G + it) * HD
+                                     : (is_k ? (int64_t)q_dim + kvh * HD : (int64_t)q_dim + kv_dim + kvh * HD));
+      float lo[PER], hi[PER];
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        lo[u] = src[lane + 32 * u];
+        hi[u] = src[lane + 32 * u + HD / 2];
+      }
+      if (is_q || is_k) {
+        const float* gain = is_q ? p.q_gain : p.k_gain;
+        if (gain != nullptr) {
+          float ss = 0.f;
+#pragma unroll
+          for (int u = 0; u < PER; ++u) ss += lo[u] * lo[u] + hi[u] * hi[u];
+          ss = warp_sum(ss);
+          const float rstd = rsqrtf(ss / (float)HD + p.eps);
+#pragma unroll
+          for (int u = 0; u < PER; ++u) {
+            lo[u] = lo[u] * rstd * gain[lane + 32 * u];
+            hi[u] = hi[u] * rstd * gain[lane + 32 * u + HD / 2];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+          const float2 cs = trow[lane + 32 * u];
+          const float a = lo[u] * cs.x - hi[u] * cs.y;
+          const float c = hi[u] * cs.x + lo[u] * cs.y;
+          lo[u] = a;
+          hi[u] = c;
+        }
+      }
+      bf16* dst;
+      if (is_q) {
+        dst = q_fin + it * HD;
+      } else {
+        const int page = bt[pos / p.page_size];
+        if (p.num_pages > 0 && (unsigned)page >= (unsigned)p.num_pages) {
+          if (lane == 0) atomicMin(p.status, (int)POP_E_INVALID);     // never turned into an address
+          continue;
+        }
+        bf16* pool = const_cast<bf16*>(is_k ? p.k_pool : p.v_pool);
+        dst = pool + (((int64_t)page * p.page_size + pos % p.page_size) * p.n_kv + kvh) * HD;
+      }
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        dst[lane + 32 * u] = __float2bfloat16_rn(lo[u]);
+        dst[lane + 32 * u + HD / 2] = __float2bfloat16_rn(hi[u]);
+      }
+    }
+    __threadfence();      // the cache rows are read back below through asynchronous copies
+    __syncthreads();
+  }
   // Q^T as the B operand: thread holds head lane/4, dims 16 ks + 2 (lane%4) + {0, 1} and + 8
   uint32_t qb[NT][2];
   {
     const int g = lane >> 2;
-    const bf16* qrow = p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + (g < G ? g : 0)) * HD + (lane & 3) * 2;
+    const bf16* qrow = (p.qkv != nullptr ? q_fin + (g < G ? g : 0) * HD
+                                         : p.q + (int64_t)b * p.ldq + (int64_t)(kvh * G + (g < G ? g : 0)) * HD) +
+                       (lane & 3) * 2;
 #pragma unroll
     for (int ks = 0; ks < NT; ++ks) {
       qb[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
@@ -388,7 +461,6 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
 #pragma unroll
   for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
-  const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dec_smem) + warp * (NST * C::STAGE);
 
   auto issue = [&](int it) {
@@ -655,9 +727,12 @@ int launch_dec_by_head_dim(const DecAttnDev& p, int head_dim, int batch, cudaStr
 }
 
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
-  if (!a.q || !a.k_pool || !a.v_pool || !a.block_table || !a.partial || !a.out) return POP_E_INVALID;
+  if ((!a.q && !a.qkv) || !a.k_pool || !a.v_pool || !a.block_table || !a.partial || !a.out) return POP_E_INVALID;
+  if (a.qkv && !a.table) return POP_E_INVALID;
   if (a.n_q % a.n_kv || a.n_q / a.n_kv > DEC_MAXG || a.kv_len < 1) return POP_E_INVALID;
   DecAttnDev p;
+  p.qkv = a.qkv; p.ld_qkv = a.ld_qkv; p.q_gain = a.q_gain; p.k_gain = a.k_gain;
+  p.table = a.table; p.table_pos0 = a.table_pos0; p.eps = a.eps;
   p.q = a.q; p.ldq = a.ldq;
   p.k_pool = a.k_pool; p.v_pool = a.v_pool;
   p.block_table = a.block_table; p.max_pages_per_seq = a.max_pages_per_seq; p.page_size = a.page_size;
@@ -748,6 +823,7 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.block_table = block_table; p.max_pages_per_seq = max_pages_per_seq; p.page_size = page_size;
   p.num_pages = 0;
   p.status = nullptr;
+  p.qkv = nullptr; p.ld_qkv = 0; p.q_gain = p.k_gain = nullptr; p.table = nullptr; p.table_pos0 = 0; p.eps = 0.f;
   p.partial = scratch;
   p.out = static_cast<bf16*>(out); p.ldo = ldo;
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
