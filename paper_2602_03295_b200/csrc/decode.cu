@@ -362,7 +362,13 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   constexpr uint32_t FULL = 0xffffffffu;
   extern __shared__ __align__(128) uint8_t dec_smem[];
   chain_trigger();
-  chain_wait();   // the query, the newest cache row and the run-time length come from earlier kernels
+  // Finished queries and the newest cache row come from the kernel just before this one. When this
+  // kernel finishes the projection itself (p.qkv), only the fp32 projection row does: the cache rows of
+  // the older positions, the block table and the run-time length were written at least two kernels
+  // back, i.e. by kernels that are complete (every kernel of a chain waits for its predecessor), so
+  // the first loads of the cache go out before the wait and overlap the predecessor's tail.
+  const bool early = p.qkv != nullptr;
+  if (!early) chain_wait();
   const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
   const int G = p.n_q / p.n_kv;   // <= DEC_MAXG
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -378,6 +384,54 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
 
   const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
   __shared__ __align__(16) bf16 q_fin[DEC_MAXG * HD];
+  // this thread's two heads are 2 (lane%4) and 2 (lane%4) + 1, its keys of a group lane/4 and lane/4 + 8
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  float o[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dec_smem) + warp * (NST * C::STAGE);
+
+  auto issue = [&](int it) {
+    const int jg = j0 + (warp + it * WARPS) * KT;
+    const uint32_t st = ring + (it % NST) * C::STAGE;
+    // lanes 0..15 (and again 16..31) each find the pool row of one key of the group; -1 past the chunk
+    const int jk = jg + (lane & 15);
+    int row = -1;
+    if (jk < j1) {
+      const int page = bt[jk / p.page_size];
+      if (p.num_pages > 0 && (unsigned)page >= (unsigned)p.num_pages)
+        atomicMin(p.status, (int)POP_E_INVALID);     // never turned into an address: the key reads as zeros
+      else
+        row = page * p.page_size + jk % p.page_size;
+    }
+#pragma unroll
+    for (int i = 0; i < KT * CH / 32; ++i) {
+      const int idx = i * 32 + lane;
+      const int key = idx / CH, ch = idx % CH;
+      const int r = __shfl_sync(FULL, row, key);
+      const int64_t off = r < 0 ? 0 : ((int64_t)r * p.n_kv + kvh) * HD + ch * 8;
+      const int nbytes = r < 0 ? 0 : 16;
+      // 16-byte chunks of a row are permuted by the key's low bits: the 8 rows one matrix load
+      // touches fall in different banks
+      const uint32_t dst = st + key * ROWB + ((ch ^ (key & 7)) << 4);
+      cp_async16(dst, p.k_pool + off, nbytes);
+      cp_async16(dst + KT * ROWB, p.v_pool + off, nbytes);
+    }
+  };
+
+  // the newest position's group (the last one of the range that holds it) has to wait for the append
+  const bool holds_new = early && kv_len - 1 >= j0 && kv_len - 1 < j1;
+  int deferred = -1;
+#pragma unroll
+  for (int i = 0; i < NST; ++i) {
+    if (i < n_mine) {
+      if (holds_new && warp == (n_groups - 1) % WARPS && i == n_mine - 1) deferred = i;
+      else issue(i);
+    }
+    cp_async_commit();
+  }
+  if (early) chain_wait();
   if (p.qkv != nullptr) {
     // Finish the projection here: per-head norm, rotary row of the newest position kv_len - 1. Every
     // CTA does its own G query heads (to shared memory); the CTA whose range holds that position also
@@ -441,6 +495,10 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
     }
     __threadfence();      // the cache rows are read back below through asynchronous copies
     __syncthreads();
+    if (deferred >= 0) {
+      issue(deferred);
+      cp_async_commit();
+    }
   }
   // Q^T as the B operand: thread holds head lane/4, dims 16 ks + 2 (lane%4) + {0, 1} and + 8
   uint32_t qb[NT][2];
@@ -455,47 +513,6 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
       qb[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
     }
   }
-  // this thread's two heads are 2 (lane%4) and 2 (lane%4) + 1, its keys of a group lane/4 and lane/4 + 8
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  float o[NT][4];
-#pragma unroll
-  for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
-
-  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dec_smem) + warp * (NST * C::STAGE);
-
-  auto issue = [&](int it) {
-    const int jg = j0 + (warp + it * WARPS) * KT;
-    const uint32_t st = ring + (it % NST) * C::STAGE;
-    // lanes 0..15 (and again 16..31) each find the pool row of one key of the group; -1 past the chunk
-    const int jk = jg + (lane & 15);
-    int row = -1;
-    if (jk < j1) {
-      const int page = bt[jk / p.page_size];
-      if (p.num_pages > 0 && (unsigned)page >= (unsigned)p.num_pages)
-        atomicMin(p.status, (int)POP_E_INVALID);     // never turned into an address: the key reads as zeros
-      else
-        row = page * p.page_size + jk % p.page_size;
-    }
-#pragma unroll
-    for (int i = 0; i < KT * CH / 32; ++i) {
-      const int idx = i * 32 + lane;
-      const int key = idx / CH, ch = idx % CH;
-      const int r = __shfl_sync(FULL, row, key);
-      const int64_t off = r < 0 ? 0 : ((int64_t)r * p.n_kv + kvh) * HD + ch * 8;
-      const int nbytes = r < 0 ? 0 : 16;
-      // 16-byte chunks of a row are permuted by the key's low bits: the 8 rows one matrix load
-      // touches fall in different banks
-      const uint32_t dst = st + key * ROWB + ((ch ^ (key & 7)) << 4);
-      cp_async16(dst, p.k_pool + off, nbytes);
-      cp_async16(dst + KT * ROWB, p.v_pool + off, nbytes);
-    }
-  };
-
-#pragma unroll
-  for (int i = 0; i < NST; ++i) {
-    if (i < n_mine) issue(i);
-    cp_async_commit();
-  }
   // matrix-load addresses of this lane (lane = 8 * matrix + row of the matrix)
   const int mi = lane >> 3, r8 = lane & 7;
   const uint32_t k_lane = ((mi & 1) * 8 + r8) * ROWB;          // K: matrices (keys 0-7 | 8-15) x (chunk 2ks | 2ks+1)
@@ -503,7 +520,8 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   const int kr = lane >> 2;
 
   for (int it = 0; it < n_mine; ++it) {
-    cp_async_wait<NST - 1>();
+    if (it == deferred) cp_async_wait<0>();      // its copies were committed after the others
+    else cp_async_wait<NST - 1>();
     __syncwarp();
     const uint32_t st = ring + (it % NST) * C::STAGE;
     const int jg = j0 + (warp + it * WARPS) * KT;
