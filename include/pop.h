@@ -222,7 +222,7 @@ int pop_decode_step(pop_model_t* m, const int32_t* tokens, int32_t pos, int32_t 
  * the token at position pos0 + i + 1. logits_scratch is device fp32 [batch][vocab] (it holds the
  * last step's logits afterwards). One step is captured into a CUDA graph whose kernels read the
  * position from device memory, and that graph is launched n_steps times on `stream`, so the host
- * issues n_steps graph launches instead of n_steps x (9 n_layers + 5) kernel launches. The call
+ * issues n_steps graph launches instead of n_steps x (7 n_layers + 5) kernel launches (9 per layer for a model with post-norms). The call
  * creates and destroys a stream and a graph of its own (host-side objects; no device memory).
  * Not available while pop_k_profile is on. The cache must have room for pos0 + n_steps positions. */
 int pop_generate_greedy(pop_model_t* m, const int32_t* first_tokens, int32_t pos0, int32_t n_steps, int32_t batch,
