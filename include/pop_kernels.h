@@ -138,6 +138,23 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
                            int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
                            int32_t head_dim, int32_t kv_len, int32_t window, void* stream);
 
+/* pop_k_decode_attention with the end of the projection folded in (paper Eq. 2-3 for the one new
+ * position, then Attn of Eq. 1; Sec. 3.3): instead of finished queries the kernel takes the fp32 row
+ * qkv[b] = [q heads | k heads | v heads] * head_dim of every sequence (ld_qkv floats apart), applies the
+ * per-head RMSNorm (q_gain / k_gain: fp32 [head_dim], or both NULL for none; eps) and the rotary row
+ * of position kv_len - 1 (table: device float2 [head_dim / 2] pairs (cos, sin) of that one position) to
+ * the queries and the key, appends key and value at position kv_len - 1 of the cache (k_pool and
+ * v_pool are WRITTEN here: one layer, [num_pages][page_size][n_kv][head_dim]), and attends over
+ * positions max(0, kv_len - window) .. kv_len - 1 (window 0: all). counters (device int32
+ * [batch * n_kv], zero before and after) are required: the call is a single launch. A block-table
+ * entry outside [0, num_pages) is never dereferenced; the status word is raised to POP_E_INVALID.
+ * This is the form the boundary-token / decode path of pop_prefill and pop_decode_step runs. */
+int pop_k_decode_attention_qkv(const float* qkv, int64_t ld_qkv, const float* q_gain, const float* k_gain, float eps,
+                               const void* rope_row, void* k_pool, void* v_pool, const int32_t* block_table,
+                               int32_t max_pages_per_seq, int32_t page_size, int32_t num_pages, float* partial,
+                               int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
+                               int32_t head_dim, int32_t kv_len, int32_t window, void* stream);
+
 /* The same single-query attention as pop_k_decode_attention for callers that have no way to hand
  * over a scratch buffer because they cannot allocate device memory at the point of the call: code
  * running inside a host callback or a real-time serving loop where cudaMalloc is forbidden, or a

@@ -99,6 +99,8 @@ SIGNATURES = {
                          + [_I32] * 8 + [_F, _P]),
     "pop_k_gemv": (C.c_int, [_P, _I64, _I32, _P, _I64, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_decode_attention": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _P, _P, _I64] + [_I32] * 6 + [_P]),
+    "pop_k_decode_attention_qkv": (C.c_int, [_P, _I64, _P, _P, C.c_float, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P,
+                                             _I64] + [_I32] * 6 + [_P]),
     "pop_k_decode_attention_static": (C.c_int, [_P, _I64, _P, _P, _P, _I32, _I32, _P, _I64] + [_I32] * 6 + [_P]),
     "pop_k_profile": (None, [_I32]),
     "pop_k_profile_summary": (C.c_int, [_I32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_I64)]),
@@ -332,6 +334,22 @@ class PopLibrary:
                                                out.data_ptr(), out.stride(0), batch, n_q, n_kv,
                                                hd, kv_len, window, _stream_ptr(stream))
         self.check(code, "pop_k_decode_attention")
+        return out
+
+    def decode_attention_qkv(self, qkv, q_gain, k_gain, eps, rope_row, k_pool, v_pool, block_table, out, n_q, n_kv, hd,
+                             kv_len, page_size, counters, window=0, partial=None, stream=None):
+        """pop_k_decode_attention_qkv: qkv fp32 [B, (n_q + 2 n_kv) hd]; rope_row float2 [hd/2] of position
+        kv_len - 1; pools of one layer [pages, page_size, n_kv, hd] (the new position is appended)."""
+        batch = qkv.shape[0]
+        if partial is None:
+            partial = torch.empty(batch * n_q * 64 * (hd + 2), dtype=torch.float32, device=qkv.device)
+        code = self.dll.pop_k_decode_attention_qkv(
+            qkv.data_ptr(), qkv.stride(0), 0 if q_gain is None else q_gain.data_ptr(),
+            0 if k_gain is None else k_gain.data_ptr(), eps, rope_row.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+            block_table.data_ptr(), block_table.shape[1], page_size, k_pool.shape[0], partial.data_ptr(),
+            counters.data_ptr(), out.data_ptr(), out.stride(0), batch, n_q, n_kv, hd, kv_len, window,
+            _stream_ptr(stream))
+        self.check(code, "pop_k_decode_attention_qkv")
         return out
 
     def decode_attention_static(self, q, k_pool, v_pool, block_table, out, n_q, n_kv, hd, kv_len, page_size,

@@ -169,6 +169,26 @@ int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const
   return launch_decode_attention(a, static_cast<cudaStream_t>(stream));
 }
 
+int pop_k_decode_attention_qkv(const float* qkv, int64_t ld_qkv, const float* q_gain, const float* k_gain, float eps,
+                               const void* rope_row, void* k_pool, void* v_pool, const int32_t* block_table,
+                               int32_t max_pages_per_seq, int32_t page_size, int32_t num_pages, float* partial,
+                               int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,
+                               int32_t head_dim, int32_t kv_len, int32_t window, void* stream) {
+  if (!qkv || !rope_row || !counters || (q_gain == nullptr) != (k_gain == nullptr)) return POP_E_INVALID;
+  if (batch < 1 || page_size < 1 || num_pages < 1 || kv_len < 1) return POP_E_INVALID;
+  if ((int64_t)ceil_div(kv_len, page_size) > max_pages_per_seq) return POP_E_NOSPACE;
+  DecAttnArgs a{};
+  a.counters = counters;
+  a.qkv = qkv; a.ld_qkv = ld_qkv; a.q_gain = q_gain; a.k_gain = k_gain; a.eps = eps;
+  a.table = static_cast<const float2*>(rope_row); a.table_pos0 = kv_len - 1;
+  a.k_pool = static_cast<const bf16*>(k_pool); a.v_pool = static_cast<const bf16*>(v_pool);
+  a.block_table = block_table; a.max_pages_per_seq = max_pages_per_seq; a.page_size = page_size;
+  a.num_pages = num_pages;
+  a.partial = partial; a.out = static_cast<bf16*>(out); a.ldo = ldo;
+  a.batch = batch; a.n_q = n_q; a.n_kv = n_kv; a.head_dim = head_dim; a.kv_len = kv_len; a.window = window;
+  return launch_decode_attention(a, static_cast<cudaStream_t>(stream));
+}
+
 const char* pop_strerror(int status) {
   switch (status) {
     case POP_OK: return "ok";

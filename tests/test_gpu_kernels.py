@@ -311,6 +311,47 @@ def test_decode_attention(L, B, S, n_q, n_kv, hd, page, window):
         assert (ctr == 0).all()
 
 
+@pytest.mark.parametrize("B,S,n_q,n_kv,hd,page,window,norm", [(1, 1, 4, 2, 64, 16, 0, False), (2, 37, 8, 2, 128, 16, 0, True),
+                                                              (1, 1000, 32, 8, 128, 128, 0, False),
+                                                              (3, 300, 4, 1, 256, 64, 96, True),
+                                                              (1, 2049, 8, 8, 64, 128, 0, True)])
+def test_decode_attention_with_the_projection_finish(L, B, S, n_q, n_kv, hd, page, window, norm):
+    # the form the boundary / decode path runs (Eq. 2-3 for the new position, then Attn of Eq. 1): fp32 QKV row in,
+    # per-head norm + RoPE + cache append inside the attention kernel
+    theta, eps = 10000.0, 1e-6
+    g = torch.Generator().manual_seed(30)
+    qkv = torch.randn(B, (n_q + 2 * n_kv) * hd, generator=g)
+    k_old, v_old = _bf((B, S, n_kv, hd), 31, 1.0), _bf((B, S, n_kv, hd), 32, 1.0)
+    kp, vp, bt = paged_pools(k_old, v_old, page)
+    # the slot of position S - 1 holds garbage until the kernel appends
+    for b in range(B):
+        kp[bt[b, (S - 1) // page].long(), (S - 1) % page] = float("nan")
+        vp[bt[b, (S - 1) // page].long(), (S - 1) % page] = float("nan")
+    qg = (1.0 + 0.1 * torch.randn(hd, generator=g)) if norm else None
+    kg = (1.0 + 0.1 * torch.randn(hd, generator=g)) if norm else None
+    table = torch.zeros(S, hd // 2, 2, dtype=torch.float32, device=DEV)
+    L.rope_table(table, S, hd, theta)
+    kp, vp = kp.to(DEV), vp.to(DEV)
+    out = torch.full((B, n_q * hd), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ctr = torch.zeros(B * n_kv, dtype=torch.int32, device=DEV)
+    L.decode_attention_qkv(qkv.to(DEV), None if qg is None else qg.to(DEV), None if kg is None else kg.to(DEV), eps,
+                           table[S - 1], kp, vp, bt.to(DEV), out, n_q, n_kv, hd, S, page, ctr, window)
+    assert L.status() == 0 and (ctr == 0).all()
+    x = qkv.double().reshape(B, 1, n_q + 2 * n_kv, hd)
+    q, kn, vn = x[:, :, :n_q], x[:, :, n_q:n_q + n_kv], x[:, :, n_q + n_kv:]
+    if norm:
+        q, kn = po.rmsnorm(q, qg.double(), eps), po.rmsnorm(kn, kg.double(), eps)
+    pos = torch.tensor([S - 1])
+    q, kn = po.rope(q, pos, theta), po.rope(kn, pos, theta)
+    for b in range(B):
+        K = torch.cat([k_old[b, : S - 1].double(), kn[b]]), torch.cat([v_old[b, : S - 1].double(), vn[b]])
+        ref = po.attention(q[b], K[0], K[1], pos, window).reshape(-1)
+        assert rel_err(out[b], ref) < 1e-2, b
+        page_id, slot = bt[b, (S - 1) // page].long(), (S - 1) % page
+        assert rel_err(kp[page_id, slot], kn[b, 0]) < 1e-2 and rel_err(vp[page_id, slot], vn[b, 0]) < 1e-2
+    assert not torch.isnan(out.float()).any()
+
+
 def test_generators_agree_between_cpu_and_gpu():
     tid = ps.tensor_id("wq", 2)
     a = ps.normal_bf16(3, tid, (300, 1000), 0.02)
