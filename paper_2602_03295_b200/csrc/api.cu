@@ -312,6 +312,7 @@ int boundary_layer(pop_model* m, const Workspace& w, int l, int N, int B, const 
   a.q_gain = c.qk_norm ? lp<float>(m, l, m->lo.q_norm) : nullptr;
   a.k_gain = c.qk_norm ? lp<float>(m, l, m->lo.k_norm) : nullptr;
   a.table = table; a.table_pos0 = table_pos0; a.eps = c.rms_eps;
+  a.cache_settled = true;   // the QKV GEMV sits between this launch and whatever wrote the cache
   a.k_pool = (const bf16*)kc->k_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.v_pool = (const bf16*)kc->v_pool + (int64_t)(l - 1) * pool_layer_stride;
   a.block_table = kc->block_table; a.max_pages_per_seq = kc->max_pages_per_seq; a.page_size = kc->page_size;

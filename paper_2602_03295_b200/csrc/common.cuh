@@ -235,6 +235,10 @@ struct DecAttnArgs {
   const float* q_gain; const float* k_gain;
   const float2* table; int table_pos0;   // as in RopeArgs
   float eps;
+  // With `qkv`: true when the cache rows of the older positions, the block table and pos_dev / cu_seqlens
+  // were written at least two launches back on the stream (the library's own chain of kernels): the
+  // kernel then starts loading the cache before it waits for its predecessor. False: it waits first.
+  bool cache_settled;
 };
 int decode_attn_splits(int kv_len, int window, int n_kv, int batch);
 int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s);

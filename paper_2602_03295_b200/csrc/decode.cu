@@ -267,6 +267,7 @@ struct DecAttnDev {
   const float* q_gain; const float* k_gain;
   const float2* table; int table_pos0;
   float eps;
+  bool cache_settled;                      // see DecAttnArgs
 };
 
 constexpr int DEC_MAXG = 8;       // query heads per kv head: the N extent of one MMA
@@ -363,11 +364,12 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   extern __shared__ __align__(128) uint8_t dec_smem[];
   chain_trigger();
   // Finished queries and the newest cache row come from the kernel just before this one. When this
-  // kernel finishes the projection itself (p.qkv), only the fp32 projection row does: the cache rows of
-  // the older positions, the block table and the run-time length were written at least two kernels
-  // back, i.e. by kernels that are complete (every kernel of a chain waits for its predecessor), so
-  // the first loads of the cache go out before the wait and overlap the predecessor's tail.
-  const bool early = p.qkv != nullptr;
+  // kernel finishes the projection itself (p.qkv) inside the library's chain of kernels, only the fp32
+  // projection row does: the cache rows of the older positions, the block table and the run-time
+  // length were written at least two kernels back, i.e. by kernels that are complete (every kernel of
+  // a chain waits for its predecessor), so the first loads of the cache go out before the wait and
+  // overlap the predecessor's tail.
+  const bool early = p.qkv != nullptr && p.cache_settled;
   if (!early) chain_wait();
   const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
   const int G = p.n_q / p.n_kv;   // <= DEC_MAXG
@@ -421,7 +423,7 @@ __global__ void __launch_bounds__(DecCfg<HD>::WARPS * 32) dec_attn_kernel(const 
   };
 
   // the newest position's group (the last one of the range that holds it) has to wait for the append
-  const bool holds_new = early && kv_len - 1 >= j0 && kv_len - 1 < j1;
+  const bool holds_new = p.qkv != nullptr && kv_len - 1 >= j0 && kv_len - 1 < j1;
   int deferred = -1;
 #pragma unroll
   for (int i = 0; i < NST; ++i) {
@@ -750,7 +752,7 @@ int launch_decode_attention(const DecAttnArgs& a, cudaStream_t s) {
   if (a.n_q % a.n_kv || a.n_q / a.n_kv > DEC_MAXG || a.kv_len < 1) return POP_E_INVALID;
   DecAttnDev p;
   p.qkv = a.qkv; p.ld_qkv = a.ld_qkv; p.q_gain = a.q_gain; p.k_gain = a.k_gain;
-  p.table = a.table; p.table_pos0 = a.table_pos0; p.eps = a.eps;
+  p.table = a.table; p.table_pos0 = a.table_pos0; p.eps = a.eps; p.cache_settled = a.cache_settled;
   p.q = a.q; p.ldq = a.ldq;
   p.k_pool = a.k_pool; p.v_pool = a.v_pool;
   p.block_table = a.block_table; p.max_pages_per_seq = a.max_pages_per_seq; p.page_size = a.page_size;
@@ -841,7 +843,7 @@ extern "C" int pop_k_decode_attention_static(const void* q, int64_t ldq, const v
   p.block_table = block_table; p.max_pages_per_seq = max_pages_per_seq; p.page_size = page_size;
   p.num_pages = 0;
   p.status = nullptr;
-  p.qkv = nullptr; p.ld_qkv = 0; p.q_gain = p.k_gain = nullptr; p.table = nullptr; p.table_pos0 = 0; p.eps = 0.f;
+  p.qkv = nullptr; p.ld_qkv = 0; p.q_gain = p.k_gain = nullptr; p.table = nullptr; p.table_pos0 = 0; p.eps = 0.f; p.cache_settled = false;
   p.partial = scratch;
   p.out = static_cast<bf16*>(out); p.ldo = ldo;
   p.n_q = n_q; p.n_kv = n_kv; p.kv_len = kv_len; p.window = window;
