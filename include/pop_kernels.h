@@ -132,7 +132,10 @@ int pop_k_gemv(const void* x, int64_t ldx, int32_t x_f32, const void* w, int64_t
  * counters: optional device int32 [batch * n_kv]. If given they must all be zero when the call's
  * kernels start and are all zero again when they end (so one zeroed array serves any number of
  * calls on one stream); the attention kernel then merges its own splits and the call is a single
- * launch. Null: a second kernel merges them. Both ways give the same bits. */
+ * launch. Null: a second kernel merges them. Both ways give the same bits. With few splits per sequence
+ * and kv head (short caches, several sequences) the splits run as one thread-block cluster and merge
+ * through distributed shared memory; partial and counters are then not touched (POP_DEC_CLUSTER=0 in the
+ * environment turns that form off). */
 int pop_k_decode_attention(const void* q, int64_t ldq, const void* k_pool, const void* v_pool,
                            const int32_t* block_table, int32_t max_pages_per_seq, int32_t page_size, float* partial,
                            int32_t* counters, void* out, int64_t ldo, int32_t batch, int32_t n_q, int32_t n_kv,

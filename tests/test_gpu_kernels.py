@@ -352,6 +352,27 @@ def test_decode_attention_with_the_projection_finish(L, B, S, n_q, n_kv, hd, pag
     assert not torch.isnan(out.float()).any()
 
 
+@pytest.mark.parametrize("B,S", [(1, 100), (8, 700), (2, 250)])
+def test_decode_attention_cluster_merge_matches_the_merge_through_memory(L, B, S, monkeypatch):
+    # few splits per (sequence, kv head): the splits form a thread-block cluster and merge through
+    # distributed shared memory; POP_DEC_CLUSTER=0 keeps partials + counters in global memory
+    n_q, n_kv, hd, page = 32, 8, 128, 64
+    q, k, v = _bf((B, n_q * hd), 40, 1.0), _bf((B, S, n_kv, hd), 41, 1.0), _bf((B, S, n_kv, hd), 42, 1.0)
+    kp, vp, bt = paged_pools(k, v, page)
+    outs = []
+    for mode in ("1", "0"):
+        monkeypatch.setenv("POP_DEC_CLUSTER", mode)
+        out = torch.full((B, n_q * hd), float("nan"), dtype=torch.bfloat16, device=DEV)
+        ctr = torch.zeros(B * n_kv, dtype=torch.int32, device=DEV)
+        L.decode_attention(q.to(DEV), kp.to(DEV), vp.to(DEV), bt.to(DEV), out, n_q, n_kv, hd, S, page, 0, counters=ctr)
+        assert (ctr == 0).all()
+        outs.append(out)
+    ref = torch.stack([po.attention(q[b].double().reshape(1, n_q, hd), k[b].double(), v[b].double(),
+                                    torch.tensor([S - 1]), 0).reshape(-1) for b in range(B)])
+    assert rel_err(outs[0], ref) < 1e-2 and rel_err(outs[1], ref) < 1e-2
+    assert rel_err(outs[0], outs[1].cpu().double()) < 1e-2
+
+
 def test_generators_agree_between_cpu_and_gpu():
     tid = ps.tensor_id("wq", 2)
     a = ps.normal_bf16(3, tid, (300, 1000), 0.02)
