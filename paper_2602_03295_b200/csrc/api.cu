@@ -34,7 +34,7 @@ struct Workspace {
   float* hb32;       // [B][d]
   bf16* hb;          // [B][d]
   float* qkvb;       // [B][qkv_dim]
-  bf16* qb;          // [B][q_dim]
+  bf16* qb;          // unused (kept for layout stability): the decode attention finishes the queries itself
   bf16* ob;          // [B][q_dim]
   bf16* ab;          // [B][F]
   float* partial;    // [B][n_q][64][hd+2]
