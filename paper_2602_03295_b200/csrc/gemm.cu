@@ -223,7 +223,8 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
 // Epilogue of one 128-row x 256-column accumulator slab held in this CTA's TMEM: the calling warp
 // (TMEM lane quarter `quarter`) owns rows row0 + quarter*32 .. +31, one row per lane. `n` is the
 // 256-column tile index, `boxes` the warp's two 32 x 32 fp32 staging boxes for TMA stores.
-template <int EPI, int HD, bool FP8>
+// TN: output columns of a tile (256; 128 for the narrow single-CTA form, see launch_gemm)
+template <int EPI, int HD, bool FP8, int TN = BN>
 __device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMap& tmO, uint8_t* boxes,
                                               uint32_t taddr, int g, int row0, int n, int quarter, int lane,
                                               uint32_t& boxes_out) {
@@ -272,8 +273,8 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMa
     // is read by the SM, rows and columns beyond the output are clipped by the hardware.
     const bool rows_in = row0 + quarter * 32 < p.M;     // uniform per warp
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
-      if (n * BN + c * 32 >= p.N) break;                 // uniform: the rest of the tile is past the last column
+    for (int c = 0; c < TN / 32; ++c) {
+      if (n * TN + c * 32 >= p.N) break;                 // uniform: the rest of the tile is past the last column
       uint32_t r[32];
       tmem_ld_32x32b_x32(taddr + c * 32, r);
       tmem_wait_ld();
@@ -295,19 +296,19 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMa
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        if (EPI == EPI_ADD_F32) tma_reduce_add_3d(&tmO, box, n * BN + c * 32, row0 + quarter * 32, g);
-        else tma_store_3d(&tmO, box, n * BN + c * 32, row0 + quarter * 32, g);
+        if (EPI == EPI_ADD_F32) tma_reduce_add_3d(&tmO, box, n * TN + c * 32, row0 + quarter * 32, g);
+        else tma_store_3d(&tmO, box, n * TN + c * 32, row0 + quarter * 32, g);
         bulk_commit();
       }
     }
   } else {
     float ss = 0.f;                       // EPI_ADD_F32 with hn_out: sum of squares of this row's new values
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
+    for (int c = 0; c < TN / 32; ++c) {
       uint32_t r[32];
       tmem_ld_32x32b_x32(taddr + c * 32, r);
       tmem_wait_ld();
-      const int col0 = n * BN + c * 32;
+      const int col0 = n * TN + c * 32;
       if (row_ok) {
         if (EPI != EPI_ADD_F32) {
 #pragma unroll
@@ -357,7 +358,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMa
 
 // FP8: the operands are E4M3 codes, a k-block of 128 bytes holds 128 of them (64 bf16 otherwise) and
 // one MMA instruction covers 32 (16): the smem tiles, descriptors and their 32-byte steps are the same.
-template <int EPI, int HD, bool FP8>
+template <int EPI, int HD, bool FP8, int TN = BN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmO, const GemmDev p,
@@ -408,9 +409,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             atomicMin(status, (int)POP_E_DEVICE_TIMEOUT);
             break;
           }
-          mbar_expect_tx(&s.full[stage], A_BYTES + B_BYTES);
+          mbar_expect_tx(&s.full[stage], A_BYTES + TN * BK * 2);
           tma_load_3d(s.a[stage], &tmA, &s.full[stage], kb * BKE, m * BM, g);
-          tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BKE, n * BN, g);
+          tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BKE, n * TN, g);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1;
@@ -423,7 +424,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // The whole warp walks this role with identical values; one elected lane issues.
     {
       const uint32_t leader = elect_one();
-      constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(BM, BN) : umma_idesc_bf16(BM, BN, 0, 0);
+      constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(BM, TN) : umma_idesc_bf16(BM, TN, 0, 0);
       const uint64_t a_desc0 = umma_smem_desc(smem_u32(s.a[0]), 16, 1024);
       const uint64_t b_desc0 = umma_smem_desc(smem_u32(s.b[0]), 16, 1024);
       int stage = 0;
@@ -438,7 +439,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * BN;
+        const uint32_t d_tmem = tmem_base + buf * TN;
         bool ok = true;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&s.full[stage], phase)) {
@@ -488,8 +489,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         break;
       }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
-      epilogue_tile<EPI, HD, FP8>(p, tmO, s.out_stage[quarter][0], taddr, g, m * BM, n, quarter, lane, boxes_out);
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * TN;
+      epilogue_tile<EPI, HD, FP8, TN>(p, tmO, s.out_stage[quarter][0], taddr, g, m * BM, n, quarter, lane, boxes_out);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s.tempty[buf]);
@@ -739,7 +740,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
 template <int EPI, int HD = 0, bool FP8 = false>
 int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmDev& p_in, int grid,
-               bool pair, cudaStream_t stream) {
+               bool pair, bool narrow, cudaStream_t stream) {
   int* status = status_word();
   if (!status) return POP_E_CUDA;
   GemmDev p = p_in;
@@ -771,6 +772,22 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? POP_OK : POP_E_CUDA;
   }
   const size_t smem = sizeof(GemmSmem) + 1024;
+  if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_ADD_F32) {
+    if (narrow) {
+      static bool configured_narrow = false;
+      if (!configured_narrow) {
+        if (cudaFuncSetAttribute(gemm_kernel<EPI, HD, FP8, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+          return POP_E_CUDA;
+        configured_narrow = true;
+      }
+      ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
+      gemm_kernel<EPI, HD, FP8, 128><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
+      count_launch();
+      return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
+    }
+  }
+  if (narrow) return POP_E_INVALID;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(gemm_kernel<EPI, HD, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -792,6 +809,17 @@ int pair_group_m(int K) {
   if (e && atoi(e) > 0) return atoi(e);
   (void)K;
   return 16;
+}
+
+// Narrow single-CTA form: 128 x 128 tiles for the plain-store and residual epilogues when 128 x 256
+// tiles would leave at least half of the SMs without a tile (short prompts: the O and down projections of
+// 512 rows are 64 tiles). POP_GEMM_NARROW=0 / 1 forces it off / on wherever it is possible.
+bool use_narrow(bool possible, int64_t tiles, int sms) {
+  if (!possible) return false;
+  const char* e = std::getenv("POP_GEMM_NARROW");
+  if (e && e[0] == '0') return false;
+  if (e && e[0] == '1') return true;
+  return tiles * 2 <= sms;      // twice as many narrow tiles are still one wave (B 8 x 32 tokens: -4.6 % per prefill)
 }
 
 bool use_pair(int M, int64_t tiles2, int sms) {
@@ -829,7 +857,11 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     return POP_E_CUDA;
   const int64_t tiles2 = int64_t(ceil_div(a.M, 2 * BM)) * ceil_div(a.N, BN) * a.batch;
   const bool pair = use_pair(a.M, tiles2, sms);
-  const uint32_t b_box = pair ? 128 : BN;      // a CTA of a pair loads its own half of the B block
+  const bool narrow = use_narrow(!pair && a.N > 128 && !a.hn_out && !a.ss_out &&
+                                     (a.epilogue == EPI_STORE_BF16 || a.epilogue == EPI_STORE_F32 ||
+                                      a.epilogue == EPI_ADD_F32),
+                                 int64_t(ceil_div(a.M, BM)) * ceil_div(a.N, BN) * a.batch, sms);
+  const uint32_t b_box = (pair || narrow) ? 128 : BN;   // a CTA of a pair loads its own half of the B block
   CUtensorMap ta, tb;
   int rc;
   if (a.fp8) {
@@ -886,7 +918,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   p.out_batch_stride = a.out_batch_stride;
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = a.batch;
   p.m_tiles = ceil_div(a.M, BM);
-  p.n_tiles = ceil_div(a.N, BN);
+  p.n_tiles = ceil_div(a.N, narrow ? 128 : BN);
   p.act = a.act;
   p.n_valid = a.n_valid;
   const int64_t total = int64_t(p.m_tiles) * p.n_tiles * p.batch;
@@ -895,30 +927,30 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   p.group_m = pair_group_m(a.K);
   if (a.fp8) {
     switch (a.epilogue) {
-      case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, pair, stream);
-      case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, pair, stream);
-      case EPI_ADD_F32: return launch_epi<EPI_ADD_F32, 0, true>(ta, tb, to, p, grid, pair, stream);
-      case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, pair, stream);
+      case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16, 0, true>(ta, tb, to, p, grid, pair, narrow, stream);
+      case EPI_STORE_F32: return launch_epi<EPI_STORE_F32, 0, true>(ta, tb, to, p, grid, pair, narrow, stream);
+      case EPI_ADD_F32: return launch_epi<EPI_ADD_F32, 0, true>(ta, tb, to, p, grid, pair, narrow, stream);
+      case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16, 0, true>(ta, tb, to, p, grid, pair, narrow, stream);
       case EPI_QKV_ROPE:
         switch (a.rope->hd) {
-          case 64: return launch_epi<EPI_QKV_ROPE, 64, true>(ta, tb, to, p, grid, pair, stream);
-          case 128: return launch_epi<EPI_QKV_ROPE, 128, true>(ta, tb, to, p, grid, pair, stream);
-          case 256: return launch_epi<EPI_QKV_ROPE, 256, true>(ta, tb, to, p, grid, pair, stream);
+          case 64: return launch_epi<EPI_QKV_ROPE, 64, true>(ta, tb, to, p, grid, pair, narrow, stream);
+          case 128: return launch_epi<EPI_QKV_ROPE, 128, true>(ta, tb, to, p, grid, pair, narrow, stream);
+          case 256: return launch_epi<EPI_QKV_ROPE, 256, true>(ta, tb, to, p, grid, pair, narrow, stream);
         }
         return POP_E_INVALID;
     }
     return POP_E_INVALID;
   }
   switch (a.epilogue) {
-    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, pair, stream);
-    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, pair, stream);
-    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, to, p, grid, pair, stream);
-    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, to, p, grid, pair, stream);
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(ta, tb, to, p, grid, pair, narrow, stream);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(ta, tb, to, p, grid, pair, narrow, stream);
+    case EPI_ADD_F32: return launch_epi<EPI_ADD_F32>(ta, tb, to, p, grid, pair, narrow, stream);
+    case EPI_GATED_BF16: return launch_epi<EPI_GATED_BF16>(ta, tb, to, p, grid, pair, narrow, stream);
     case EPI_QKV_ROPE:
       switch (a.rope->hd) {
-        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, to, p, grid, pair, stream);
-        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, to, p, grid, pair, stream);
-        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, to, p, grid, pair, stream);
+        case 64: return launch_epi<EPI_QKV_ROPE, 64>(ta, tb, to, p, grid, pair, narrow, stream);
+        case 128: return launch_epi<EPI_QKV_ROPE, 128>(ta, tb, to, p, grid, pair, narrow, stream);
+        case 256: return launch_epi<EPI_QKV_ROPE, 256>(ta, tb, to, p, grid, pair, narrow, stream);
       }
       return POP_E_INVALID;
   }

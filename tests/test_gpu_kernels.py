@@ -23,11 +23,13 @@ def L():
     return pk.lib()
 
 
-@pytest.fixture(params=["single", "pair"])
+@pytest.fixture(params=["single", "pair", "narrow"])
 def gemm_form(request, monkeypatch):
-    """Runs a GEMM test twice: with one CTA per 128 x 256 tile and with a CTA pair per 256 x 256 tile
-    (POP_GEMM_PAIR forces either form whatever the problem size)."""
+    """Runs a GEMM test three times: with one CTA per 128 x 256 tile, with a CTA pair per 256 x 256 tile,
+    and with one CTA per 128 x 128 tile (the plain-store and residual epilogues only; the other epilogues
+    then run the 128 x 256 form). POP_GEMM_PAIR / POP_GEMM_NARROW force a form whatever the problem size."""
     monkeypatch.setenv("POP_GEMM_PAIR", "1" if request.param == "pair" else "0")
+    monkeypatch.setenv("POP_GEMM_NARROW", "1" if request.param == "narrow" else "0")
     return request.param
 
 

@@ -32,9 +32,10 @@ def L():
     return pk.lib()
 
 
-@pytest.fixture(params=["single", "pair"])
+@pytest.fixture(params=["single", "pair", "narrow"])
 def gemm_form(request, monkeypatch):
     monkeypatch.setenv("POP_GEMM_PAIR", "1" if request.param == "pair" else "0")
+    monkeypatch.setenv("POP_GEMM_NARROW", "1" if request.param == "narrow" else "0")
     return request.param
 
 
