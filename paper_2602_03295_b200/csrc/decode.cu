@@ -215,6 +215,16 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
   }
 }
 
+// The tensor-core GEMV costs the same for 1 to 8 activation rows; the scalar one is faster for one or
+// two rows and several times slower for eight (c2 shapes, 8 rows, us per launch alone and cold, scalar /
+// tensor-core: QKV 34.7 / 19.7, O 36.6 / 12.8, gate-up 126 / 61, down 106 / 34). POP_GEMV_MMA=0 keeps the
+// scalar kernel everywhere.
+constexpr int GEMV_MMA_MIN_ROWS = 3;
+bool gemv_mma_enabled() {
+  const char* e = getenv("POP_GEMV_MMA");
+  return !(e && e[0] == '0');
+}
+
 template <bool X_F32, bool GATED, int KS, bool W8>
 void launch_gemv_nb(const GemvDev& p, int blocks, int threads, cudaStream_t s) {
   if (p.B <= 1) launch_chained(gemv_kernel<X_F32, 1, GATED, KS, W8>, dim3(blocks), dim3(threads), 0, s, p);
@@ -234,6 +244,161 @@ void launch_gemv_ks(const GemvDev& p, int row_warps, int ks, cudaStream_t s) {
     case 4: launch_gemv_nb<X_F32, GATED, 4, W8>(p, blocks, 256, s); break;
     case 2: launch_gemv_nb<X_F32, GATED, 2, W8>(p, blocks, 256, s); break;
     default: launch_gemv_nb<X_F32, GATED, 1, W8>(p, blocks, wpc * 32, s); break;
+  }
+}
+
+// ------------------------------------------------------------------------------ tensor-core GEMV
+// bf16 activations x bf16 weights on the warp-level MMA (m16n8k16): the weight rows are the M side, the
+// (up to 8) activation rows the N side. A lane (g = lane / 4, t = lane % 4) loads 16 bytes = 8 consecutive
+// k of weight rows g and g + 8 and of activation row g at the same k offset 32 s + 8 t; the four
+// register pairs of each load feed two MMAs as (a0, a2) / (a1, a3) / (b0, b1). The k index inside an
+// MMA is then a permutation of the real one, the same for A and B, which a dot product does not see.
+// One instruction does the work of 256 conversions and FMAs of the scalar kernel, and the sums come
+// out complete in the accumulator: no shuffles. Gated form: rows g are gate rows, rows g + 8 their
+// up rows, so one thread ends up with both sums of an output.
+// KS warps of a CTA share a row group and take k-steps s = slice, slice + KS, ...
+constexpr int MMA_U = 4;     // k-steps per batch of loads (two batches in flight)
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// X32: the activations are fp32 (the output head's input). Each value goes in as two bf16, its rounding and
+// the rounding of what the first one missed, through two MMAs on the same weights: the product keeps
+// about 16 bits of the activation instead of 8.
+template <bool GATED, int KS, bool X32>
+__global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvDev p) {
+  const int lane = threadIdx.x & 31, wic = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int slice = wic % KS;
+  const int group = blockIdx.x * (8 / KS) + wic / KS;
+  const int n_out = GATED ? p.N / 2 : p.N;
+  chain_trigger();
+  // rows of this lane; past the end they repeat the last row (loaded, never stored)
+  int64_t r_lo, r_hi;
+  if (GATED) {
+    const int o = min(group * 8 + g, n_out - 1);
+    r_lo = (int64_t)(o >> 7) * 256 + (o & 127);
+    r_hi = r_lo + 128;
+  } else {
+    r_lo = min(group * 16 + g, n_out - 1);
+    r_hi = min(group * 16 + g + 8, n_out - 1);
+  }
+  const bf16* wlo = static_cast<const bf16*>(p.w) + r_lo * p.ldw + t * 8;
+  const bf16* whi = static_cast<const bf16*>(p.w) + r_hi * p.ldw + t * 8;
+  const bf16* xr = static_cast<const bf16*>(p.x) + (int64_t)g * p.ldx + t * 8;
+  const float* xr32 = static_cast<const float*>(p.x) + (int64_t)g * p.ldx + t * 8;
+  const bool has_x = g < p.B;
+  const int n_steps = p.K / 32;
+  float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+  uint4 wa[2][MMA_U], wb[2][MMA_U];
+  auto load_batch = [&](int buf, int s0) {
+#pragma unroll
+    for (int u = 0; u < MMA_U; ++u) {
+      const int s = s0 + u * KS;
+      if (s < n_steps) {
+        wa[buf][u] = ld_stream(wlo + s * 32);
+        wb[buf][u] = ld_stream(whi + s * 32);
+      }
+    }
+  };
+  // the first two batches of weight loads go out before the wait on the preceding kernel
+  load_batch(0, slice);
+  load_batch(1, slice + MMA_U * KS);
+  chain_wait();
+  int buf = 0;
+  for (int s0 = slice; s0 < n_steps; s0 += MMA_U * KS) {
+#pragma unroll
+    for (int u = 0; u < MMA_U; ++u) {
+      const int s = s0 + u * KS;
+      if (s < n_steps) {
+        const uint4 a = buf ? wa[1][u] : wa[0][u], b = buf ? wb[1][u] : wb[0][u];
+        if (X32) {
+          float xf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          if (has_x) {
+            const float4 x0 = *reinterpret_cast<const float4*>(xr32 + s * 32);
+            const float4 x1 = *reinterpret_cast<const float4*>(xr32 + s * 32 + 4);
+            xf[0] = x0.x; xf[1] = x0.y; xf[2] = x0.z; xf[3] = x0.w;
+            xf[4] = x1.x; xf[5] = x1.y; xf[6] = x1.z; xf[7] = x1.w;
+          }
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(xf[2 * i], xf[2 * i + 1]);
+            const float2 hf = __bfloat1622float2(h);
+            const __nv_bfloat162 l = __floats2bfloat162_rn(xf[2 * i] - hf.x, xf[2 * i + 1] - hf.y);
+            hi[i] = *reinterpret_cast<const uint32_t*>(&h);
+            lo[i] = *reinterpret_cast<const uint32_t*>(&l);
+          }
+          mma_bf16_16816(d0, a.x, b.x, a.y, b.y, hi[0], hi[1]);
+          mma_bf16_16816(d1, a.z, b.z, a.w, b.w, hi[2], hi[3]);
+          mma_bf16_16816(d0, a.x, b.x, a.y, b.y, lo[0], lo[1]);
+          mma_bf16_16816(d1, a.z, b.z, a.w, b.w, lo[2], lo[3]);
+        } else {
+          const uint4 xv = has_x ? *reinterpret_cast<const uint4*>(xr + s * 32) : make_uint4(0, 0, 0, 0);
+          mma_bf16_16816(d0, a.x, b.x, a.y, b.y, xv.x, xv.y);
+          mma_bf16_16816(d1, a.z, b.z, a.w, b.w, xv.z, xv.w);
+        }
+      }
+    }
+    if (buf) load_batch(1, s0 + 2 * MMA_U * KS); else load_batch(0, s0 + 2 * MMA_U * KS);
+    buf ^= 1;
+  }
+  float c[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) c[i] = d0[i] + d1[i];
+  if (KS > 1) {
+    // slice 0 of every group adds the other slices' sums in slice order
+    __shared__ float part[8][32][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) part[wic][lane][i] = c[i];
+    __syncthreads();
+    if (slice != 0) return;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float v = 0.f;
+#pragma unroll
+      for (int sl = 0; sl < KS; ++sl) v += part[wic + sl][lane][i];
+      c[i] = v;
+    }
+  }
+  // c[0], c[1]: row g (gated: gate sum) for sequences 2t, 2t + 1; c[2], c[3]: row g + 8 (gated: up sum)
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int b = 2 * t + j;
+    if (b >= p.B) continue;
+    if (GATED) {
+      const int o = group * 8 + g;
+      if (o < n_out && o < p.n_valid)
+        reinterpret_cast<bf16*>(p.out)[(int64_t)b * p.ldo + o] = __float2bfloat16_rn(act_fn(c[j], p.act) * c[2 + j]);
+    } else {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int o = group * 16 + g + 8 * h;
+        if (o >= n_out) continue;
+        float* dst = reinterpret_cast<float*>(p.out) + (int64_t)b * p.ldo + o;
+        if (p.mode == 0) *dst = c[2 * h + j];
+        else *dst += c[2 * h + j];
+      }
+    }
+  }
+}
+
+template <bool GATED, bool X32>
+void launch_gemv_mma(const GemvDev& p, int ks, cudaStream_t s) {
+  const int n_out = GATED ? p.N / 2 : p.N;
+  const int groups = ceil_div(n_out, GATED ? 8 : 16);
+  const int blocks = ceil_div(groups * ks, 8);
+  switch (ks) {
+    case 8: launch_chained(gemv_mma_kernel<GATED, 8, X32>, dim3(blocks), dim3(256), 0, s, p); break;
+    case 4: launch_chained(gemv_mma_kernel<GATED, 4, X32>, dim3(blocks), dim3(256), 0, s, p); break;
+    case 2: launch_chained(gemv_mma_kernel<GATED, 2, X32>, dim3(blocks), dim3(256), 0, s, p); break;
+    default: launch_chained(gemv_mma_kernel<GATED, 1, X32>, dim3(blocks), dim3(256), 0, s, p); break;
   }
 }
 
@@ -778,6 +943,20 @@ int launch_gemv(const GemvArgs& a, cudaStream_t s) {
     p.B = a.B - b0 < GEMV_MAXB ? a.B - b0 : GEMV_MAXB;
     p.N = a.N; p.K = a.K; p.mode = a.mode; p.act = a.act; p.n_valid = a.n_valid;
     ProfScope prof(PROF_GEMV, (double)a.N * a.K * (a.w_fp8 ? 1 : 2), s);
+    if (!a.w_fp8 && a.K % 32 == 0 && p.B >= GEMV_MMA_MIN_ROWS && gemv_mma_enabled()) {
+      // K split over the 8 warps of a CTA while every warp keeps at least two batches of k-steps
+      int mks = 1;
+      while (mks < 8 && a.K / 32 >= 2 * MMA_U * mks * 2) mks *= 2;
+      if (a.mode == 3) {
+        if (a.x_f32) launch_gemv_mma<true, true>(p, mks, s);
+        else launch_gemv_mma<true, false>(p, mks, s);
+      } else {
+        if (a.x_f32) launch_gemv_mma<false, true>(p, mks, s);
+        else launch_gemv_mma<false, false>(p, mks, s);
+      }
+      count_launch();
+      continue;
+    }
     if (a.mode == 3) {
       if (a.w_fp8) launch_gemv_ks<false, true, true>(p, warps, ks, s);
       else if (a.x_f32) launch_gemv_ks<true, true>(p, warps, ks, s);

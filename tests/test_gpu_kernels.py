@@ -260,9 +260,18 @@ def test_fused_qkv_projection_rope_and_cache_write(L, gemm_form, hd, n_q, n_kv, 
     assert (kpool[0] == canary).all() and (kpool[1 + groups:] == canary).all()
 
 
+@pytest.fixture(params=["auto", "scalar"])
+def gemv_form(request, monkeypatch):
+    """GEMV tests run twice: with the library's choice (the tensor-core kernel from three activation rows
+    on, bf16 activations, K a multiple of 32) and with the scalar kernel everywhere (POP_GEMV_MMA=0)."""
+    monkeypatch.setenv("POP_GEMV_MMA", "0" if request.param == "scalar" else "1")
+    return request.param
+
+
 @pytest.mark.parametrize("B,N,K,xf32", [(1, 1024, 4096, False), (8, 520, 688, False), (3, 1000, 256, True),
-                                        (11, 64, 64, False)])
-def test_gemv_store_and_add(L, B, N, K, xf32):
+                                        (11, 64, 64, False), (8, 4096, 4096, False), (5, 1000, 512, False),
+                                        (3, 24, 96, False), (4, 4096, 14336, False), (8, 4096, 4096, True)])
+def test_gemv_store_and_add(L, gemv_form, B, N, K, xf32):
     W = _bf((N, K), 15)
     x = _bf((B, K), 16)
     xin = x.float() if xf32 else x
@@ -274,8 +283,8 @@ def test_gemv_store_and_add(L, B, N, K, xf32):
     assert rel_err(out, 2 * ref) < 1e-4
 
 
-def test_gemv_gated(L):
-    B, F, K = 4, 688, 256
+@pytest.mark.parametrize("B,F,K", [(4, 688, 256), (8, 14336, 4096), (3, 100, 64), (1, 688, 256)])
+def test_gemv_gated(L, gemv_form, B, F, K):
     Wg, Wu, x = _bf((F, K), 17), _bf((F, K), 18), _bf((B, K), 19)
     f_pad = (F + 127) // 128 * 128
     Wgu = torch.zeros(2 * f_pad, K, dtype=torch.bfloat16)
