@@ -273,49 +273,72 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 // about 16 bits of the activation instead of 8.
 template <bool GATED, int KS, bool X32>
 __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvDev p) {
+  constexpr int GPC = 8 / KS;                       // row groups a CTA works on at a time
   const int lane = threadIdx.x & 31, wic = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int slice = wic % KS;
-  const int group = blockIdx.x * (8 / KS) + wic / KS;
   const int n_out = GATED ? p.N / 2 : p.N;
+  const int n_groups = (n_out + (GATED ? 8 : 16) - 1) / (GATED ? 8 : 16);
+  const int n_rounds = (n_groups + GPC - 1) / GPC;  // rounds of GPC groups; this CTA takes blockIdx.x, + gridDim.x, ..
+  const int my_rounds = n_rounds > (int)blockIdx.x ? (n_rounds - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int n_steps = p.K / 32;
+  // batches of MMA_U k-steps per round, the same for every slice (steps past the end are skipped), so
+  // that the warps of a CTA finish a round together; batches are numbered through all the rounds and
+  // two of them are always in flight, also across the end of a round
+  const int nb_round = ((n_steps + KS - 1) / KS + MMA_U - 1) / MMA_U;
+  const int n_batches = my_rounds * nb_round;
   chain_trigger();
-  // rows of this lane; past the end they repeat the last row (loaded, never stored)
-  int64_t r_lo, r_hi;
-  if (GATED) {
-    const int o = min(group * 8 + g, n_out - 1);
-    r_lo = (int64_t)(o >> 7) * 256 + (o & 127);
-    r_hi = r_lo + 128;
-  } else {
-    r_lo = min(group * 16 + g, n_out - 1);
-    r_hi = min(group * 16 + g + 8, n_out - 1);
-  }
-  const bf16* wlo = static_cast<const bf16*>(p.w) + r_lo * p.ldw + t * 8;
-  const bf16* whi = static_cast<const bf16*>(p.w) + r_hi * p.ldw + t * 8;
   const bf16* xr = static_cast<const bf16*>(p.x) + (int64_t)g * p.ldx + t * 8;
   const float* xr32 = static_cast<const float*>(p.x) + (int64_t)g * p.ldx + t * 8;
   const bool has_x = g < p.B;
-  const int n_steps = p.K / 32;
+  auto group_of = [&](int round_i) { return ((int)blockIdx.x + round_i * (int)gridDim.x) * GPC + wic / KS; };
   float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
   uint4 wa[2][MMA_U], wb[2][MMA_U];
-  auto load_batch = [&](int buf, int s0) {
+  // load side: walks the same (round, batch) sequence two batches ahead of the compute side
+  const bf16* wlo = nullptr;
+  const bf16* whi = nullptr;
+  int l_ri = 0, l_lb = 0;
+  auto set_rows = [&](int round_i) {
+    const int group = group_of(round_i);
+    // rows of this lane; past the end they repeat the last row (loaded, never stored)
+    int64_t r_lo, r_hi;
+    if (GATED) {
+      const int o = min(group * 8 + g, n_out - 1);
+      r_lo = (int64_t)(o >> 7) * 256 + (o & 127);
+      r_hi = r_lo + 128;
+    } else {
+      r_lo = min(group * 16 + g, n_out - 1);
+      r_hi = min(group * 16 + g + 8, n_out - 1);
+    }
+    wlo = static_cast<const bf16*>(p.w) + r_lo * p.ldw + t * 8;
+    whi = static_cast<const bf16*>(p.w) + r_hi * p.ldw + t * 8;
+  };
+  if (my_rounds > 0) set_rows(0);
+  auto load_next = [&](int buf) {
+    if (l_ri >= my_rounds) return;
 #pragma unroll
     for (int u = 0; u < MMA_U; ++u) {
-      const int s = s0 + u * KS;
+      const int s = slice + KS * (l_lb * MMA_U + u);
       if (s < n_steps) {
         wa[buf][u] = ld_stream(wlo + s * 32);
         wb[buf][u] = ld_stream(whi + s * 32);
       }
     }
+    if (++l_lb == nb_round) {
+      l_lb = 0;
+      if (++l_ri < my_rounds) set_rows(l_ri);
+    }
   };
   // the first two batches of weight loads go out before the wait on the preceding kernel
-  load_batch(0, slice);
-  load_batch(1, slice + MMA_U * KS);
+  load_next(0);
+  load_next(1);
   chain_wait();
-  int buf = 0;
-  for (int s0 = slice; s0 < n_steps; s0 += MMA_U * KS) {
+  __shared__ float part[8][32][4];
+  int buf = 0, lb = 0, ri = 0;
+  for (int fb = 0; fb < n_batches; ++fb) {
 #pragma unroll
     for (int u = 0; u < MMA_U; ++u) {
-      const int s = s0 + u * KS;
+      const int s = slice + KS * (lb * MMA_U + u);
       if (s < n_steps) {
         const uint4 a = buf ? wa[1][u] : wa[0][u], b = buf ? wb[1][u] : wb[0][u];
         if (X32) {
@@ -346,46 +369,59 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvDev p) {
         }
       }
     }
-    if (buf) load_batch(1, s0 + 2 * MMA_U * KS); else load_batch(0, s0 + 2 * MMA_U * KS);
+    if (buf) load_next(1); else load_next(0);
     buf ^= 1;
-  }
-  float c[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) c[i] = d0[i] + d1[i];
-  if (KS > 1) {
-    // slice 0 of every group adds the other slices' sums in slice order
-    __shared__ float part[8][32][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) part[wic][lane][i] = c[i];
-    __syncthreads();
-    if (slice != 0) return;
+    if (++lb < nb_round) continue;
+    // ---- end of a round: the sums of this warp's rows are complete (up to the K split)
+    float c[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      float v = 0.f;
-#pragma unroll
-      for (int sl = 0; sl < KS; ++sl) v += part[wic + sl][lane][i];
-      c[i] = v;
+      c[i] = d0[i] + d1[i];
+      d0[i] = d1[i] = 0.f;
     }
-  }
-  // c[0], c[1]: row g (gated: gate sum) for sequences 2t, 2t + 1; c[2], c[3]: row g + 8 (gated: up sum)
+    const int group = group_of(ri);
+    bool store = true;
+    if (KS > 1) {
+      // slice 0 of every group adds the other slices' sums in slice order
+      __syncthreads();                               // the previous round's sums have been read
 #pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    const int b = 2 * t + j;
-    if (b >= p.B) continue;
-    if (GATED) {
-      const int o = group * 8 + g;
-      if (o < n_out && o < p.n_valid)
-        reinterpret_cast<bf16*>(p.out)[(int64_t)b * p.ldo + o] = __float2bfloat16_rn(act_fn(c[j], p.act) * c[2 + j]);
-    } else {
+      for (int i = 0; i < 4; ++i) part[wic][lane][i] = c[i];
+      __syncthreads();
+      store = slice == 0;
+      if (store) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int o = group * 16 + g + 8 * h;
-        if (o >= n_out) continue;
-        float* dst = reinterpret_cast<float*>(p.out) + (int64_t)b * p.ldo + o;
-        if (p.mode == 0) *dst = c[2 * h + j];
-        else *dst += c[2 * h + j];
+        for (int i = 0; i < 4; ++i) {
+          float v = 0.f;
+#pragma unroll
+          for (int sl = 0; sl < KS; ++sl) v += part[wic + sl][lane][i];
+          c[i] = v;
+        }
       }
     }
+    if (store) {
+      // c[0], c[1]: row g (gated: gate sum) for sequences 2t, 2t + 1; c[2], c[3]: row g + 8 (gated: up sum)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int b = 2 * t + j;
+        if (b >= p.B) continue;
+        if (GATED) {
+          const int o = group * 8 + g;
+          if (o < n_out && o < p.n_valid)
+            reinterpret_cast<bf16*>(p.out)[(int64_t)b * p.ldo + o] = __float2bfloat16_rn(act_fn(c[j], p.act) * c[2 + j]);
+        } else {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int o = group * 16 + g + 8 * h;
+            if (o >= n_out) continue;
+            float* dst = reinterpret_cast<float*>(p.out) + (int64_t)b * p.ldo + o;
+            if (p.mode == 0) *dst = c[2 * h + j];
+            else *dst += c[2 * h + j];
+          }
+        }
+      }
+    }
+    lb = 0;
+    ++ri;
   }
 }
 
@@ -393,7 +429,17 @@ template <bool GATED, bool X32>
 void launch_gemv_mma(const GemvDev& p, int ks, cudaStream_t s) {
   const int n_out = GATED ? p.N / 2 : p.N;
   const int groups = ceil_div(n_out, GATED ? 8 : 16);
-  const int blocks = ceil_div(groups * ks, 8);
+  const int rounds = ceil_div(groups * ks, 8);
+  // two CTAs fit an SM (registers); each walks its rounds with the load pipeline kept full between them
+  static int slots = 0;
+  if (slots == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+    slots = 2 * n;
+  }
+  const int blocks = rounds < slots ? rounds : slots;
   switch (ks) {
     case 8: launch_chained(gemv_mma_kernel<GATED, 8, X32>, dim3(blocks), dim3(256), 0, s, p); break;
     case 4: launch_chained(gemv_mma_kernel<GATED, 4, X32>, dim3(blocks), dim3(256), 0, s, p); break;
