@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvDev p) {
 
 // The tensor-core GEMV costs the same for 1 to 8 activation rows; the scalar one is faster for one or
 // two rows and several times slower for eight (c2 shapes, 8 rows, us per launch alone and cold, scalar /
-// tensor-core: QKV 34.7 / 19.7, O 36.6 / 12.8, gate-up 126 / 61, down 106 / 34). POP_GEMV_MMA=0 keeps the
+// tensor-core: QKV 34.7 / 17.6, O 36.6 / 14.3, gate-up 126 / 48, down 106 / 32). POP_GEMV_MMA=0 keeps the
 // scalar kernel everywhere.
 constexpr int GEMV_MMA_MIN_ROWS = 3;
 bool gemv_mma_enabled() {
