@@ -34,6 +34,7 @@ import pop_synth as ps  # noqa: E402
 METRIC = "pop_prefill_tokens_per_s"
 UNIT = "tokens/s"
 KERNELS = ["gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down", "kvproj", "attention", "attention_local", "gemv_head",
+           "gemv_gateup",
            "decode_attention", "decode_step", "rmsnorm", "rope_cache", "gemm_gateup_fp8", "gemm_qkvshape_fp8",
            "rmsnorm_fp8"]
 
@@ -539,6 +540,18 @@ def run_kernel(a, wl):
 
         def launch(i):
             lib.gemv(x, W, out, mode=0)
+    elif k == "gemv_gateup":
+        # the boundary / decode path's widest matrix for wl.batch activation rows (--batch N): the scalar GEMV for
+        # one or two rows, the tensor-core GEMV from three on; four weight sets so that L2 never helps
+        bound = "hbm"
+        F = (cfg.d_ffn + 127) // 128 * 128
+        Ws = [rnd(2 * F, d, std=0.02) for _ in range(4)]
+        x = rnd(wl.batch, d, std=1.0)
+        out = torch.zeros(wl.batch, cfg.d_ffn, dtype=torch.bfloat16, device=dev)
+        work = 2.0 * 2 * F * d
+
+        def launch(i):
+            lib.gemv(x, Ws[i % 4], out, mode=3, act=cfg.act, n_valid=cfg.d_ffn)
     elif k == "decode_attention":
         from paper_2602_03295_b200.binding import KVCache
         bound = "hbm"
