@@ -285,6 +285,26 @@ def test_true_width_reduced_depth():
         assert rel_err(k, ref["K"][l]) <= KV_TOL and rel_err(v, ref["V"][l]) <= KV_TOL
 
 
+def test_true_width_batch_of_short_prompts():
+    # 8 prompts of 32 tokens at the Llama-3.1-8B layer shapes (2 layers, vocabulary 8192), the shape class of the
+    # paper's Table 2: 256 rows per GEMM, where the O and down projections run as 128 x 128 tiles, and the boundary
+    # pass of 8 rows runs the tensor-core GEMV. Against the oracle, and twice for equal bits.
+    cfg = ps.C2_LLAMA8B.replace(n_layers=2, vocab=8192, name="llama8b-width-2-layers")
+    tokens = ps.uniform_tokens(21, 8, 32, cfg.vocab)
+    w = CachedWeights(DeviceDrawnWeights(cfg))
+    ref = po.pop_prefill(cfg, w, tokens, None, 1, dtype=torch.float64)
+    model = build(cfg)
+    logits, cache = run_gpu(model, cfg, tokens, None, 1, page=16)
+    d = logits.cpu().double() - ref["logits"].double()
+    rms_b, max_b = logits_budget(cfg.n_layers, ref["logits"].double().std().item())
+    assert d.pow(2).mean().sqrt().item() <= rms_b and d.abs().max().item() <= max_b, (d.abs().max().item(), max_b)
+    for l in range(cfg.n_layers):
+        k, v = cache.gather(l)
+        assert rel_err(k, ref["K"][l]) <= KV_TOL and rel_err(v, ref["V"][l]) <= KV_TOL
+    logits2, cache2 = run_gpu(model, cfg, tokens, None, 1, page=16)
+    assert torch.equal(logits, logits2) and torch.equal(cache.k, cache2.k) and torch.equal(cache.v, cache2.v)
+
+
 @pytest.mark.parametrize("l_keep", [3, 1])
 def test_first_token_on_true_width_prompts(l_keep):
     # 16 seeded prompts at the Llama-3.1-8B layer shapes (3 layers, 256 tokens, vocabulary 32000): the
