@@ -26,12 +26,18 @@ constexpr int GROUP_M = 16;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int OUT_STAGE_BYTES = 32 * 32 * 4;
 
+// Operand ring of the single-CTA form: four stages of a 128 x 64 A block and a 256 x 64 B block, or, with
+// 128-column tiles, six stages with a 128 x 64 B block (small problems stream their weights and are bound by
+// how many k-blocks a CTA keeps in flight, not by the tensor pipe).
+template <int TN>
 struct __align__(1024) GemmSmem {
-  uint8_t a[STAGES][A_BYTES];
-  uint8_t b[STAGES][B_BYTES];
+  static constexpr int NST = TN == 128 ? 6 : STAGES;
+  static constexpr int TB_BYTES = TN * BK * 2;
+  uint8_t a[NST][A_BYTES];
+  uint8_t b[NST][TB_BYTES];
   uint8_t out_stage[4][2][OUT_STAGE_BYTES];   // per epilogue warp: two 32-row x 32-float boxes for TMA stores
-  uint64_t full[STAGES];
-  uint64_t empty[STAGES];
+  uint64_t full[NST];
+  uint64_t empty[NST];
   uint64_t tfull[2];
   uint64_t tempty[2];
   uint32_t tmem_base;
@@ -364,7 +370,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const __grid_constant__ CUtensorMap tmO, const GemmDev p,
             int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
-  GemmSmem& s = *reinterpret_cast<GemmSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using Smem = GemmSmem<TN>;
+  constexpr int NST = Smem::NST;
+  Smem& s = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
@@ -373,7 +381,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (status_raised(status, &s.raised)) return;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; ++i) {
+    for (int i = 0; i < NST; ++i) {
       mbar_init(&s.full[i], 1);
       mbar_init(&s.empty[i], 1);
     }
@@ -412,7 +420,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           mbar_expect_tx(&s.full[stage], A_BYTES + TN * BK * 2);
           tma_load_3d(s.a[stage], &tmA, &s.full[stage], kb * BKE, m * BM, g);
           tma_load_3d(s.b[stage], &tmB, &s.full[stage], kb * BKE, n * TN, g);
-          if (++stage == STAGES) {
+          if (++stage == NST) {
             stage = 0;
             phase ^= 1;
           }
@@ -449,7 +457,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tc_fence_after();
           // only the 16-byte-granular start address in the descriptor's low bits moves
           const uint64_t ad0 = a_desc0 + uint64_t(stage * (A_BYTES >> 4));
-          const uint64_t bd0 = b_desc0 + uint64_t(stage * (B_BYTES >> 4));
+          const uint64_t bd0 = b_desc0 + uint64_t(stage * (Smem::TB_BYTES >> 4));
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             if constexpr (FP8)
@@ -460,7 +468,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                              (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit_w(leader, &s.empty[stage]);
-          if (++stage == STAGES) {
+          if (++stage == NST) {
             stage = 0;
             phase ^= 1;
           }
@@ -771,18 +779,19 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     count_launch();
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? POP_OK : POP_E_CUDA;
   }
-  const size_t smem = sizeof(GemmSmem) + 1024;
+  const size_t smem = sizeof(GemmSmem<BN>) + 1024;
   if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_ADD_F32) {
     if (narrow) {
       static bool configured_narrow = false;
+      const size_t smem_n = sizeof(GemmSmem<128>) + 1024;
       if (!configured_narrow) {
         if (cudaFuncSetAttribute(gemm_kernel<EPI, HD, FP8, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem) != cudaSuccess)
+                                 (int)smem_n) != cudaSuccess)
           return POP_E_CUDA;
         configured_narrow = true;
       }
       ProfScope prof(PROF_GEMM, 2.0 * p.M * p.N * p.K * p.batch, stream);
-      gemm_kernel<EPI, HD, FP8, 128><<<grid, GEMM_THREADS, smem, stream>>>(ta, tb, to, p, status);
+      gemm_kernel<EPI, HD, FP8, 128><<<grid, GEMM_THREADS, smem_n, stream>>>(ta, tb, to, p, status);
       count_launch();
       return cudaGetLastError() == cudaSuccess ? POP_OK : POP_E_CUDA;
     }
