@@ -99,11 +99,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Epilogue of the fused QKV projection (paper Eq. 2-3; Eq. 14 for pruned layers): the thread owns one
-// token row of the 128 x 256 accumulator tile, which holds 256 / HD whole heads. q and k heads get
+// token row of the 128 x TN accumulator tile, which holds TN / HD whole heads (TN = 256, or 128 in the narrow form). q and k heads get
 // the optional per-head RMSNorm and RoPE (pair (j, j + HD/2), so two 32-column chunks of TMEM are
 // processed together), everything is rounded to bf16; q goes to its row buffer, k and v straight
 // into the token's slot of the paged cache. All tcgen05.ld are executed by every lane.
-template <int HD>
+template <int HD, int TN = BN>
 __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t taddr, int g, int n, int row,
                                                   bool row_ok, float rs) {
   const RopeEpi& r = p.rope;
@@ -139,8 +139,8 @@ __device__ __forceinline__ void qkv_rope_epilogue(const GemmDev& p, uint32_t tad
   }
   const float2* tab = r.table + (int64_t)pos * (HD / 2);
 #pragma unroll 1
-  for (int hh = 0; hh < 256 / HD; ++hh) {
-    const int head = n * (256 / HD) + hh;
+  for (int hh = 0; hh < TN / HD; ++hh) {
+    const int head = n * (TN / HD) + hh;
     if (head >= total_heads) break;                      // uniform: depends on the tile only
     const uint32_t haddr = taddr + hh * HD;
     const bool is_q = head < r.n_q;
@@ -245,7 +245,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, const CUtensorMa
   }
   if (FP8 && row_ok) rs = p.a_scale[row] * *p.b_scale;     // codes -> values: row scale x matrix scale
   if (EPI == EPI_QKV_ROPE) {
-    qkv_rope_epilogue<HD == 0 ? 64 : HD>(p, taddr, g, n, row, row_ok, rs);
+    qkv_rope_epilogue<HD == 0 ? 64 : HD, TN>(p, taddr, g, n, row, row_ok, rs);
   } else if (EPI == EPI_GATED_BF16) {
     bf16* out = reinterpret_cast<bf16*>(p.out) + int64_t(g) * p.out_batch_stride + int64_t(row) * p.ldo;
 #pragma unroll 1
@@ -780,7 +780,8 @@ int launch_epi(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? POP_OK : POP_E_CUDA;
   }
   const size_t smem = sizeof(GemmSmem<BN>) + 1024;
-  if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_ADD_F32) {
+  if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_ADD_F32 ||
+                (EPI == EPI_QKV_ROPE && HD >= 64 && HD <= 128)) {
     if (narrow) {
       static bool configured_narrow = false;
       const size_t smem_n = sizeof(GemmSmem<128>) + 1024;
@@ -820,7 +821,7 @@ int pair_group_m(int K) {
   return 16;
 }
 
-// Narrow single-CTA form: 128 x 128 tiles for the plain-store and residual epilogues when 128 x 256
+// Narrow single-CTA form: 128 x 128 tiles for the plain-store, residual and (head_dim <= 128) QKV epilogues when 128 x 256
 // tiles would leave at least half of the SMs without a tile (short prompts: the O and down projections of
 // 512 rows are 64 tiles). POP_GEMM_NARROW=0 / 1 forces it off / on wherever it is possible.
 bool use_narrow(bool possible, int64_t tiles, int sms) {
@@ -868,7 +869,8 @@ int launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   const bool pair = use_pair(a.M, tiles2, sms);
   const bool narrow = use_narrow(!pair && a.N > 128 && !a.hn_out && !a.ss_out &&
                                      (a.epilogue == EPI_STORE_BF16 || a.epilogue == EPI_STORE_F32 ||
-                                      a.epilogue == EPI_ADD_F32),
+                                      a.epilogue == EPI_ADD_F32 ||
+                                      (a.epilogue == EPI_QKV_ROPE && a.rope && a.rope->hd <= 128)),
                                  int64_t(ceil_div(a.M, BM)) * ceil_div(a.N, BN) * a.batch, sms);
   const uint32_t b_box = (pair || narrow) ? 128 : BN;   // a CTA of a pair loads its own half of the B block
   CUtensorMap ta, tb;
